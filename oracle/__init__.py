@@ -1,0 +1,200 @@
+"""numpy front end of the CPU oracle (``qbert_oracle.cpp``).
+
+TEST INFRASTRUCTURE ONLY: imported by ``tests/``, by the smoke check and by the
+CPU-baseline leg of ``bench.py``.  The CUDA library never imports this package
+and this package never imports the CUDA library.
+
+Two builds of the same source are kept side by side:
+
+* ``libqbert_oracle.so``      ``-O2 -ffp-contract=off``, single thread: the parity oracle.
+* ``libqbert_oracle_omp.so``  ``-O3 -ffp-contract=off -fopenmp``: the same loops on all host
+  cores, used only when the oracle is *timed* as the CPU baseline.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from pathlib import Path
+
+import numpy as np
+
+_HERE = Path(__file__).resolve().parent
+_SRC = _HERE / "qbert_oracle.cpp"
+_LIBS = {
+    False: (_HERE / "libqbert_oracle.so", ["-O2"]),
+    True: (_HERE / "libqbert_oracle_omp.so", ["-O3", "-fopenmp"]),
+}
+_loaded: dict[bool, ctypes.CDLL] = {}
+
+OK = 0
+ERR_INVALID = -1
+ERR_NONFINITE = -5
+
+
+def build(force: bool = False) -> None:
+    """Compile both builds of the oracle with g++ if missing or older than the source."""
+    for _omp, (lib, flags) in _LIBS.items():
+        if not force and lib.exists() and lib.stat().st_mtime >= _SRC.stat().st_mtime:
+            continue
+        cmd = ["g++", "-std=c++17", *flags, "-ffp-contract=off", "-fno-fast-math", "-fPIC", "-shared",
+               str(_SRC), "-o", str(lib) + ".tmp"]
+        subprocess.run(cmd, check=True)
+        os.replace(str(lib) + ".tmp", lib)
+
+
+def _lib(omp: bool = False) -> ctypes.CDLL:
+    if omp not in _loaded:
+        build()
+        lib = ctypes.CDLL(str(_LIBS[omp][0]))
+        i64, i32, vp, f32 = ctypes.c_int64, ctypes.c_int, ctypes.c_void_p, ctypes.c_float
+        lib.qo_num_threads.restype = i32
+        lib.qo_quantize_weights.argtypes = [vp, i64, i64, i32, i32, vp, vp, vp, vp, vp]
+        lib.qo_quantize_weights.restype = i32
+        lib.qo_dequantize_weights.argtypes = [vp, i64, i64, i32, vp, vp, vp]
+        lib.qo_dequantize_weights.restype = None
+        lib.qo_pack.argtypes = [vp, i64, i64, i32, vp]
+        lib.qo_pack.restype = i32
+        lib.qo_unpack.argtypes = [vp, i64, i64, i32, vp]
+        lib.qo_unpack.restype = i32
+        lib.qo_quantize_act.argtypes = [vp, i64, i64, vp, vp, vp]
+        lib.qo_quantize_act.restype = i32
+        lib.qo_int_gemm.argtypes = [vp, vp, i64, i64, i64, vp, vp]
+        lib.qo_int_gemm.restype = None
+        lib.qo_dequant_epilogue.argtypes = [vp, vp, f32, vp, vp, vp, i64, i64, i32, i32, vp]
+        lib.qo_dequant_epilogue.restype = None
+        lib.qo_linear_fp64.argtypes = [vp, f32, vp, vp, vp, vp, i64, i64, i64, i32, vp]
+        lib.qo_linear_fp64.restype = None
+        _loaded[omp] = lib
+    return _loaded[omp]
+
+
+def num_threads(omp: bool = False) -> int:
+    return int(_lib(omp).qo_num_threads())
+
+
+def _c(a: np.ndarray, dtype) -> np.ndarray:
+    a = np.ascontiguousarray(a, dtype=dtype)
+    return a
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def quantize_weights(w, bits: int, groups: int, range_lo=None, range_hi=None, omp: bool = False):
+    """Group-wise uniform quantizer Q (Section 3.3, Appendix A).
+
+    Returns ``(status, codes uint8 [N,K], delta f32 [G], q0 f32 [G])``.
+    """
+    w = _c(w, np.float32)
+    N, K = w.shape
+    codes = np.empty((N, K), np.uint8)
+    delta = np.empty(groups, np.float32)
+    q0 = np.empty(groups, np.float32)
+    lo = None if range_lo is None else _c(range_lo, np.float32)
+    hi = None if range_hi is None else _c(range_hi, np.float32)
+    st = _lib(omp).qo_quantize_weights(_p(w), N, K, bits, groups, _p(lo), _p(hi), _p(codes), _p(delta),
+                                       _p(q0))
+    return st, codes, delta, q0
+
+
+def dequantize_weights(codes, groups: int, delta, q0):
+    """Q(W) = Delta * X^I + q0 (Appendix A) as fp32 fused multiply-add."""
+    codes = _c(codes, np.uint8)
+    N, K = codes.shape
+    delta = _c(delta, np.float32)
+    q0 = _c(q0, np.float32)
+    out = np.empty((N, K), np.float32)
+    _lib().qo_dequantize_weights(_p(codes), N, K, groups, _p(delta), _p(q0), _p(out))
+    return out
+
+
+def pack(codes, bits: int):
+    """Dense little-endian k-bit packing: uint32 [N, K*bits/32]."""
+    codes = _c(codes, np.uint8)
+    N, K = codes.shape
+    if (K * bits) % 32:
+        raise ValueError("K*bits must be a multiple of 32")
+    words = np.empty((N, K * bits // 32), np.uint32)
+    st = _lib().qo_pack(_p(codes), N, K, bits, _p(words))
+    if st != OK:
+        raise ValueError(f"qo_pack status {st}")
+    return words
+
+
+def unpack(words, K: int, bits: int):
+    words = _c(words, np.uint32)
+    N = words.shape[0]
+    codes = np.empty((N, K), np.uint8)
+    st = _lib().qo_unpack(_p(words), N, K, bits, _p(codes))
+    if st != OK:
+        raise ValueError(f"qo_unpack status {st}")
+    return codes
+
+
+def quantize_act(x, omp: bool = False):
+    """Per-tensor 8-bit activation quantizer: ``(status, xq int8 [M,K], scale f32, rowsum i32 [M])``."""
+    x = _c(x, np.float32)
+    M, K = x.shape
+    xq = np.empty((M, K), np.int8)
+    scale = np.empty(1, np.float32)
+    rowsum = np.empty(M, np.int32)
+    st = _lib(omp).qo_quantize_act(_p(x), M, K, _p(xq), _p(scale), _p(rowsum))
+    return st, xq, np.float32(scale[0]), rowsum
+
+
+def int_gemm(xq, codes, want64: bool = False, omp: bool = False):
+    """acc[m,n] = sum_k xq[m,k] * u[n,k] in int32 (and int64 when ``want64``)."""
+    xq = _c(xq, np.int8)
+    codes = _c(codes, np.uint8)
+    M, K = xq.shape
+    N, K2 = codes.shape
+    assert K == K2
+    acc = np.empty((M, N), np.int32)
+    acc64 = np.empty((M, N), np.int64) if want64 else None
+    _lib(omp).qo_int_gemm(_p(xq), _p(codes), M, N, K, _p(acc), _p(acc64))
+    return (acc, acc64) if want64 else acc
+
+
+def dequant_epilogue(acc, rowsum, act_scale, delta, q0, bias, bits: int, groups: int, omp: bool = False):
+    """fp32 'gathered dequantization' of the int32 accumulators (Appendix A)."""
+    acc = _c(acc, np.int32)
+    rowsum = _c(rowsum, np.int32)
+    delta = _c(delta, np.float32)
+    q0 = _c(q0, np.float32)
+    b = None if bias is None else _c(bias, np.float32)
+    M, N = acc.shape
+    y = np.empty((M, N), np.float32)
+    _lib(omp).qo_dequant_epilogue(_p(acc), _p(rowsum), float(act_scale), _p(delta), _p(q0), _p(b), M, N,
+                                  bits, groups, _p(y))
+    return y
+
+
+def linear_fp64(xq, act_scale, codes, delta, q0, bias, groups: int, omp: bool = False):
+    """The quantized linear layer from the definitions, accumulated in double precision."""
+    xq = _c(xq, np.int8)
+    codes = _c(codes, np.uint8)
+    delta = _c(delta, np.float32)
+    q0 = _c(q0, np.float32)
+    b = None if bias is None else _c(bias, np.float32)
+    M, K = xq.shape
+    N = codes.shape[0]
+    y = np.empty((M, N), np.float64)
+    _lib(omp).qo_linear_fp64(_p(xq), float(act_scale), _p(codes), _p(delta), _p(q0), _p(b), M, N, K, groups,
+                             _p(y))
+    return y
+
+
+def linear(x, w, bias, bits: int, groups: int, omp: bool = False):
+    """Whole path on the CPU: quantize activations and weights, pack, integer GEMM, epilogue.
+
+    Returns a dict with every intermediate the parity tests compare.
+    """
+    st_a, xq, s_a, rowsum = quantize_act(x, omp=omp)
+    st_w, codes, delta, q0 = quantize_weights(w, bits, groups, omp=omp)
+    words = pack(codes, bits)
+    acc = int_gemm(xq, codes, omp=omp)
+    y = dequant_epilogue(acc, rowsum, s_a, delta, q0, bias, bits, groups, omp=omp)
+    return dict(status_act=st_a, status_w=st_w, xq=xq, act_scale=s_a, rowsum=rowsum, codes=codes,
+                delta=delta, q0=q0, words=words, acc=acc, y=y)
