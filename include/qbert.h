@@ -1,0 +1,163 @@
+/*
+ * libqbert — group-wise k-bit quantized transformer linear layers on NVIDIA B200 (sm_100a).
+ *
+ * The library implements the inference path of Q-BERT ("Hessian Based Ultra Low Precision
+ * Quantization of BERT"): weights quantized by the paper's uniform quantizer Q with one range
+ * per group of output neurons, 8-bit activations, an integer matrix product on the integer
+ * codes and one dequantization at the end.
+ *
+ * Conventions shared by every entry point
+ * ---------------------------------------
+ *  - Pure C ABI.  Pointers marked "dev" are CUDA device pointers on the current device, pointers
+ *    marked "host" are ordinary host pointers.  The caller owns every buffer; the library keeps no
+ *    pointer after a call returns and allocates no device memory.
+ *  - All device work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = the
+ *    legacy default stream) and is asynchronous with respect to the host.
+ *  - Argument errors are detected on the host, before anything is launched, and returned as a
+ *    negative qb_status.  Conditions only the device can see (a non-finite input, a bounded wait
+ *    that expired) are recorded in the status word at the head of the workspace `ws` (first error
+ *    wins, it is never cleared by a kernel) and read back with qb_read_status.  After such a
+ *    condition the outputs of that call are unspecified, but every write stays in bounds.
+ *  - Matrices are row-major.  X is [M][K] (tokens x input features), W is [N][K] (output neurons x
+ *    input features, the orientation of W in y = W x of Section 3.3), Y is [M][N].
+ *  - bits (k) is one of 2, 3, 4, 8.  `groups` (G) splits the N rows of W into G blocks of
+ *    R = N / G consecutive rows; N % G must be 0.  K must be a multiple of 128.
+ *  - There is no CPU fallback: on a device that is not sm_100 every compute call returns
+ *    QB_ERR_CUDA.
+ */
+#ifndef QBERT_H_
+#define QBERT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t qb_status;
+
+enum {
+  QB_OK = 0,
+  QB_ERR_INVALID = -1,   /* null pointer, bits not in {2,3,4,8}, G < 1, N % G != 0, size <= 0 or too large */
+  QB_ERR_ALIGN = -2,     /* pointer not 16-byte aligned, or K not a multiple of 128 */
+  QB_ERR_WORKSPACE = -3, /* workspace pointer null or smaller than qb_workspace_bytes() */
+  QB_ERR_CUDA = -4,      /* CUDA runtime / driver error or unsupported device; text in qb_last_error() */
+  QB_ERR_NONFINITE = -5, /* status word only: NaN or Inf met while reducing a range */
+  QB_ERR_TIMEOUT = -6    /* status word only: a bounded device-side wait expired */
+};
+
+/* Largest sizes accepted (int32 accumulators stay exact: 127 * 255 * K < 2^31). */
+#define QB_MAX_K 65536
+#define QB_MAX_MN (1 << 24)
+
+int qb_version(void);
+const char* qb_status_string(qb_status s);
+/* Text of the last error raised on the calling thread ("" if none).  Host pointer, valid until the
+ * next failing call on this thread. */
+const char* qb_last_error(void);
+
+/* Number of 32-bit words of the packed form of an [N][K] matrix at `bits` bits per weight:
+ * N * K * bits / 32 (Table 1 counts exactly k bits per weight).  0 on invalid arguments. */
+size_t qb_packed_words(int64_t N, int64_t K, int bits);
+
+/* Bytes of workspace any call on a problem of this size needs (>= 256).  Pass 0 for dimensions a
+ * call does not have.  The workspace is device memory owned by the caller; one workspace may serve
+ * consecutive calls on one stream.  It must be zeroed once with qb_workspace_init before first use. */
+size_t qb_workspace_bytes(int64_t M, int64_t N, int64_t K, int bits, int groups);
+
+/* Zero the workspace (status word included) on the stream. */
+qb_status qb_workspace_init(void* ws /*dev*/, size_t ws_bytes, void* cuda_stream);
+
+/* Synchronize the stream and return the status word of the workspace: QB_OK, QB_ERR_NONFINITE or
+ * QB_ERR_TIMEOUT (or QB_ERR_CUDA if the copy itself failed). */
+qb_status qb_read_status(const void* ws /*dev*/, void* cuda_stream);
+
+/*
+ * 8-bit activation quantizer (Table 1 caption: every quantized model uses 8-bit activations).
+ * The paper gives no further detail; this is Appendix A's uniform quantizer on the symmetric
+ * per-tensor range [-a, a], a = max|x|, with 255 points and the codes shifted to [-127, 127]:
+ *     act_scale = a / 127,   xq = clamp(round_half_even(x * (127 / a)), -127, 127),
+ *     rowsum[m] = sum_k xq[m][k].
+ * An all-zero tensor gives act_scale = 1 and zero codes.
+ *   x         dev, fp32 [M][K], 16-byte aligned          (read)
+ *   xq        dev, int8 [M][K], 16-byte aligned          (written)
+ *   act_scale dev, fp32 [1]                              (written)
+ *   rowsum    dev, int32 [M]                             (written)
+ * Two kernels: a grid-wide max-abs reduction into the workspace, then round/clamp/store.
+ */
+qb_status qb_quantize_act(const float* x, int64_t M, int64_t K, int8_t* xq, float* act_scale,
+                          int32_t* rowsum, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Group-wise weight quantizer and packer (Section 3.3 group-wise quantization; Appendix A):
+ * for each group g of R = N / G consecutive rows, q0 = min, qmax = max over the group,
+ *     Delta = (qmax - q0) / (2^k - 1),
+ *     code  = clamp(round_half_even((clamp(w, q0, qmax) - q0) * (1 / Delta)), 0, 2^k - 1).
+ * A constant group gets Delta = 1 and zero codes.  Codes are packed densely: row n is a
+ * little-endian bit stream with code j in bits [k*j, k*j + k), stored as K*k/32 uint32 words.
+ * G = 1 is the paper's layer-wise ("DirectQ") setting, G = N one range per output neuron.
+ *   w        dev, fp32 [N][K], 16-byte aligned           (read)
+ *   packed   dev, uint32 [N][K*bits/32], 16-byte aligned (written)
+ *   delta,q0 dev, fp32 [G]                               (written)
+ *   range_lo, range_hi: dev fp32 [G] or both NULL.  When given they replace the group's min and
+ *            max (Appendix A: the range "can be a subinterval of [min, max]"); values outside are
+ *            clamped.  They must be finite with range_lo <= range_hi.
+ * Two kernels: per-group min/max reduction into the workspace, then round/clamp/pack.
+ */
+qb_status qb_quantize_pack_weights(const float* w, int64_t N, int64_t K, int bits, int groups,
+                                   const float* range_lo, const float* range_hi, uint32_t* packed,
+                                   float* delta, float* q0, void* ws, size_t ws_bytes,
+                                   void* cuda_stream);
+
+/*
+ * Quantized linear layer (Appendix A: "integer arithmetic for the matrix multiplication with X^I,
+ * and then followed by a gathered dequantization operation").
+ *     acc[m][n] = sum_k xq[m][k] * code[n][k]                       (int32, exact)
+ *     y[m][n]   = act_scale * (Delta_g * acc + q0_g * rowsum[m]) + bias[n],   g = n / R
+ * The dequantization is evaluated in fp32 about the centre code c = 2^(k-1):
+ *     Ac = acc - c * rowsum[m];  zc = fma(Delta_g, c, q0_g);  alpha = act_scale * Delta_g;
+ *     beta = act_scale * zc;     y = fma(alpha, (float)Ac, fma(beta, (float)rowsum[m], bias[n])).
+ * Packed codes are expanded to 8 bits in shared memory (Section 4: low-bit values are loaded and
+ * cast to 8 bits in the execution units) and multiplied on the tensor cores.
+ *   xq, act_scale, rowsum: dev, as written by qb_quantize_act         (read)
+ *   packed, delta, q0:     dev, as written by qb_quantize_pack_weights (read)
+ *   bias     dev fp32 [N] or NULL                                     (read)
+ *   y        dev fp32 [M][N]                                          (written)
+ *   acc_out  dev int32 [M][N] or NULL: the accumulators acc[m][n]     (written)
+ * xq and packed must be 16-byte aligned.
+ */
+qb_status qb_gemm(const int8_t* xq, const float* act_scale, const int32_t* rowsum,
+                  const uint32_t* packed, const float* delta, const float* q0, const float* bias,
+                  int64_t M, int64_t N, int64_t K, int bits, int groups, float* y, int32_t* acc_out,
+                  void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* One linear of a stack: the arguments of qb_gemm. */
+typedef struct {
+  const int8_t* xq;
+  const float* act_scale;
+  const int32_t* rowsum;
+  const uint32_t* packed;
+  const float* delta;
+  const float* q0;
+  const float* bias; /* may be NULL */
+  int64_t M, N, K;
+  int32_t bits, groups;
+  float* y;
+} qb_linear_desc;
+
+/*
+ * Encoder-layer linear stack with per-layer bit widths (the appendix tables "Bits setting for
+ * 2/3-bit / 2/4-bit Q-BERT MP" give one weight bit width per encoder layer; the Hessian-based
+ * assignment that produces them is an input here).  `descs` is a HOST array of `count`
+ * descriptors, e.g. four per encoder layer in the order QKV, attention output, FFN1, FFN2; each is
+ * an independent problem with its own input, and the result of each equals qb_gemm on the same
+ * arguments bit for bit.  All descriptors are validated before anything is launched.
+ */
+qb_status qb_layer_linears(const qb_linear_desc* descs /*host*/, int32_t count, void* ws,
+                           size_t ws_bytes, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QBERT_H_ */

@@ -1,0 +1,207 @@
+"""Python binding of libqbert: argument marshalling only.
+
+Every step of the path (activation quantizer, group-wise weight quantizer and packer, integer
+GEMM with dequantizing epilogue, encoder-layer linear stack) runs in the CUDA kernels behind the C
+ABI declared in ``include/qbert.h``.  torch is used for device buffers and the current stream.
+There is no CPU fallback: if ``libqbert.so`` has not been built, importing works but the first call
+raises ``QbertError``.
+"""
+from __future__ import annotations
+
+import ctypes
+from dataclasses import dataclass
+from pathlib import Path
+from typing import Optional, Sequence
+
+import torch
+
+_PKG = Path(__file__).resolve().parent
+LIB_PATH = _PKG / "libqbert.so"
+
+QB_OK = 0
+QB_ERR_INVALID = -1
+QB_ERR_ALIGN = -2
+QB_ERR_WORKSPACE = -3
+QB_ERR_CUDA = -4
+QB_ERR_NONFINITE = -5
+QB_ERR_TIMEOUT = -6
+
+EXPORTS = (
+    "qb_version", "qb_status_string", "qb_last_error", "qb_packed_words", "qb_workspace_bytes",
+    "qb_workspace_init", "qb_read_status", "qb_quantize_act", "qb_quantize_pack_weights", "qb_gemm",
+    "qb_layer_linears",
+)
+
+
+class QbertError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"{message} (status {status})")
+        self.status = status
+
+
+class LinearDescC(ctypes.Structure):
+    """Mirror of ``qb_linear_desc``."""
+    _fields_ = [
+        ("xq", ctypes.c_void_p), ("act_scale", ctypes.c_void_p), ("rowsum", ctypes.c_void_p),
+        ("packed", ctypes.c_void_p), ("delta", ctypes.c_void_p), ("q0", ctypes.c_void_p),
+        ("bias", ctypes.c_void_p),
+        ("M", ctypes.c_int64), ("N", ctypes.c_int64), ("K", ctypes.c_int64),
+        ("bits", ctypes.c_int32), ("groups", ctypes.c_int32),
+        ("y", ctypes.c_void_p),
+    ]
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load ``libqbert.so`` (built in-tree by ``paper_1909_05840_b200.build``)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not LIB_PATH.exists():
+        raise QbertError(QB_ERR_CUDA, f"{LIB_PATH} is missing: build it with "
+                                      "`python -m paper_1909_05840_b200.build`; there is no CPU fallback")
+    L = ctypes.CDLL(str(LIB_PATH))
+    i64, i32, vp, sz = ctypes.c_int64, ctypes.c_int32, ctypes.c_void_p, ctypes.c_size_t
+    L.qb_version.restype = ctypes.c_int
+    L.qb_status_string.argtypes = [i32]
+    L.qb_status_string.restype = ctypes.c_char_p
+    L.qb_last_error.restype = ctypes.c_char_p
+    L.qb_packed_words.argtypes = [i64, i64, ctypes.c_int]
+    L.qb_packed_words.restype = sz
+    L.qb_workspace_bytes.argtypes = [i64, i64, i64, ctypes.c_int, ctypes.c_int]
+    L.qb_workspace_bytes.restype = sz
+    L.qb_workspace_init.argtypes = [vp, sz, vp]
+    L.qb_workspace_init.restype = i32
+    L.qb_read_status.argtypes = [vp, vp]
+    L.qb_read_status.restype = i32
+    L.qb_quantize_act.argtypes = [vp, i64, i64, vp, vp, vp, vp, sz, vp]
+    L.qb_quantize_act.restype = i32
+    L.qb_quantize_pack_weights.argtypes = [vp, i64, i64, ctypes.c_int, ctypes.c_int, vp, vp, vp, vp, vp, vp, sz, vp]
+    L.qb_quantize_pack_weights.restype = i32
+    L.qb_gemm.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, ctypes.c_int, ctypes.c_int, vp, vp, vp, sz, vp]
+    L.qb_gemm.restype = i32
+    L.qb_layer_linears.argtypes = [ctypes.POINTER(LinearDescC), i32, vp, sz, vp]
+    L.qb_layer_linears.restype = i32
+    _lib = L
+    return L
+
+
+def _check(status: int, what: str) -> None:
+    if status != QB_OK:
+        L = lib()
+        name = L.qb_status_string(status).decode()
+        raise QbertError(status, f"{what}: {name}: {L.qb_last_error().decode()}")
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def version() -> int:
+    return int(lib().qb_version())
+
+
+def packed_words(N: int, K: int, bits: int) -> int:
+    return int(lib().qb_packed_words(N, K, bits))
+
+
+def workspace_bytes(M: int = 0, N: int = 0, K: int = 0, bits: int = 0, groups: int = 0) -> int:
+    return int(lib().qb_workspace_bytes(M, N, K, bits, groups))
+
+
+def workspace(groups: int = 4096, device="cuda") -> torch.Tensor:
+    """A zero-initialised workspace large enough for any call with up to ``groups`` groups."""
+    ws = torch.empty(workspace_bytes(groups=groups), dtype=torch.uint8, device=device)
+    _check(lib().qb_workspace_init(ws.data_ptr(), ws.numel(), _stream()), "qb_workspace_init")
+    return ws
+
+
+def read_status(ws: torch.Tensor) -> int:
+    """Synchronise the current stream and return the workspace's status word."""
+    return int(lib().qb_read_status(ws.data_ptr(), _stream()))
+
+
+def quantize_act(x: torch.Tensor, ws: torch.Tensor, xq: Optional[torch.Tensor] = None,
+                 act_scale: Optional[torch.Tensor] = None, rowsum: Optional[torch.Tensor] = None):
+    """``qb_quantize_act``: fp32 [M,K] -> (int8 codes [M,K], fp32 scale [1], int32 row sums [M])."""
+    assert x.is_cuda and x.dtype == torch.float32 and x.dim() == 2 and x.is_contiguous()
+    M, K = x.shape
+    xq = torch.empty((M, K), dtype=torch.int8, device=x.device) if xq is None else xq
+    act_scale = torch.empty(1, dtype=torch.float32, device=x.device) if act_scale is None else act_scale
+    rowsum = torch.empty(M, dtype=torch.int32, device=x.device) if rowsum is None else rowsum
+    _check(lib().qb_quantize_act(x.data_ptr(), M, K, xq.data_ptr(), act_scale.data_ptr(), rowsum.data_ptr(),
+                                 ws.data_ptr(), ws.numel(), _stream()), "qb_quantize_act")
+    return xq, act_scale, rowsum
+
+
+def quantize_pack_weights(w: torch.Tensor, bits: int, groups: int, ws: torch.Tensor,
+                          range_lo: Optional[torch.Tensor] = None, range_hi: Optional[torch.Tensor] = None,
+                          packed: Optional[torch.Tensor] = None, delta: Optional[torch.Tensor] = None,
+                          q0: Optional[torch.Tensor] = None):
+    """``qb_quantize_pack_weights``: fp32 [N,K] -> (int32-viewed packed words [N, K*bits/32], delta [G], q0 [G])."""
+    assert w.is_cuda and w.dtype == torch.float32 and w.dim() == 2 and w.is_contiguous()
+    N, K = w.shape
+    if packed is None:
+        words_per_row = max(1, K * bits // 32)
+        packed = torch.empty((N, words_per_row), dtype=torch.int32, device=w.device)
+    delta = torch.empty(max(groups, 1), dtype=torch.float32, device=w.device) if delta is None else delta
+    q0 = torch.empty(max(groups, 1), dtype=torch.float32, device=w.device) if q0 is None else q0
+    _check(lib().qb_quantize_pack_weights(w.data_ptr(), N, K, bits, groups, _ptr(range_lo), _ptr(range_hi),
+                                          packed.data_ptr(), delta.data_ptr(), q0.data_ptr(), ws.data_ptr(),
+                                          ws.numel(), _stream()), "qb_quantize_pack_weights")
+    return packed, delta, q0
+
+
+def gemm(xq: torch.Tensor, act_scale: torch.Tensor, rowsum: torch.Tensor, packed: torch.Tensor,
+         delta: torch.Tensor, q0: torch.Tensor, bias: Optional[torch.Tensor], N: int, bits: int, groups: int,
+         ws: torch.Tensor, y: Optional[torch.Tensor] = None, acc_out: Optional[torch.Tensor] = None,
+         want_acc: bool = False):
+    """``qb_gemm``: returns ``y`` fp32 [M,N] (and the int32 accumulators when ``want_acc``)."""
+    assert xq.is_cuda and xq.dtype == torch.int8 and xq.is_contiguous()
+    M, K = xq.shape
+    y = torch.empty((M, N), dtype=torch.float32, device=xq.device) if y is None else y
+    if want_acc and acc_out is None:
+        acc_out = torch.empty((M, N), dtype=torch.int32, device=xq.device)
+    _check(lib().qb_gemm(xq.data_ptr(), act_scale.data_ptr(), rowsum.data_ptr(), packed.data_ptr(),
+                         delta.data_ptr(), q0.data_ptr(), _ptr(bias), M, N, K, bits, groups, y.data_ptr(),
+                         _ptr(acc_out), ws.data_ptr(), ws.numel(), _stream()), "qb_gemm")
+    return (y, acc_out) if (want_acc or acc_out is not None) else y
+
+
+@dataclass
+class LinearDesc:
+    """One linear of a stack: tensors as produced by ``quantize_act`` / ``quantize_pack_weights``."""
+    xq: torch.Tensor
+    act_scale: torch.Tensor
+    rowsum: torch.Tensor
+    packed: torch.Tensor
+    delta: torch.Tensor
+    q0: torch.Tensor
+    bias: Optional[torch.Tensor]
+    N: int
+    bits: int
+    groups: int
+    y: torch.Tensor
+
+
+def make_desc_array(descs: Sequence[LinearDesc]):
+    """Marshal descriptors into a C array once; reuse it across calls on the same buffers."""
+    arr = (LinearDescC * len(descs))()
+    for i, d in enumerate(descs):
+        M, K = d.xq.shape
+        arr[i] = LinearDescC(d.xq.data_ptr(), d.act_scale.data_ptr(), d.rowsum.data_ptr(), d.packed.data_ptr(),
+                             d.delta.data_ptr(), d.q0.data_ptr(), _ptr(d.bias), M, d.N, K, d.bits, d.groups,
+                             d.y.data_ptr())
+    return arr
+
+
+def layer_linears(descs, ws: torch.Tensor) -> None:
+    """``qb_layer_linears`` over a list of ``LinearDesc`` (or an array from ``make_desc_array``)."""
+    arr = descs if isinstance(descs, ctypes.Array) else make_desc_array(descs)
+    _check(lib().qb_layer_linears(arr, len(arr), ws.data_ptr(), ws.numel(), _stream()), "qb_layer_linears")

@@ -1,0 +1,67 @@
+// Shared host/device helpers of libqbert: workspace layout, status word, error text.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "qbert.h"
+
+namespace qb {
+
+// ---- workspace layout (device memory owned by the caller) ------------------------------------
+// [0]   int32  status   first device-side error, never cleared by a kernel
+// [4]   int32  detail   where a bounded wait gave up (role << 16 | stage), diagnostics only
+// [16]  uint32 act_absmax_bits   bit pattern of max|x| of the last qb_quantize_act
+// [256] uint32 range_hi_enc[G], uint32 range_lo_inv[G]   ordered encodings of per-group max / min
+constexpr size_t kWsStatusOff = 0;
+constexpr size_t kWsDetailOff = 4;
+constexpr size_t kWsActMaxOff = 16;
+constexpr size_t kWsRangeOff = 256;
+constexpr size_t kWsMinBytes = 256;
+
+struct WsHeader {
+  int32_t status;
+  int32_t detail;
+  uint32_t pad[2];
+  uint32_t act_absmax_bits;
+};
+
+inline size_t ws_bytes_needed(int groups) {
+  size_t b = kWsRangeOff + (groups > 0 ? size_t(groups) * 8 : 0);
+  return (b + 255) / 256 * 256;
+}
+
+// ---- host-side error plumbing ------------------------------------------------------------------
+void set_last_error(const char* fmt, ...);
+qb_status cuda_fail(cudaError_t e, const char* what);
+// QB_OK if the current device is sm_100; caches the answer and the SM count per device.
+qb_status require_sm100(int* sm_count);
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool valid_bits(int b) { return b == 2 || b == 3 || b == 4 || b == 8; }
+
+#define QB_CUDA_TRY(expr)                                   \
+  do {                                                      \
+    cudaError_t e__ = (expr);                               \
+    if (e__ != cudaSuccess) return qb::cuda_fail(e__, #expr); \
+  } while (0)
+
+// ---- device-side helpers -----------------------------------------------------------------------
+#ifdef __CUDACC__
+__device__ __forceinline__ void report_status(void* ws, int32_t code, int32_t detail = 0) {
+  WsHeader* h = reinterpret_cast<WsHeader*>(ws);
+  if (atomicCAS(&h->status, 0, code) == 0) h->detail = detail;
+}
+
+// Monotone map from float bit patterns to unsigned integers (so that integer atomicMax orders floats).
+__device__ __forceinline__ uint32_t float_to_ordered(float f) {
+  uint32_t b = __float_as_uint(f);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float ordered_to_float(uint32_t e) {
+  uint32_t b = (e & 0x80000000u) ? (e & 0x7fffffffu) : ~e;
+  return __uint_as_float(b);
+}
+#endif
+
+}  // namespace qb

@@ -1,0 +1,559 @@
+// qb_gemm: integer matrix product on the quantization codes followed by one dequantization
+// (Appendix A), for weights stored at k in {2,3,4,8} bits per code.
+//
+// Orientation.  The tensor-core product is computed transposed, D[n][m] = sum_k Wc[n][k] * xq[m][k]:
+//   * the 128 rows of the MMA's A operand are 128 output neurons (weight rows), expanded from the
+//     packed k-bit words to signed 8-bit values in shared memory (Section 4: low-bit values are
+//     loaded and cast to 8 bits for execution);
+//   * the MMA's B operand is a tile of BT tokens (128 or 256) of the int8 activations, staged by TMA;
+//   * the int32 accumulator tile lives in tensor memory: TMEM lane = output neuron, column = token.
+// With this orientation the per-neuron dequantization constants are per-thread registers in the
+// epilogue and, for a fixed token, the 32 lanes of a warp hold 32 consecutive outputs of one row of
+// Y, so every store instruction writes one full 128-byte line.
+//
+// Codes are fed to the MMA recentred and pre-scaled, v = (code - 2^(k-1)) << (8-k), as s8.  The
+// shift makes the expansion a mask and an xor per word; the epilogue shifts the exact int32 sum
+// back.  |sum| <= 127 * 128 * K < 2^31 for K <= 65536.
+//
+// One persistent CTA per SM, ten warps:
+//   warp 0        TMA producer for the token tiles               (one lane)
+//   warp 1        tcgen05.mma issuer, owns the TMEM allocation   (one lane)
+//   warps 2..5    weight expanders: thread r owns weight row r of the tile
+//   warps 6..9    epilogue: TMEM -> registers -> fp32 -> global
+// Shared-memory ring of STAGES stages (16 KB weights + BT*128 B tokens each, 128-byte swizzle, K
+// block of 128), two accumulator tiles in TMEM so the epilogue of tile i overlaps the MMAs of tile
+// i+1.  Every wait is bounded: on expiry the CTA records QB_ERR_TIMEOUT and leaves through the
+// normal exit path (TMEM freed).
+#include <cuda.h>
+
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace qb {
+
+constexpr int kGemmThreads = 320;
+constexpr int kTileN = 128;          // output neurons per tile (MMA M)
+constexpr int kBlockK = 128;         // K elements (= bytes) per pipeline stage
+constexpr int kWBytes = kTileN * kBlockK;
+constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
+
+struct GemmParams {
+  const float* act_scale;
+  const int32_t* rowsum;
+  const uint32_t* packed;
+  const float* delta;
+  const float* q0;
+  const float* bias;
+  float* y;
+  int32_t* acc_out;
+  void* ws;
+  int32_t M, N, K;
+  int32_t rows_per_group;
+  int32_t n_tiles, m_tiles;
+};
+
+template <int BT>
+struct GemmCfg {
+  static constexpr int kXBytes = BT * kBlockK;
+  static constexpr int kStageBytes = kWBytes + kXBytes;
+  static constexpr int kStages = (BT == 256) ? 4 : 6;
+  static constexpr int kTmemCols = 2 * BT;
+  static constexpr int kBarBytes = 256;
+  static constexpr int kSmemBytes = kStages * kStageBytes + kBarBytes + 1024;  // + alignment slack
+};
+
+// Bounded wait on an mbarrier phase.  Returns false if the wait expired or another role aborted.
+__device__ __forceinline__ bool wait_barrier(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (ptx::mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = ptx::globaltimer_ns();
+  for (uint32_t spin = 1;; ++spin) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    if ((spin & 63u) == 0u) {
+      if (*abort_flag) return false;
+      if (ptx::globaltimer_ns() - t0 > kWaitLimitNs) return false;
+    }
+  }
+}
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes, groups of
+// 8 rows 1024 bytes apart.  Fields: start address >> 4 (bits 0-13), leading byte offset >> 4 (16-29,
+// unused for swizzled K-major, set to 1), stride byte offset >> 4 (32-45), descriptor version 1
+// (bits 46-47), layout type 2 = SWIZZLE_128B (bits 61-63).
+__device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)1 << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+
+// Instruction descriptor for kind::i8: D = s32 (bits 4-5 = 2), A = s8 (bits 7-9 = 1), B = s8
+// (bits 10-12 = 1), both operands K-major (bits 15, 16 = 0), N >> 3 in bits 17-22, M >> 4 in 24-28.
+__host__ __device__ constexpr uint32_t make_idesc_i8(int mma_m, int mma_n) {
+  return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(mma_n >> 3) << 17) | ((uint32_t)(mma_m >> 4) << 24);
+}
+
+// Expand the 128 codes of one weight row and one K block (BITS 16-byte words) to 128 signed bytes
+// v = (code - 2^(BITS-1)) << (8-BITS), returned as 32 words (word j = codes 4j..4j+3).
+template <int BITS>
+__device__ __forceinline__ void expand_codes(const uint32_t (&in)[4 * BITS], uint32_t (&out)[32]) {
+  if constexpr (BITS == 8) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) out[i] = in[i] ^ 0x80808080u;
+  } else if constexpr (BITS == 4) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const uint32_t w = in[i];
+      const uint32_t even = ((w << 4) & 0xF0F0F0F0u) ^ 0x80808080u;  // codes 0,2,4,6 of this word
+      const uint32_t odd = (w & 0xF0F0F0F0u) ^ 0x80808080u;          // codes 1,3,5,7
+      out[2 * i] = __byte_perm(even, odd, 0x5140);                    // codes 0,1,2,3
+      out[2 * i + 1] = __byte_perm(even, odd, 0x7362);                // codes 4,5,6,7
+    }
+  } else if constexpr (BITS == 2) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const uint32_t w = in[i];
+      const uint32_t t0 = ((w << 6) & 0xC0C0C0C0u) ^ 0x80808080u;  // codes 0,4,8,12
+      const uint32_t t1 = ((w << 4) & 0xC0C0C0C0u) ^ 0x80808080u;  // codes 1,5,9,13
+      const uint32_t t2 = ((w << 2) & 0xC0C0C0C0u) ^ 0x80808080u;  // codes 2,6,10,14
+      const uint32_t t3 = (w & 0xC0C0C0C0u) ^ 0x80808080u;         // codes 3,7,11,15
+      const uint32_t a_lo = __byte_perm(t0, t1, 0x5140);           // codes 0,1,4,5
+      const uint32_t b_lo = __byte_perm(t2, t3, 0x5140);           // codes 2,3,6,7
+      const uint32_t a_hi = __byte_perm(t0, t1, 0x7362);           // codes 8,9,12,13
+      const uint32_t b_hi = __byte_perm(t2, t3, 0x7362);           // codes 10,11,14,15
+      out[4 * i] = __byte_perm(a_lo, b_lo, 0x5410);                // codes 0..3
+      out[4 * i + 1] = __byte_perm(a_lo, b_lo, 0x7632);            // codes 4..7
+      out[4 * i + 2] = __byte_perm(a_hi, b_hi, 0x5410);            // codes 8..11
+      out[4 * i + 3] = __byte_perm(a_hi, b_hi, 0x7632);            // codes 12..15
+    }
+  } else {  // BITS == 3: 32 codes = 96 bits = 3 words; 4 codes = 12 bits per output word
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int bit = 12 * j;
+        const int wi = bit >> 5, sh = bit & 31;
+        uint32_t f;
+        if (sh + 12 > 32)
+          f = __funnelshift_r(in[3 * t + wi], in[3 * t + wi + 1], sh);
+        else
+          f = in[3 * t + wi] >> sh;
+        out[8 * t + j] = 0x80808080u ^ ((f << 5) & 0x000000E0u) ^ ((f << 10) & 0x0000E000u) ^
+                         ((f << 15) & 0x00E00000u) ^ ((f << 20) & 0xE0000000u);
+      }
+    }
+  }
+}
+
+template <int BT, int BITS>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+qb_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p) {
+  using Cfg = GemmCfg<BT>;
+  constexpr int kStages = Cfg::kStages;
+  extern __shared__ uint8_t smem_raw[];
+  // 128-byte swizzle patterns repeat every 1024 bytes: stage bases must be 1024-byte aligned
+  const uint32_t raw_addr = ptx::smem_u32(smem_raw);
+  uint8_t* smem = smem_raw + ((1024u - (raw_addr & 1023u)) & 1023u);
+  const uint32_t smem_base = ptx::smem_u32(smem);
+  const uint32_t bar_base = smem_base + kStages * Cfg::kStageBytes;
+  uint8_t* bar_ptr = smem + kStages * Cfg::kStageBytes;
+  auto full_x = [&](int s) { return bar_base + 8u * s; };
+  auto full_w = [&](int s) { return bar_base + 8u * (kStages + s); };
+  auto empty = [&](int s) { return bar_base + 8u * (2 * kStages + s); };
+  auto acc_full = [&](int a) { return bar_base + 8u * (3 * kStages + a); };
+  auto acc_empty = [&](int a) { return bar_base + 8u * (3 * kStages + 2 + a); };
+  const uint32_t drain_bar = bar_base + 8u * (3 * kStages + 4);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_ptr + 8 * (3 * kStages + 5));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  auto stage_w = [&](int s) { return smem_base + s * Cfg::kStageBytes; };
+  auto stage_x = [&](int s) { return smem_base + s * Cfg::kStageBytes + kWBytes; };
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      ptx::mbar_init(full_x(s), 1);
+      ptx::mbar_init(full_w(s), 128);
+      ptx::mbar_init(empty(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      ptx::mbar_init(acc_full(a), 1);
+      ptx::mbar_init(acc_empty(a), 128);
+    }
+    ptx::mbar_init(drain_bar, 1);
+    *abort_flag = 0;
+    ptx::fence_mbar_init();
+    ptx::prefetch_tensormap(&tmap_x);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(ptx::smem_u32(tmem_slot), Cfg::kTmemCols);
+    ptx::tmem_relinquish_alloc_permit();
+  }
+  ptx::tcgen05_fence_before_sync();
+  __syncthreads();
+  ptx::tcgen05_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int total_tiles = p.n_tiles * p.m_tiles;
+  const int k_blocks = p.K / kBlockK;
+  bool timed_out = false;
+  int where = 0;
+
+  if (warp == 0) {
+    // ---------------- TMA producer: token tiles -------------------------------------------------
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      for (int t = blockIdx.x; t < total_tiles && !timed_out; t += gridDim.x) {
+        const int m0 = (t / p.n_tiles) * BT;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!wait_barrier(empty(stage), phase ^ 1u, abort_flag)) {
+            timed_out = true;
+            where = (0 << 16) | stage;
+            break;
+          }
+          ptx::mbar_arrive_expect_tx(full_x(stage), Cfg::kXBytes);
+          ptx::tma_load_2d(stage_x(stage), &tmap_x, full_x(stage), kb * kBlockK, m0);
+          if (++stage == kStages) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+      }
+      if (timed_out) {
+        // let copies already in flight land before the CTA's shared memory is released
+        const uint64_t t0 = ptx::globaltimer_ns();
+        while (ptx::globaltimer_ns() - t0 < 200000ull) {
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------------------------------------------------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc_i8(kTileN, BT);
+      int stage = 0;
+      uint32_t phase = 0;
+      int it = 0;
+      for (int t = blockIdx.x; t < total_tiles && !timed_out; t += gridDim.x, ++it) {
+        const int a = it & 1;
+        const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
+        if (!wait_barrier(acc_empty(a), aphase ^ 1u, abort_flag)) {
+          timed_out = true;
+          where = (1 << 16) | 0x100 | a;
+          break;
+        }
+        ptx::tcgen05_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(a * BT);
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!wait_barrier(full_x(stage), phase, abort_flag) || !wait_barrier(full_w(stage), phase, abort_flag)) {
+            timed_out = true;
+            where = (1 << 16) | stage;
+            break;
+          }
+          ptx::tcgen05_fence_after_sync();
+          const uint64_t a_desc = make_kmajor_sw128_desc(stage_w(stage));
+          const uint64_t b_desc = make_kmajor_sw128_desc(stage_x(stage));
+#pragma unroll
+          for (int j = 0; j < kBlockK / 32; ++j)  // 32 bytes of K per instruction: +2 in the address field
+            ptx::mma_i8_ss(d_tmem, a_desc + 2u * j, b_desc + 2u * j, idesc, (kb | j) != 0 ? 1u : 0u);
+          ptx::mma_commit(empty(stage));
+          if (++stage == kStages) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+        if (timed_out) break;
+        ptx::mma_commit(acc_full(a));
+      }
+      if (timed_out) {
+        // wait (bounded) for the MMAs already issued before tensor memory is freed
+        ptx::mma_commit(drain_bar);
+        const uint64_t t0 = ptx::globaltimer_ns();
+        while (!ptx::mbar_try_wait(drain_bar, 0) && ptx::globaltimer_ns() - t0 < 200000000ull) {
+        }
+      }
+    }
+  } else if (warp < 6) {
+    // ---------------- weight expanders ------------------------------------------------------------
+    const int r = threadIdx.x - 64;  // weight row inside the tile
+    const int units_per_row = p.K / 128 * BITS;  // 16-byte words per packed row
+    int stage = 0;
+    uint32_t phase = 0;
+    for (int t = blockIdx.x; t < total_tiles && !timed_out; t += gridDim.x) {
+      const int n = (t % p.n_tiles) * kTileN + r;
+      const bool valid = n < p.N;
+      const uint4* src = reinterpret_cast<const uint4*>(p.packed) + (size_t)(valid ? n : 0) * units_per_row;
+      uint32_t cur[4 * BITS], nxt[4 * BITS];
+      auto load_block = [&](int kb, uint32_t (&dst)[4 * BITS]) {
+#pragma unroll
+        for (int i = 0; i < BITS; ++i) {
+          uint4 v = valid ? __ldg(src + (size_t)kb * BITS + i) : make_uint4(0, 0, 0, 0);
+          dst[4 * i] = v.x;
+          dst[4 * i + 1] = v.y;
+          dst[4 * i + 2] = v.z;
+          dst[4 * i + 3] = v.w;
+        }
+      };
+      load_block(0, nxt);
+      for (int kb = 0; kb < k_blocks; ++kb) {
+#pragma unroll
+        for (int i = 0; i < 4 * BITS; ++i) cur[i] = nxt[i];
+        if (kb + 1 < k_blocks) load_block(kb + 1, nxt);
+        uint32_t out[32];
+        expand_codes<BITS>(cur, out);
+        if (!valid) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) out[i] = 0u;
+        }
+        if (!wait_barrier(empty(stage), phase ^ 1u, abort_flag)) {
+          timed_out = true;
+          where = (2 << 16) | stage;
+          break;
+        }
+        uint8_t* row_ptr = smem + stage * Cfg::kStageBytes + r * 128;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          uint4 v = make_uint4(out[4 * c], out[4 * c + 1], out[4 * c + 2], out[4 * c + 3]);
+          *reinterpret_cast<uint4*>(row_ptr + ((c ^ (r & 7)) << 4)) = v;
+        }
+        ptx::fence_proxy_async_smem();
+        ptx::mbar_arrive(full_w(stage));
+        if (++stage == kStages) {
+          stage = 0;
+          phase ^= 1u;
+        }
+      }
+    }
+  } else {
+    // ---------------- epilogue --------------------------------------------------------------------
+    const int quarter = warp & 3;              // TMEM lanes this warp may access: 32*quarter ..
+    const int r = quarter * 32 + lane;         // output neuron inside the tile
+    const float s_a = __ldg(p.act_scale);
+    constexpr int c_code = 1 << (BITS - 1);
+    int it = 0;
+    for (int t = blockIdx.x; t < total_tiles && !timed_out; t += gridDim.x, ++it) {
+      const int a = it & 1;
+      const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
+      const int n = (t % p.n_tiles) * kTileN + r;
+      const int m0 = (t / p.n_tiles) * BT;
+      const bool nvalid = n < p.N;
+      float alpha = 0.f, beta = 0.f, b = 0.f;
+      if (nvalid) {
+        const int g = n / p.rows_per_group;
+        const float dlt = __ldg(p.delta + g);
+        const float z = __ldg(p.q0 + g);
+        const float zc = __fmaf_rn(dlt, (float)c_code, z);
+        alpha = __fmul_rn(s_a, dlt);
+        beta = __fmul_rn(s_a, zc);
+        b = p.bias ? __ldg(p.bias + n) : 0.0f;
+      }
+      if (!wait_barrier(acc_full(a), aphase, abort_flag)) {
+        timed_out = true;
+        where = (3 << 16) | a;
+        break;
+      }
+      ptx::tcgen05_fence_after_sync();
+      const uint32_t t_base = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * BT);
+#pragma unroll 1
+      for (int ch = 0; ch < BT / 32; ++ch) {
+        const int mc = m0 + ch * 32;
+        if (mc >= p.M) break;  // warp-uniform
+        uint32_t v[32];
+        ptx::tmem_ld_32x32b_x32(t_base + (uint32_t)(ch * 32), v);
+        ptx::tmem_ld_wait();
+        float* yrow = p.y + (size_t)mc * p.N + n;
+        int32_t* arow = p.acc_out ? p.acc_out + (size_t)mc * p.N + n : nullptr;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          if (mc + j < p.M) {
+            const int rs = __ldg(p.rowsum + mc + j);
+            const int ac = ((int)v[j]) >> (8 - BITS);
+            const float yv = __fmaf_rn(alpha, (float)ac, __fmaf_rn(beta, (float)rs, b));
+            if (nvalid) {
+              __stcs(yrow + (size_t)j * p.N, yv);
+              if (arow) arow[(size_t)j * p.N] = ac + c_code * rs;
+            }
+          }
+        }
+      }
+      ptx::tcgen05_fence_before_sync();
+      ptx::mbar_arrive(acc_empty(a));
+    }
+  }
+
+  if (timed_out) {
+    *abort_flag = 1;
+    report_status(p.ws, QB_ERR_TIMEOUT, where);
+  }
+  // ---------------- teardown ----------------------------------------------------------------------
+  ptx::tcgen05_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    ptx::tcgen05_fence_after_sync();
+    ptx::tmem_dealloc(tmem_base, Cfg::kTmemCols);
+  }
+}
+
+// ---- host side -----------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static qb_status get_encode_fn(EncodeTiledFn* out) {
+  static EncodeTiledFn cached = nullptr;
+  if (!cached) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    QB_CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+    if (qres != cudaDriverEntryPointSuccess || !fn) {
+      set_last_error("cuTensorMapEncodeTiled not available from the driver");
+      return QB_ERR_CUDA;
+    }
+    cached = reinterpret_cast<EncodeTiledFn>(fn);
+  }
+  *out = cached;
+  return QB_OK;
+}
+
+// int8 activations [M][K], K contiguous; box = 128 bytes of K x `box_rows` tokens, 128-byte swizzle.
+static qb_status make_x_tensormap(CUtensorMap* tm, const int8_t* xq, int64_t M, int64_t K, int box_rows) {
+  EncodeTiledFn encode = nullptr;
+  qb_status st = get_encode_fn(&encode);
+  if (st != QB_OK) return st;
+  const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
+  const cuuint64_t strides[1] = {(cuuint64_t)K};
+  const cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)box_rows};
+  const cuuint32_t elem[2] = {1, 1};
+  CUresult r = encode(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(xq), dims, strides, box, elem,
+                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    set_last_error("cuTensorMapEncodeTiled failed with CUresult %d (M=%lld K=%lld)", (int)r, (long long)M,
+                   (long long)K);
+    return QB_ERR_CUDA;
+  }
+  return QB_OK;
+}
+
+template <int BT, int BITS>
+static qb_status launch_gemm_inst(const CUtensorMap& tm, const GemmParams& p, int grid, cudaStream_t stream) {
+  using Cfg = GemmCfg<BT>;
+  auto kernel = qb_gemm_kernel<BT, BITS>;
+  QB_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
+  kernel<<<grid, kGemmThreads, Cfg::kSmemBytes, stream>>>(tm, p);
+  QB_CUDA_TRY(cudaGetLastError());
+  return QB_OK;
+}
+
+template <int BT>
+static qb_status launch_gemm_bits(int bits, const CUtensorMap& tm, const GemmParams& p, int grid,
+                                  cudaStream_t stream) {
+  switch (bits) {
+    case 2: return launch_gemm_inst<BT, 2>(tm, p, grid, stream);
+    case 3: return launch_gemm_inst<BT, 3>(tm, p, grid, stream);
+    case 4: return launch_gemm_inst<BT, 4>(tm, p, grid, stream);
+    case 8: return launch_gemm_inst<BT, 8>(tm, p, grid, stream);
+    default: return QB_ERR_INVALID;
+  }
+}
+
+// Token-tile width: 256 tokens per tile when that still gives every SM at least two tiles.
+static int choose_token_tile(int64_t M, int64_t N, int sm_count) {
+  if (M <= 128) return 128;
+  const int64_t n_tiles = (N + kTileN - 1) / kTileN;
+  const int64_t tiles256 = n_tiles * ((M + 255) / 256);
+  return tiles256 >= 2 * (int64_t)sm_count ? 256 : 128;
+}
+
+static qb_status validate_gemm(const int8_t* xq, const float* act_scale, const int32_t* rowsum,
+                               const uint32_t* packed, const float* delta, const float* q0, int64_t M, int64_t N,
+                               int64_t K, int bits, int groups, const float* y, const void* ws, size_t ws_bytes) {
+  if (!xq || !act_scale || !rowsum || !packed || !delta || !q0 || !y || M <= 0 || N <= 0 || K <= 0 ||
+      M > QB_MAX_MN || N > QB_MAX_MN || K > QB_MAX_K || !valid_bits(bits) || groups < 1 || N % groups != 0) {
+    set_last_error("qb_gemm: invalid argument (M=%lld N=%lld K=%lld bits=%d groups=%d)", (long long)M,
+                   (long long)N, (long long)K, bits, groups);
+    return QB_ERR_INVALID;
+  }
+  if (K % 128 != 0 || !aligned16(xq) || !aligned16(packed)) {
+    set_last_error("qb_gemm: K must be a multiple of 128 and xq, packed 16-byte aligned");
+    return QB_ERR_ALIGN;
+  }
+  if (!ws || ws_bytes < kWsMinBytes) {
+    set_last_error("qb_gemm: workspace null or too small");
+    return QB_ERR_WORKSPACE;
+  }
+  return QB_OK;
+}
+
+static qb_status launch_gemm(const int8_t* xq, const float* act_scale, const int32_t* rowsum,
+                             const uint32_t* packed, const float* delta, const float* q0, const float* bias,
+                             int64_t M, int64_t N, int64_t K, int bits, int groups, float* y, int32_t* acc_out,
+                             void* ws, int sm_count, cudaStream_t stream) {
+  const int bt = choose_token_tile(M, N, sm_count);
+  CUtensorMap tm;
+  qb_status st = make_x_tensormap(&tm, xq, M, K, bt);
+  if (st != QB_OK) return st;
+  GemmParams p;
+  p.act_scale = act_scale;
+  p.rowsum = rowsum;
+  p.packed = packed;
+  p.delta = delta;
+  p.q0 = q0;
+  p.bias = bias;
+  p.y = y;
+  p.acc_out = acc_out;
+  p.ws = ws;
+  p.M = (int32_t)M;
+  p.N = (int32_t)N;
+  p.K = (int32_t)K;
+  p.rows_per_group = (int32_t)(N / groups);
+  p.n_tiles = (int32_t)((N + kTileN - 1) / kTileN);
+  p.m_tiles = (int32_t)((M + bt - 1) / bt);
+  const int64_t tiles = (int64_t)p.n_tiles * p.m_tiles;
+  const int grid = (int)(tiles < sm_count ? tiles : sm_count);
+  return bt == 256 ? launch_gemm_bits<256>(bits, tm, p, grid, stream)
+                   : launch_gemm_bits<128>(bits, tm, p, grid, stream);
+}
+
+}  // namespace qb
+
+extern "C" qb_status qb_gemm(const int8_t* xq, const float* act_scale, const int32_t* rowsum,
+                             const uint32_t* packed, const float* delta, const float* q0, const float* bias,
+                             int64_t M, int64_t N, int64_t K, int bits, int groups, float* y, int32_t* acc_out,
+                             void* ws, size_t ws_bytes, void* cuda_stream) {
+  qb_status st = qb::validate_gemm(xq, act_scale, rowsum, packed, delta, q0, M, N, K, bits, groups, y, ws, ws_bytes);
+  if (st != QB_OK) return st;
+  int sms = 0;
+  st = qb::require_sm100(&sms);
+  if (st != QB_OK) return st;
+  return qb::launch_gemm(xq, act_scale, rowsum, packed, delta, q0, bias, M, N, K, bits, groups, y, acc_out, ws, sms,
+                         (cudaStream_t)cuda_stream);
+}
+
+extern "C" qb_status qb_layer_linears(const qb_linear_desc* descs, int32_t count, void* ws, size_t ws_bytes,
+                                      void* cuda_stream) {
+  if (!descs || count <= 0) {
+    qb::set_last_error("qb_layer_linears: descs null or count <= 0");
+    return QB_ERR_INVALID;
+  }
+  for (int i = 0; i < count; ++i) {
+    const qb_linear_desc& d = descs[i];
+    qb_status st = qb::validate_gemm(d.xq, d.act_scale, d.rowsum, d.packed, d.delta, d.q0, d.M, d.N, d.K, d.bits,
+                                     d.groups, d.y, ws, ws_bytes);
+    if (st != QB_OK) return st;
+  }
+  int sms = 0;
+  qb_status st = qb::require_sm100(&sms);
+  if (st != QB_OK) return st;
+  for (int i = 0; i < count; ++i) {
+    const qb_linear_desc& d = descs[i];
+    st = qb::launch_gemm(d.xq, d.act_scale, d.rowsum, d.packed, d.delta, d.q0, d.bias, d.M, d.N, d.K, d.bits,
+                         d.groups, d.y, nullptr, ws, sms, (cudaStream_t)cuda_stream);
+    if (st != QB_OK) return st;
+  }
+  return QB_OK;
+}

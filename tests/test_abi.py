@@ -1,0 +1,94 @@
+"""CPU-side checks of the C ABI: the library loads, exports every declared symbol, and rejects bad
+arguments on the host before any launch (these calls never reach a kernel)."""
+import ctypes
+import re
+from pathlib import Path
+
+import pytest
+
+import paper_1909_05840_b200 as qb
+from paper_1909_05840_b200 import build as qb_build
+
+ROOT = Path(__file__).resolve().parent.parent
+
+
+@pytest.fixture(scope="module")
+def lib():
+    qb_build.build()
+    return qb.lib()
+
+
+def _declared_functions():
+    text = (ROOT / "include" / "qbert.h").read_text()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(qb_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = _declared_functions()
+    assert "qb_gemm" in names and "qb_quantize_act" in names and "qb_layer_linears" in names
+    for name in names:
+        assert hasattr(lib, name), f"{name} declared in qbert.h but not exported"
+    assert set(qb.EXPORTS) <= set(names)
+
+
+def test_version_and_status_strings(lib):
+    assert qb.version() >= 100
+    assert lib.qb_status_string(0) == b"QB_OK"
+    assert lib.qb_status_string(-6) == b"QB_ERR_TIMEOUT"
+    assert lib.qb_status_string(-5) == b"QB_ERR_NONFINITE"
+
+
+def test_packed_words_and_workspace_sizes(lib):
+    assert qb.packed_words(768, 768, 4) == 768 * 768 * 4 // 32
+    assert qb.packed_words(768, 768, 3) == 768 * 768 * 3 // 32
+    assert qb.packed_words(768, 768, 5) == 0
+    assert qb.packed_words(0, 768, 4) == 0
+    assert qb.workspace_bytes() >= 256
+    assert qb.workspace_bytes(groups=768) >= 256 + 8 * 768
+    assert qb.workspace_bytes(groups=768) % 256 == 0
+
+
+def test_desc_struct_layout_matches_header():
+    # 7 pointers, 3 int64, 2 int32, 1 pointer on a 64-bit ABI
+    assert ctypes.sizeof(qb.LinearDescC) == 7 * 8 + 3 * 8 + 2 * 4 + 8
+
+
+def test_argument_errors_are_returned_before_any_launch(lib):
+    A = 0x1000  # fake, 16-byte aligned "device" addresses: validation never dereferences them
+    ws_bytes = qb.workspace_bytes(groups=128)
+    # null pointer
+    assert lib.qb_quantize_act(None, 4, 128, A, A, A, A, ws_bytes, None) == qb.QB_ERR_INVALID
+    # K not a multiple of 128
+    assert lib.qb_quantize_act(A, 4, 100, A, A, A, A, ws_bytes, None) == qb.QB_ERR_ALIGN
+    # misaligned pointer
+    assert lib.qb_quantize_act(A + 4, 4, 128, A, A, A, A, ws_bytes, None) == qb.QB_ERR_ALIGN
+    # workspace too small / null
+    assert lib.qb_quantize_act(A, 4, 128, A, A, A, A, 8, None) == qb.QB_ERR_WORKSPACE
+    assert lib.qb_quantize_act(A, 4, 128, A, A, A, None, ws_bytes, None) == qb.QB_ERR_WORKSPACE
+    # weights: bad bit width, groups that do not divide N, one-sided range
+    assert lib.qb_quantize_pack_weights(A, 12, 128, 5, 1, None, None, A, A, A, A, ws_bytes, None) == qb.QB_ERR_INVALID
+    assert lib.qb_quantize_pack_weights(A, 12, 128, 4, 5, None, None, A, A, A, A, ws_bytes, None) == qb.QB_ERR_INVALID
+    assert lib.qb_quantize_pack_weights(A, 12, 128, 4, 3, A, None, A, A, A, A, ws_bytes, None) == qb.QB_ERR_INVALID
+    assert lib.qb_quantize_pack_weights(A, 1024, 128, 4, 1024, None, None, A, A, A, A, 256, None) == qb.QB_ERR_WORKSPACE
+    # gemm
+    assert lib.qb_gemm(A, A, A, A, A, A, None, 8, 12, 128, 4, 5, A, None, A, ws_bytes, None) == qb.QB_ERR_INVALID
+    assert lib.qb_gemm(A, A, A, A, A, A, None, 8, 12, 192, 4, 3, A, None, A, ws_bytes, None) == qb.QB_ERR_ALIGN
+    assert lib.qb_gemm(A, A, A, A, A, A, None, 8, 12, 128, 4, 3, None, None, A, ws_bytes, None) == qb.QB_ERR_INVALID
+    assert lib.qb_gemm(A, A, A, A, A, A, None, 8, 12, 1 << 20, 4, 3, A, None, A, ws_bytes, None) == qb.QB_ERR_INVALID
+    assert b"qb_gemm" in lib.qb_last_error()
+    # stack: every descriptor is validated before the first launch
+    good = qb.LinearDescC(A, A, A, A, A, A, None, 8, 12, 128, 4, 3, A)
+    bad = qb.LinearDescC(A, A, A, A, A, A, None, 8, 12, 128, 7, 3, A)
+    arr = (qb.LinearDescC * 2)(good, bad)
+    assert lib.qb_layer_linears(arr, 2, A, ws_bytes, None) == qb.QB_ERR_INVALID
+    assert lib.qb_layer_linears(None, 2, A, ws_bytes, None) == qb.QB_ERR_INVALID
+
+
+def test_no_cpu_fallback_without_a_device(lib):
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a CUDA device is present")
+    A = 0x1000
+    st = lib.qb_quantize_act(A, 4, 128, A, A, A, A, qb.workspace_bytes(), None)
+    assert st == qb.QB_ERR_CUDA  # valid arguments, but no sm_100 device: an error, never a CPU path

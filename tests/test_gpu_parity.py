@@ -1,0 +1,253 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by element.
+
+Integer results (activation codes, row sums, packed words, int32 accumulators) must be bit exact;
+fp32 outputs must agree within 1e-6 relative.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_1909_05840_b200 as qb
+from paper_1909_05840_b200 import synth
+
+import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+
+BITS = (2, 3, 4, 8)
+
+
+@pytest.fixture(scope="module")
+def ws():
+    gu.ensure_built()
+    return qb.workspace(groups=8192)
+
+
+# ------------------------------------------------------------------ quantizers alone
+@pytest.mark.parametrize("M,K", [(1, 128), (7, 256), (300, 384), (1024, 768), (129, 3072)])
+def test_quantize_act_matches_oracle(ws, M, K):
+    x = synth.activations(M, K, seed=M + K)
+    xq, sc, rs = gu.gpu_quantize_act(x, ws)
+    st, o_xq, o_s, o_rs = oracle.quantize_act(x)
+    assert qb.read_status(ws) == qb.QB_OK
+    assert np.array_equal(xq.cpu().numpy(), o_xq)
+    assert np.array_equal(rs.cpu().numpy(), o_rs)
+    assert sc.cpu().numpy()[0] == o_s
+
+
+def test_quantize_act_ties_zero_and_nonfinite(ws):
+    # exact midpoints (a = 127 makes x*inv = x): half-to-even on both sides
+    x = np.zeros((2, 128), np.float32)
+    x[0, :8] = [127.0, -127.0, 0.5, 1.5, 2.5, -0.5, -1.5, -2.5]
+    xq, sc, rs = gu.gpu_quantize_act(x, ws)
+    st, o_xq, o_s, o_rs = oracle.quantize_act(x)
+    assert xq.cpu().numpy()[0, :8].tolist() == [127, -127, 0, 2, 2, 0, -2, -2]
+    assert np.array_equal(xq.cpu().numpy(), o_xq) and sc.cpu().numpy()[0] == o_s == 1.0
+    # all-zero tensor: scale 1, zero codes
+    xq, sc, rs = gu.gpu_quantize_act(np.zeros((3, 128), np.float32), ws)
+    assert sc.item() == 1.0 and not xq.any().item() and not rs.any().item()
+    assert qb.read_status(ws) == qb.QB_OK
+    # NaN / Inf: reported through the status word of the workspace, as the oracle reports it
+    for bad in (np.nan, np.inf, -np.inf):
+        ws2 = qb.workspace(groups=16)
+        x = synth.activations(5, 128, seed=3)
+        x[4, 100] = bad
+        gu.gpu_quantize_act(x, ws2)
+        assert qb.read_status(ws2) == qb.QB_ERR_NONFINITE
+        assert oracle.quantize_act(x)[0] == oracle.ERR_NONFINITE
+
+
+@pytest.mark.parametrize("bits", BITS)
+@pytest.mark.parametrize("N,K,groups", [(12, 128, 1), (12, 128, 12), (24, 384, 4), (768, 768, 128),
+                                        (768, 768, 12), (264, 256, 11), (96, 3072, 96), (768, 768, 1)])
+def test_quantize_pack_weights_matches_oracle(ws, bits, N, K, groups):
+    w = synth.weights(N, K, seed=N + K + groups + bits)
+    packed, delta, q0 = gu.gpu_quantize_weights(w, bits, groups, ws)
+    assert qb.read_status(ws) == qb.QB_OK
+    st, codes, o_delta, o_q0 = oracle.quantize_weights(w, bits, groups)
+    assert np.array_equal(gu.words_np(packed), oracle.pack(codes, bits))
+    assert np.array_equal(delta.cpu().numpy(), o_delta)
+    assert np.array_equal(q0.cpu().numpy(), o_q0)
+    # run-to-run determinism (order-independent integer reductions): any difference would be a race
+    packed2, delta2, q02 = gu.gpu_quantize_weights(w, bits, groups, ws)
+    assert torch.equal(packed, packed2) and torch.equal(delta, delta2) and torch.equal(q0, q02)
+
+
+def test_quantize_weights_edge_cases(ws):
+    # constant group, exact ties, caller-supplied (clipping) ranges, non-finite input
+    w = synth.weights(8, 128, seed=1)
+    w[:2] = 0.125
+    w[2, :8] = [0.0, 0.5, 1.5, 2.5, 3.0, 1.0, 2.0, 0.25]
+    w[2, 8:] = 1.0
+    w[3] = w[2]
+    for bits in BITS:
+        packed, delta, q0 = gu.gpu_quantize_weights(w, bits, 4, ws)
+        st, codes, o_delta, o_q0 = oracle.quantize_weights(w, bits, 4)
+        assert np.array_equal(gu.words_np(packed), oracle.pack(codes, bits))
+        assert np.array_equal(delta.cpu().numpy(), o_delta) and np.array_equal(q0.cpu().numpy(), o_q0)
+        assert delta.cpu().numpy()[0] == 1.0
+        lo = np.full(4, -0.03, np.float32)
+        hi = np.full(4, 0.05, np.float32)
+        packed, delta, q0 = gu.gpu_quantize_weights(w, bits, 4, ws, lo, hi)
+        st, codes, o_delta, o_q0 = oracle.quantize_weights(w, bits, 4, lo, hi)
+        assert st == oracle.OK
+        assert np.array_equal(gu.words_np(packed), oracle.pack(codes, bits))
+        assert np.array_equal(delta.cpu().numpy(), o_delta) and np.array_equal(q0.cpu().numpy(), o_q0)
+    assert qb.read_status(ws) == qb.QB_OK
+    ws2 = qb.workspace(groups=16)
+    w[5, 77] = np.nan
+    gu.gpu_quantize_weights(w, 4, 4, ws2)
+    assert qb.read_status(ws2) == qb.QB_ERR_NONFINITE
+    assert oracle.quantize_weights(w, 4, 4)[0] == oracle.ERR_NONFINITE
+
+
+# ------------------------------------------------------------------ whole linear layer
+@pytest.mark.parametrize("bits", BITS)
+@pytest.mark.parametrize("M,N,K,groups", [
+    (128, 128, 128, 1),      # exactly one tile, one K block
+    (1, 8, 128, 8),          # smallest: one token, one row per group
+    (127, 24, 256, 4),       # ragged token tile, tiny N (6-row groups as in 128-group BERT-base)
+    (300, 264, 384, 11),     # several token and neuron tiles, both ragged, groups straddle tiles
+    (260, 768, 1024, 128),   # more K blocks than pipeline stages
+])
+def test_linear_matches_oracle(ws, bits, M, N, K, groups):
+    x = synth.activations(M, K, seed=11 * M + bits)
+    w = synth.weights(N, K, seed=13 * N + bits)
+    b = synth.bias(N, seed=17 * N + bits)
+    gu.check_linear(x, w, b, bits, groups, ws)
+
+
+@pytest.mark.parametrize("bits", BITS)
+def test_linear_wide_token_tiles(ws, bits):
+    # enough tiles that the 256-token tile configuration is selected; ragged in M and N
+    M, N, K, groups = 2040, 4730, 128, 10
+    x = synth.activations(M, K, seed=bits)
+    w = synth.weights(N, K, seed=100 + bits)
+    b = synth.bias(N, seed=200 + bits)
+    gu.check_linear(x, w, b, bits, groups, ws, use_omp=True)
+
+
+def test_linear_without_bias_and_with_positive_activations(ws):
+    M, N, K, groups = 200, 256, 512, 32
+    x = np.abs(synth.activations(M, K, seed=5))   # large row sums: the offset term dominates
+    w = synth.weights(N, K, seed=6)
+    for bits in BITS:
+        gu.check_linear(x, w, None, bits, groups, ws)
+
+
+def test_gemm_one_hot_and_extreme_codes(ws):
+    # one-hot activations return single weight codes: a layout or descriptor slip shows as a permutation
+    K, N = 256, 136
+    x = np.zeros((K, K), np.float32)
+    np.fill_diagonal(x, 1.0)
+    w = synth.weights(N, K, seed=9)
+    for bits in BITS:
+        r = gu.check_linear(x, w, None, bits, 1, ws)
+        st, codes, _, _ = oracle.quantize_weights(w, bits, 1)
+        assert np.array_equal(r["acc"].cpu().numpy(), 127 * codes.T.astype(np.int32))
+    # largest magnitudes: every activation code +-127, every weight code 0 or 2^k-1
+    x = np.where(np.random.default_rng(1).random((130, 4096)) < 0.5, -1.0, 1.0).astype(np.float32)
+    w = np.where(np.random.default_rng(2).random((128, 4096)) < 0.5, -1.0, 1.0).astype(np.float32)
+    for bits in BITS:
+        gu.check_linear(x, w, None, bits, 1, ws)
+
+
+def test_gemm_is_deterministic(ws):
+    M, N, K, bits, groups = 515, 384, 768, 3, 64
+    x = synth.activations(M, K, seed=1)
+    w = synth.weights(N, K, seed=2)
+    b = synth.bias(N, seed=3)
+    r1 = gu.check_linear(x, w, b, bits, groups, ws)
+    y2 = torch.empty_like(r1["y"])
+    qb.gemm(r1["xq"], r1["act_scale"], r1["rowsum"], r1["packed"], r1["delta"], r1["q0"], gu.dev(b), N, bits,
+            groups, ws, y=y2)
+    assert torch.equal(r1["y"], y2)
+
+
+# ------------------------------------------------------------------ the benchmark configurations
+def test_config0_query_projection(ws):
+    wl = synth.workload(0)
+    s = wl.linears[0]
+    x = synth.activations(wl.M, s.K, seed=0)
+    w = synth.weights(s.N, s.K, seed=0)
+    b = synth.bias(s.N, seed=0)
+    gu.check_linear(x, w, b, wl.bits[0], s.groups, ws, use_omp=True)
+
+
+def _check_stack(ws, wl, layers, rows_per_tile=2):
+    """quantize everything, run the stack through qb_layer_linears, compare with the oracle."""
+    descs, refs = [], []
+    for layer in layers:
+        bits = wl.bits[layer]
+        for mi, s in enumerate(wl.linears):
+            seed = synth.seed_for(wl.config, layer, mi)
+            x = synth.activations(wl.M, s.K, seed)
+            w = synth.weights(s.N, s.K, seed)
+            b = synth.bias(s.N, seed)
+            xq, sc, rs = gu.gpu_quantize_act(x, ws)
+            packed, delta, q0 = gu.gpu_quantize_weights(w, bits, s.groups, ws)
+            y = gu.poison(torch.empty((wl.M, s.N), dtype=torch.float32, device="cuda"))
+            descs.append(qb.LinearDesc(xq, sc, rs, packed, delta, q0, gu.dev(b), s.N, bits, s.groups, y))
+            refs.append((x, w, b, bits, s))
+    qb.layer_linears(descs, ws)
+    assert qb.read_status(ws) == qb.QB_OK
+    for d, (x, w, b, bits, s) in zip(descs, refs):
+        rows = gu.sample_rows(wl.M, per_tile=rows_per_tile, seed=s.N + bits)
+        st_a, o_xq, o_s, o_rs = oracle.quantize_act(x, omp=True)
+        st_w, codes, o_delta, o_q0 = oracle.quantize_weights(w, bits, s.groups, omp=True)
+        assert np.array_equal(d.xq.cpu().numpy(), o_xq)
+        assert np.array_equal(d.rowsum.cpu().numpy(), o_rs)
+        assert np.array_equal(gu.words_np(d.packed), oracle.pack(codes, bits))
+        assert np.array_equal(d.delta.cpu().numpy(), o_delta) and np.array_equal(d.q0.cpu().numpy(), o_q0)
+        o_acc = oracle.int_gemm(o_xq[rows], codes, omp=True)
+        o_y = oracle.dequant_epilogue(o_acc, o_rs[rows], o_s, o_delta, o_q0, b, bits, s.groups)
+        gu.assert_y_close(d.y[torch.from_numpy(rows).cuda()].cpu().numpy(), o_y)
+        # the stack must equal the single call bit for bit
+        y1, acc1 = qb.gemm(d.xq, d.act_scale, d.rowsum, d.packed, d.delta, d.q0, d.bias, d.N, bits, s.groups, ws,
+                           want_acc=True)
+        assert torch.equal(y1, d.y)
+        assert np.array_equal(acc1[torch.from_numpy(rows).cuda()].cpu().numpy(), o_acc)
+
+
+def test_config1_encoder_layer_linears(ws):
+    _check_stack(ws, synth.workload(1), layers=[0])
+
+
+def test_config2_mixed_precision_stack(ws):
+    wl = synth.workload(2)
+    assert sum(b == 2 for b in wl.bits) >= 6 and set(wl.bits) <= set(synth.BITS_CHOICES)
+    _check_stack(ws, wl, layers=range(wl.layers), rows_per_tile=8)
+
+
+@pytest.mark.parametrize("preset", ["2/3-MP SST-2", "2/4-MP SST-2"])
+def test_paper_bit_presets_stack(ws, preset):
+    # the per-layer bit widths printed in the paper's appendix tables, first four layers' worth of bits
+    base = synth.workload(2)
+    wl = synth.Workload(2, preset, 128, 12, base.linears, synth.MP_PRESETS[preset])
+    _check_stack(ws, wl, layers=[0, 2, 3, 5], rows_per_tile=8)
+
+
+def test_config3_bert_large_layer_sampled(ws):
+    # full-size M = 24576 in the launch configuration the benchmark times; one layer, sampled rows
+    _check_stack(ws, synth.workload(3), layers=[0], rows_per_tile=1)
+
+
+def test_config4_quantizer_sweep_sample(ws):
+    # the distinct shapes of the sweep (incl. the 768 x 30720 embedding-shaped matrix) at every k and
+    # a spread of group counts; the activation tensor of the sweep at full size
+    shapes = sorted(set(synth.quantizer_sweep_shapes()))
+    for i, (N, K) in enumerate(shapes):
+        w = synth.weights(N, K, seed=synth.seed_for(4, 0, i))
+        for bits, groups in ((2, 1), (3, 12), (4, 128), (8, 768)):
+            packed, delta, q0 = gu.gpu_quantize_weights(w, bits, groups, ws)
+            st, codes, o_delta, o_q0 = oracle.quantize_weights(w, bits, groups, omp=True)
+            assert np.array_equal(gu.words_np(packed), oracle.pack(codes, bits)), (N, K, bits, groups)
+            assert np.array_equal(delta.cpu().numpy(), o_delta) and np.array_equal(q0.cpu().numpy(), o_q0)
+    M, K = synth.QUANTIZER_SWEEP_ACT
+    x = synth.activations(M, K, seed=synth.seed_for(4))
+    xq, sc, rs = gu.gpu_quantize_act(x, ws)
+    st, o_xq, o_s, o_rs = oracle.quantize_act(x, omp=True)
+    assert np.array_equal(xq.cpu().numpy(), o_xq) and np.array_equal(rs.cpu().numpy(), o_rs)
+    assert sc.item() == o_s
+    assert qb.read_status(ws) == qb.QB_OK
