@@ -1,0 +1,441 @@
+#!/usr/bin/env python
+"""Benchmark of the quantized-linear hot path on B200.
+
+One *step* is one pass of the whole path over one batch of synthetic input: for each linear of the
+workload, quantize the activations (2 kernels), quantize and pack the weights (2 kernels), then run
+the stack of integer GEMMs with dequantizing epilogue (1 kernel per linear).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference]
+
+prints ONE JSON line.  With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank
+runs its own batch (the path shards over tokens with no exchange: weak scaling) and rank 0 reports
+the aggregate over the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import sys
+import threading
+import time
+from pathlib import Path
+
+import numpy as np
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+from paper_1909_05840_b200 import synth  # noqa: E402
+
+METRIC = "group-wise k-bit qb_gemm TOPS and GB/s on 1 B200 (% of int8 / HBM roofline)"
+UNIT = "TOPS"
+NOMINAL_INT8_OVER_BF16 = 2.0  # dense int8 peak / dense bf16 peak (4.5 / 2.25 PFLOP/s nominal)
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# DRAM traffic of qb_gemm per launch (dram__bytes_read.sum + dram__bytes_write.sum averaged over the
+# launches of one step), from an ncu capture; valid only for the kernel source it was taken on.
+NCU_GEMM_TRAFFIC = {
+    # "<sha256 of csrc/gemm.cu + csrc/ptx.cuh>": {<config>: bytes per launch}
+}
+
+
+def kernel_source_hash() -> str:
+    h = hashlib.sha256()
+    for name in ("gemm.cu", "ptx.cuh"):
+        h.update((ROOT / "paper_1909_05840_b200" / "csrc" / name).read_bytes())
+    return h.hexdigest()[:16]
+
+
+def measured_peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        d = json.loads(p.read_text())
+        return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# --------------------------------------------------------------------------- workload arithmetic
+def linear_list(wl: synth.Workload):
+    """[(layer, matrix index, shape, bits)] in execution order."""
+    return [(layer, mi, s, wl.bits[layer]) for layer in range(wl.layers) for mi, s in enumerate(wl.linears)]
+
+
+def gemm_ops(wl: synth.Workload, M=None) -> float:
+    M = wl.M if M is None else M
+    return float(sum(2.0 * M * s.N * s.K for _, _, s, _ in linear_list(wl)))
+
+
+def gemm_algorithmic_bytes(wl: synth.Workload) -> float:
+    """int8 activations + packed weights + fp32 outputs + bias, row sums and group tables."""
+    tot = 0.0
+    for _, _, s, bits in linear_list(wl):
+        tot += wl.M * s.K + s.N * s.K * bits / 8 + 4.0 * wl.M * s.N + 4 * s.N + 4 * wl.M + 8 * s.groups
+    return tot
+
+
+def act_quant_algorithmic_bytes(wl: synth.Workload) -> float:
+    """two reads of the fp32 tensor (max pass + round pass), one int8 write, row sums."""
+    return float(sum(9.0 * wl.M * s.K + 4 * wl.M for _, _, s, _ in linear_list(wl)))
+
+
+def weight_quant_algorithmic_bytes(wl: synth.Workload) -> float:
+    """one DRAM read of the fp32 matrix (the second pass re-reads it from L2) + k/8 bytes written."""
+    return float(sum(s.N * s.K * (4.0 + bits / 8.0) + 8 * s.groups for _, _, s, bits in linear_list(wl)))
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons with NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.samples = []
+        self.period = period_s
+        self._stop = threading.Event()
+        self._thread = None
+        self.max_mhz = None
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                mhz = int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    reasons = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    reasons = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                self.samples.append((time.time(), mhz, reasons))
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self.ok:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread:
+            self._thread.join(timeout=2)
+
+    def summary(self, t0: float, t1: float):
+        if not self.ok:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvml unavailable"]}
+        sel = [s for s in self.samples if t0 <= s[0] <= t1] or self.samples
+        names = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+                 0x4: "sw_power_cap", 0x80: "hw_power_brake_slowdown"}
+        seen = sorted({n for s in sel for bit, n in names.items() if s[2] & bit})
+        return {"sm_mhz": float(np.median([s[1] for s in sel])) if sel else None, "sm_max_mhz": self.max_mhz,
+                "reasons": seen, "samples": len(sel)}
+
+
+# --------------------------------------------------------------------------- reference arm (oracle)
+def run_reference(args, wl):
+    """Time the CPU oracle, as it stands, on a bounded sample of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    m_sample = min(wl.M, args.ref_rows)
+    lin = linear_list(wl)[: len(wl.linears)]  # first layer
+    data = []
+    for layer, mi, s, bits in lin:
+        seed = synth.seed_for(wl.config, layer, mi)
+        data.append((synth.activations(m_sample, s.K, seed), synth.weights(s.N, s.K, seed), synth.bias(s.N, seed),
+                     bits, s))
+    ops = sum(2.0 * m_sample * s.N * s.K for *_, s in data)
+
+    def step():
+        for x, w, b, bits, s in data:
+            oracle.linear(x, w, b, bits, s.groups, omp=True)
+
+    for _ in range(max(1, min(args.warmup, 1))):
+        step()
+    steps = max(1, min(args.steps, args.ref_steps))
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()
+    dt = (time.perf_counter() - t0) / steps
+    value = ops / dt / 1e12
+    cores = oracle.num_threads(omp=True)
+    sample = (f"first layer of the workload ({len(data)} linears) on the first {m_sample} of {wl.M} token rows: "
+              "quantize activations and weights, pack, integer GEMM, epilogue")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": 1, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int8", "data": "synthetic",
+        "config": {"workload": wl.name, "config_index": wl.config, "M": wl.M, "sample_rows": m_sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------- our arm
+def aggregate_over_ranks(local_ms: float, local_units: float, world: int, dist=None, device=None):
+    """Whole-job throughput: units of all ranks divided by the slowest rank's time."""
+    if world == 1 or dist is None:
+        return local_ms, local_units
+    import torch
+    t = torch.tensor([local_ms], dtype=torch.float64, device=device)
+    u = torch.tensor([local_units], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+def run_ours(args, wl):
+    import torch
+    import paper_1909_05840_b200 as qb
+    from paper_1909_05840_b200 import build as qb_build
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: libqbert has no CPU path")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=device)
+    if rank == 0:
+        qb_build.build()
+    if dist is not None:
+        dist.barrier()
+    qb.lib()
+
+    # ---- inputs: pinned host copies (for the end-to-end arm) and resident device copies ------------
+    lin = linear_list(wl)
+    host, devb = [], []
+    max_groups = max(s.groups for *_, s, _ in lin)
+    ws = qb.workspace(groups=max_groups, device=device)
+    cache = {}
+    for layer, mi, s, bits in lin:
+        seed = synth.seed_for(wl.config, layer, mi) + 100000 * rank
+        key = (s.N, s.K) if wl.layers > 4 else None  # deep stacks: reuse the host arrays per shape
+        if key is not None and key in cache:
+            x, w, b = cache[key]
+        else:
+            x = torch.from_numpy(synth.activations(wl.M, s.K, seed)).pin_memory()
+            w = torch.from_numpy(synth.weights(s.N, s.K, seed)).pin_memory()
+            b = torch.from_numpy(synth.bias(s.N, seed)).pin_memory()
+            if key is not None:
+                cache[key] = (x, w, b)
+        host.append((x, w, b))
+        d = dict(
+            x=x.to(device), w=w.to(device), b=b.to(device),
+            xq=torch.empty((wl.M, s.K), dtype=torch.int8, device=device),
+            sc=torch.empty(1, dtype=torch.float32, device=device),
+            rs=torch.empty(wl.M, dtype=torch.int32, device=device),
+            packed=torch.empty((s.N, s.K * bits // 32), dtype=torch.int32, device=device),
+            delta=torch.empty(s.groups, dtype=torch.float32, device=device),
+            q0=torch.empty(s.groups, dtype=torch.float32, device=device),
+            y=torch.empty((wl.M, s.N), dtype=torch.float32, device=device),
+            bits=bits, s=s)
+        devb.append(d)
+    descs = qb.make_desc_array([qb.LinearDesc(d["xq"], d["sc"], d["rs"], d["packed"], d["delta"], d["q0"], d["b"],
+                                              d["s"].N, d["bits"], d["s"].groups, d["y"]) for d in devb])
+    launches_per_step = 5 * len(lin)  # 2 + 2 + 1 kernels per linear
+
+    def phase_act():
+        for d in devb:
+            qb.quantize_act(d["x"], ws, d["xq"], d["sc"], d["rs"])
+
+    def phase_weights():
+        for d in devb:
+            qb.quantize_pack_weights(d["w"], d["bits"], d["s"].groups, ws, None, None, d["packed"], d["delta"], d["q0"])
+
+    def phase_gemm():
+        qb.layer_linears(descs, ws)
+
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=device)  # > L2 (126 MB)
+
+    def sync_all():
+        torch.cuda.synchronize(device)
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize(device)
+
+    for _ in range(max(3, args.warmup)):
+        phase_act(); phase_weights(); phase_gemm()
+    sync_all()
+    assert qb.read_status(ws) == qb.QB_OK, "device status word reports an error"
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    # keep the GPU busy for a moment so that the clock samples are taken under load
+    t_busy = time.time()
+    while time.time() - t_busy < args.busy_ms * 1e-3:
+        phase_act(); phase_weights(); phase_gemm()
+    sync_all()
+
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    sync_all()
+    t_wall0 = time.time()
+    for i in range(args.steps):
+        flush.fill_(i & 0xFF)                # untimed: evict the previous step's tensors from L2
+        ev[i][0].record(); phase_act()
+        ev[i][1].record(); phase_weights()
+        ev[i][2].record(); phase_gemm()
+        ev[i][3].record()
+    sync_all()
+    t_wall1 = time.time()
+    sampler.stop()
+    assert qb.read_status(ws) == qb.QB_OK, "device status word reports an error"
+    ms_act = float(np.mean([e[0].elapsed_time(e[1]) for e in ev]))
+    ms_w = float(np.mean([e[1].elapsed_time(e[2]) for e in ev]))
+    ms_gemm = float(np.mean([e[2].elapsed_time(e[3]) for e in ev]))
+    ms_step = float(np.mean([e[0].elapsed_time(e[3]) for e in ev]))
+
+    # ---- end to end: host buffers in, results out, copies inside the timed region ------------------
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))  # a shorter loop: each step moves ~250 MB over PCIe
+    y_host = [torch.empty((wl.M, d["s"].N), dtype=torch.float32).pin_memory() for d in devb]
+    h2d = sum(x.numel() * 4 + w.numel() * 4 + b.numel() * 4 for x, w, b in host)
+    d2h = sum(y.numel() * 4 for y in y_host)
+
+    def e2e_step():
+        for (x, w, b), d in zip(host, devb):
+            d["x"].copy_(x, non_blocking=True)
+            d["w"].copy_(w, non_blocking=True)
+            d["b"].copy_(b, non_blocking=True)
+        phase_act(); phase_weights(); phase_gemm()
+        for yh, d in zip(y_host, devb):
+            yh.copy_(d["y"], non_blocking=True)
+
+    e2e_step()
+    sync_all()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    sync_all()
+    ms_e2e = e0.elapsed_time(e1) / e2e_steps
+
+    ops = gemm_ops(wl)
+    ms_job, ops_job = aggregate_over_ranks(ms_step, ops, world, dist, device)
+    ms_e2e_job, _ = aggregate_over_ranks(ms_e2e, ops, world, dist, device)
+    ms_gemm_job, _ = aggregate_over_ranks(ms_gemm, ops, world, dist, device)
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks, peak_kind = measured_peaks()
+    n_gemm = len(lin)
+    gemm_bytes = gemm_algorithmic_bytes(wl)
+    gemm_s_per_launch = ms_gemm * 1e-3 / n_gemm
+    achieved_gbs = gemm_bytes / n_gemm / gemm_s_per_launch / 1e9
+    achieved_tops = ops / n_gemm / gemm_s_per_launch / 1e12
+    int8_peak = peaks["bf16_tflops_sustained"] * NOMINAL_INT8_OVER_BF16
+    t_hbm = gemm_bytes / (peaks["hbm_gbs"] * 1e9)
+    t_tensor = ops / (int8_peak * 1e12)
+    if t_hbm >= t_tensor:
+        roof = {"bound": "hbm", "achieved": achieved_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved_gbs / peaks["hbm_gbs"]}
+    else:
+        roof = {"bound": "tensor", "achieved": achieved_tops, "peak": int8_peak, "unit": "TOP/s",
+                "frac": achieved_tops / int8_peak}
+    traffic = NCU_GEMM_TRAFFIC.get(kernel_source_hash(), {}).get(str(wl.config))
+    roof.update({
+        "traffic": traffic, "kernel": "qb_gemm_kernel", "launches_per_step": n_gemm,
+        "us_per_launch": gemm_s_per_launch * 1e6, "algorithmic_bytes_per_launch": gemm_bytes / n_gemm,
+        "peak_source": f"{peak_kind} (MEASURED_PEAKS.json)" if peak_kind == "measured" else "fallback",
+        "tensor_frac_of_int8_peak": achieved_tops / int8_peak,
+        "int8_peak_note": "sustained bf16 measured peak x nominal int8/bf16 ratio 2.0",
+        "hbm_frac": achieved_gbs / peaks["hbm_gbs"],
+    })
+
+    line = {
+        "metric": METRIC, "value": ops_job / (ms_job * 1e-3) / 1e12, "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_job, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": wl.name, "config_index": wl.config, "M": wl.M, "linears": n_gemm,
+                   "bits": sorted(set(wl.bits)), "l2": "512 MiB flush write between timed steps (untimed)",
+                   "step": "quantize_act + quantize_pack_weights + layer_linears for every linear"},
+        "clocks": sampler.summary(t_wall0, t_wall1),
+        "e2e": {"value": ops_job / (ms_e2e_job * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e_job, "steps": e2e_steps},
+        "gpu_launches": launches_per_step * args.steps,
+        "roofline": roof,
+        "phases": {
+            "quantize_act": {"ms": ms_act, "GBps": act_quant_algorithmic_bytes(wl) / (ms_act * 1e-3) / 1e9,
+                             "frac_hbm": act_quant_algorithmic_bytes(wl) / (ms_act * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+            "quantize_pack_weights": {"ms": ms_w,
+                                      "GBps": weight_quant_algorithmic_bytes(wl) / (ms_w * 1e-3) / 1e9,
+                                      "frac_hbm": weight_quant_algorithmic_bytes(wl) / (ms_w * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+            "gemm": {"ms": ms_gemm_job, "TOPS": ops / (ms_gemm * 1e-3) / 1e12,
+                     "GBps": gemm_bytes / (ms_gemm * 1e-3) / 1e9},
+        },
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(wl, args)
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def cpu_baseline(wl, args):
+    """The oracle, as it stands, on the host cores, on a bounded sample of the same workload."""
+    import oracle
+    oracle.build()
+    m_sample = min(wl.M, args.ref_rows)
+    lin = linear_list(wl)[: len(wl.linears)]
+    data = []
+    for layer, mi, s, bits in lin:
+        seed = synth.seed_for(wl.config, layer, mi)
+        data.append((synth.activations(m_sample, s.K, seed), synth.weights(s.N, s.K, seed), synth.bias(s.N, seed),
+                     bits, s))
+    ops = sum(2.0 * m_sample * s.N * s.K for *_, s in data)
+    t0 = time.perf_counter()
+    reps = 0
+    while reps < 1 or (time.perf_counter() - t0 < 10.0 and reps < 50):
+        for x, w, b, bits, s in data:
+            oracle.linear(x, w, b, bits, s.groups, omp=True)
+        reps += 1
+    dt = (time.perf_counter() - t0) / reps
+    return {"value": ops / dt / 1e12, "unit": UNIT, "cores": oracle.num_threads(omp=True), "kind": "oracle",
+            "sample": f"first layer ({len(data)} linears), first {m_sample} of {wl.M} token rows, whole path, "
+                      f"{reps} repetitions, {dt * 1e3:.1f} ms each"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--config", type=int, default=1, help="workload index 0-3 (see synth.workload)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--ref-rows", type=int, default=256, help="token rows of the oracle's bounded sample")
+    ap.add_argument("--ref-steps", type=int, default=5)
+    ap.add_argument("--e2e-steps", type=int, default=20)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--busy-ms", type=float, default=300.0,
+                    help="untimed load before the timed steps so that clocks are sampled under load")
+    args = ap.parse_args()
+    wl = synth.workload(args.config)
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()
