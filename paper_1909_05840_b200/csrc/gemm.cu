@@ -15,11 +15,13 @@
 // shift makes the expansion a mask and an xor per word; the epilogue shifts the exact int32 sum
 // back.  |sum| <= 127 * 128 * K < 2^31 for K <= 65536.
 //
-// One persistent CTA per SM, ten warps:
+// One persistent CTA per SM, 22 warps:
 //   warp 0        TMA producer for the token tiles               (one lane)
 //   warp 1        tcgen05.mma issuer, owns the TMEM allocation   (one lane)
-//   warps 2..5    weight expanders: thread r owns weight row r of the tile
-//   warps 6..9    epilogue: TMEM -> registers -> fp32 -> global
+//   warps 2..13   weight expanders in three teams of four warps; team g fills the K blocks whose
+//                 running index is g mod 3, thread r of a team owns weight row r of the tile
+//   warps 14..21  epilogue: TMEM -> registers -> fp32 -> shared memory -> TMA store; two warps per
+//                 TMEM lane quarter, each taking every other chunk of 32 tokens
 // Shared-memory ring of STAGES stages (16 KB weights + BT*128 B tokens each, 128-byte swizzle, K
 // block of 128), two accumulator tiles in TMEM so the epilogue of tile i overlaps the MMAs of tile
 // i+1.  Every wait is bounded: on expiry the CTA records QB_ERR_TIMEOUT and leaves through the
@@ -31,11 +33,15 @@
 
 namespace qb {
 
-constexpr int kGemmThreads = 320;
+constexpr int kExpandTeams = 3;     // teams of 128 expander threads
+constexpr int kEpilogueWarps = 8;
+constexpr int kFirstEpilogueWarp = 2 + 4 * kExpandTeams;
+constexpr int kEpilogueThread0 = 32 * kFirstEpilogueWarp;
+constexpr int kGemmThreads = kEpilogueThread0 + 32 * kEpilogueWarps;
 constexpr int kTileN = 128;          // output neurons per tile (MMA M)
 constexpr int kBlockK = 128;         // K elements (= bytes) per pipeline stage
 constexpr int kWBytes = kTileN * kBlockK;
-constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
+constexpr long long kWaitLimitCycles = 4000000000ll;  // about 2 s at 2 GHz
 
 struct GemmParams {
   const float* act_scale;
@@ -50,6 +56,7 @@ struct GemmParams {
   int32_t M, N, K;
   int32_t rows_per_group;
   int32_t n_tiles, m_tiles;
+  int32_t tma_store;  // 1: Y rows are 16-byte aligned, the epilogue stores through TMA
 };
 
 template <int BT>
@@ -58,19 +65,24 @@ struct GemmCfg {
   static constexpr int kStageBytes = kWBytes + kXBytes;
   static constexpr int kStages = (BT == 256) ? 4 : 6;
   static constexpr int kTmemCols = 2 * BT;
-  static constexpr int kBarBytes = 256;
-  static constexpr int kSmemBytes = kStages * kStageBytes + kBarBytes + 1024;  // + alignment slack
+  static constexpr int kBarBytes = 256 + 2 * 256 * 4;  // barriers + two row-sum tiles
+  static constexpr int kOutStageBytes = kEpilogueWarps * 32 * 32 * 4;  // per epilogue warp: 32 tokens x 32 neurons fp32
+  static constexpr int kSmemBytes = kStages * kStageBytes + kOutStageBytes + kBarBytes;
 };
 
 // Bounded wait on an mbarrier phase.  Returns false if the wait expired or another role aborted.
+// The bound is counted in SM clock cycles (clock64 is a cheap register read; the global nanosecond
+// timer costs about a microsecond per read and would dominate short waits).
 __device__ __forceinline__ bool wait_barrier(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  if (ptx::mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = ptx::globaltimer_ns();
+#pragma unroll 1
+  for (int quick = 0; quick < 64; ++quick)
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
   for (uint32_t spin = 1;; ++spin) {
     if (ptx::mbar_try_wait(bar, parity)) return true;
-    if ((spin & 63u) == 0u) {
+    if ((spin & 255u) == 0u) {
       if (*abort_flag) return false;
-      if (ptx::globaltimer_ns() - t0 > kWaitLimitNs) return false;
+      if (clock64() - t0 > kWaitLimitCycles) return false;
     }
   }
 }
@@ -95,16 +107,16 @@ __host__ __device__ constexpr uint32_t make_idesc_i8(int mma_m, int mma_n) {
   return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(mma_n >> 3) << 17) | ((uint32_t)(mma_m >> 4) << 24);
 }
 
-// Expand the 128 codes of one weight row and one K block (BITS 16-byte words) to 128 signed bytes
-// v = (code - 2^(BITS-1)) << (8-BITS), returned as 32 words (word j = codes 4j..4j+3).
+// Expand one item of 32 consecutive codes (BITS packed 32-bit words) to 32 signed bytes
+// v = (code - 2^(BITS-1)) << (8-BITS), returned as 8 words (word j = codes 4j..4j+3).
 template <int BITS>
-__device__ __forceinline__ void expand_codes(const uint32_t (&in)[4 * BITS], uint32_t (&out)[32]) {
+__device__ __forceinline__ void expand_item(const uint32_t* in, uint32_t (&out)[8]) {
   if constexpr (BITS == 8) {
 #pragma unroll
-    for (int i = 0; i < 32; ++i) out[i] = in[i] ^ 0x80808080u;
+    for (int i = 0; i < 8; ++i) out[i] = in[i] ^ 0x80808080u;
   } else if constexpr (BITS == 4) {
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
+    for (int i = 0; i < 4; ++i) {
       const uint32_t w = in[i];
       const uint32_t even = ((w << 4) & 0xF0F0F0F0u) ^ 0x80808080u;  // codes 0,2,4,6 of this word
       const uint32_t odd = (w & 0xF0F0F0F0u) ^ 0x80808080u;          // codes 1,3,5,7
@@ -113,7 +125,7 @@ __device__ __forceinline__ void expand_codes(const uint32_t (&in)[4 * BITS], uin
     }
   } else if constexpr (BITS == 2) {
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
+    for (int i = 0; i < 2; ++i) {
       const uint32_t w = in[i];
       const uint32_t t0 = ((w << 6) & 0xC0C0C0C0u) ^ 0x80808080u;  // codes 0,4,8,12
       const uint32_t t1 = ((w << 4) & 0xC0C0C0C0u) ^ 0x80808080u;  // codes 1,5,9,13
@@ -130,35 +142,57 @@ __device__ __forceinline__ void expand_codes(const uint32_t (&in)[4 * BITS], uin
     }
   } else {  // BITS == 3: 32 codes = 96 bits = 3 words; 4 codes = 12 bits per output word
 #pragma unroll
-    for (int t = 0; t < 4; ++t) {
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const int bit = 12 * j;
-        const int wi = bit >> 5, sh = bit & 31;
-        uint32_t f;
-        if (sh + 12 > 32)
-          f = __funnelshift_r(in[3 * t + wi], in[3 * t + wi + 1], sh);
-        else
-          f = in[3 * t + wi] >> sh;
-        out[8 * t + j] = 0x80808080u ^ ((f << 5) & 0x000000E0u) ^ ((f << 10) & 0x0000E000u) ^
-                         ((f << 15) & 0x00E00000u) ^ ((f << 20) & 0xE0000000u);
-      }
+    for (int j = 0; j < 8; ++j) {
+      const int bit = 12 * j;
+      const int wi = bit >> 5, sh = bit & 31;
+      uint32_t f;
+      if (sh + 12 > 32)
+        f = __funnelshift_r(in[wi], in[wi + 1], sh);
+      else
+        f = in[wi] >> sh;
+      out[j] = 0x80808080u ^ ((f << 5) & 0x000000E0u) ^ ((f << 10) & 0x0000E000u) ^ ((f << 15) & 0x00E00000u) ^
+               ((f << 20) & 0xE0000000u);
     }
+  }
+}
+
+// Load one item (32 codes = BITS words, 4*BITS bytes) with the widest aligned access.
+template <int BITS>
+__device__ __forceinline__ void load_item(const uint32_t* __restrict__ src, uint32_t* dst) {
+  if constexpr (BITS == 8) {
+    const uint4 a = __ldg(reinterpret_cast<const uint4*>(src));
+    const uint4 b = __ldg(reinterpret_cast<const uint4*>(src) + 1);
+    dst[0] = a.x; dst[1] = a.y; dst[2] = a.z; dst[3] = a.w;
+    dst[4] = b.x; dst[5] = b.y; dst[6] = b.z; dst[7] = b.w;
+  } else if constexpr (BITS == 4) {
+    const uint4 a = __ldg(reinterpret_cast<const uint4*>(src));
+    dst[0] = a.x; dst[1] = a.y; dst[2] = a.z; dst[3] = a.w;
+  } else if constexpr (BITS == 2) {
+    const uint2 a = __ldg(reinterpret_cast<const uint2*>(src));
+    dst[0] = a.x; dst[1] = a.y;
+  } else {
+    dst[0] = __ldg(src); dst[1] = __ldg(src + 1); dst[2] = __ldg(src + 2);
   }
 }
 
 template <int BT, int BITS>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-qb_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p) {
+qb_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_y,
+               const GemmParams p) {
   using Cfg = GemmCfg<BT>;
   constexpr int kStages = Cfg::kStages;
-  extern __shared__ uint8_t smem_raw[];
-  // 128-byte swizzle patterns repeat every 1024 bytes: stage bases must be 1024-byte aligned
-  const uint32_t raw_addr = ptx::smem_u32(smem_raw);
-  uint8_t* smem = smem_raw + ((1024u - (raw_addr & 1023u)) & 1023u);
+  // 128-byte swizzle patterns repeat every 1024 bytes: stage bases must be 1024-byte aligned.  The
+  // kernel has no static shared memory, so the dynamic segment starts at offset 0 of the CTA's window.
+  extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t smem_base = ptx::smem_u32(smem);
-  const uint32_t bar_base = smem_base + kStages * Cfg::kStageBytes;
-  uint8_t* bar_ptr = smem + kStages * Cfg::kStageBytes;
+  if ((smem_base & 1023u) != 0u) {  // never expected; leave without touching anything
+    if (threadIdx.x == 0) report_status(p.ws, QB_ERR_CUDA, (int)smem_base);
+    return;
+  }
+  // after the ring: fp32 output staging for the TMA stores (1024-byte aligned), then barriers
+  float* out_stage = reinterpret_cast<float*>(smem + kStages * Cfg::kStageBytes);
+  const uint32_t bar_base = smem_base + kStages * Cfg::kStageBytes + Cfg::kOutStageBytes;
+  uint8_t* bar_ptr = smem + kStages * Cfg::kStageBytes + Cfg::kOutStageBytes;
   auto full_x = [&](int s) { return bar_base + 8u * s; };
   auto full_w = [&](int s) { return bar_base + 8u * (kStages + s); };
   auto empty = [&](int s) { return bar_base + 8u * (2 * kStages + s); };
@@ -167,6 +201,7 @@ qb_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p) {
   const uint32_t drain_bar = bar_base + 8u * (3 * kStages + 4);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_ptr + 8 * (3 * kStages + 5));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float* rs_tile = reinterpret_cast<float*>(bar_ptr + 256);  // [2][256] row sums of a tile's tokens, as fp32
   auto stage_w = [&](int s) { return smem_base + s * Cfg::kStageBytes; };
   auto stage_x = [&](int s) { return smem_base + s * Cfg::kStageBytes + kWBytes; };
 
@@ -181,12 +216,13 @@ qb_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p) {
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(acc_full(a), 1);
-      ptx::mbar_init(acc_empty(a), 128);
+      ptx::mbar_init(acc_empty(a), 32 * kEpilogueWarps);
     }
     ptx::mbar_init(drain_bar, 1);
     *abort_flag = 0;
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&tmap_x);
+    if (p.tma_store) ptx::prefetch_tensormap(&tmap_y);
   }
   if (warp == 1) {
     ptx::tmem_alloc(ptx::smem_u32(tmem_slot), Cfg::kTmemCols);
@@ -225,8 +261,8 @@ qb_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p) {
       }
       if (timed_out) {
         // let copies already in flight land before the CTA's shared memory is released
-        const uint64_t t0 = ptx::globaltimer_ns();
-        while (ptx::globaltimer_ns() - t0 < 200000ull) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 400000ll) {
         }
       }
     }
@@ -271,60 +307,80 @@ qb_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p) {
       if (timed_out) {
         // wait (bounded) for the MMAs already issued before tensor memory is freed
         ptx::mma_commit(drain_bar);
-        const uint64_t t0 = ptx::globaltimer_ns();
-        while (!ptx::mbar_try_wait(drain_bar, 0) && ptx::globaltimer_ns() - t0 < 200000000ull) {
+        const long long t0 = clock64();
+        while (!ptx::mbar_try_wait(drain_bar, 0) && clock64() - t0 < 400000000ll) {
         }
       }
     }
-  } else if (warp < 6) {
+  } else if (warp < kFirstEpilogueWarp) {
     // ---------------- weight expanders ------------------------------------------------------------
-    const int r = threadIdx.x - 64;  // weight row inside the tile
-    const int units_per_row = p.K / 128 * BITS;  // 16-byte words per packed row
-    int stage = 0;
-    uint32_t phase = 0;
-    for (int t = blockIdx.x; t < total_tiles && !timed_out; t += gridDim.x) {
-      const int n = (t % p.n_tiles) * kTileN + r;
-      const bool valid = n < p.N;
-      const uint4* src = reinterpret_cast<const uint4*>(p.packed) + (size_t)(valid ? n : 0) * units_per_row;
-      uint32_t cur[4 * BITS], nxt[4 * BITS];
-      auto load_block = [&](int kb, uint32_t (&dst)[4 * BITS]) {
+    // A K block of the tile is 128 rows x 4 items of 32 codes.  Thread i of a team takes items
+    // i, i+128, i+256, i+384: piece i%4 of rows i/4 + 32j.  Four neighbouring lanes read one row's
+    // 16*BITS contiguous bytes, so a warp-wide load touches 8 rows instead of 32.
+    const int team = (warp - 2) >> 2;
+    const int i_team = (threadIdx.x - 64) & 127;
+    const int piece = i_team & 3;
+    const int row0 = i_team >> 2;
+    const int words_per_row = p.K / 32 * BITS;
+    const int my_tiles = (total_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int total_q = my_tiles * k_blocks;     // K blocks this CTA processes, in order
+    // position of the next block to fetch: tile iteration ld_ti, K block ld_kb, first weight row ld_n0
+    int ld_ti = team / k_blocks;
+    int ld_kb = team - ld_ti * k_blocks;
+    auto n0_of_tile = [&](int ti) { return (int)((blockIdx.x + ti * gridDim.x) % p.n_tiles) * kTileN; };
+    int ld_n0 = n0_of_tile(ld_ti);
+    uint32_t nxt[4 * BITS];
+    auto load_next = [&]() {
 #pragma unroll
-        for (int i = 0; i < BITS; ++i) {
-          uint4 v = valid ? __ldg(src + (size_t)kb * BITS + i) : make_uint4(0, 0, 0, 0);
-          dst[4 * i] = v.x;
-          dst[4 * i + 1] = v.y;
-          dst[4 * i + 2] = v.z;
-          dst[4 * i + 3] = v.w;
-        }
-      };
-      load_block(0, nxt);
-      for (int kb = 0; kb < k_blocks; ++kb) {
+      for (int j = 0; j < 4; ++j) {
+        const int n = ld_n0 + row0 + 32 * j;
+        if (n < p.N) {
+          load_item<BITS>(p.packed + (size_t)n * words_per_row + ld_kb * (4 * BITS) + piece * BITS, nxt + j * BITS);
+        } else {
+          // rows past N: their accumulators are never stored, any operand value will do
 #pragma unroll
-        for (int i = 0; i < 4 * BITS; ++i) cur[i] = nxt[i];
-        if (kb + 1 < k_blocks) load_block(kb + 1, nxt);
-        uint32_t out[32];
-        expand_codes<BITS>(cur, out);
-        if (!valid) {
+          for (int w = 0; w < BITS; ++w) nxt[j * BITS + w] = 0u;
+        }
+      }
+      ld_kb += kExpandTeams;
+      if (ld_kb >= k_blocks) {  // next tile(s) of this CTA
+        do {
+          ld_kb -= k_blocks;
+          ++ld_ti;
+        } while (ld_kb >= k_blocks);
+        ld_n0 = n0_of_tile(ld_ti);
+      }
+    };
+    if (team < total_q) load_next();
+    int stage = team % kStages;
+    uint32_t phase = (uint32_t)(team / kStages) & 1u;
+    for (int q = team; q < total_q; q += kExpandTeams) {
+      uint32_t cur[4 * BITS];
 #pragma unroll
-          for (int i = 0; i < 32; ++i) out[i] = 0u;
-        }
-        if (!wait_barrier(empty(stage), phase ^ 1u, abort_flag)) {
-          timed_out = true;
-          where = (2 << 16) | stage;
-          break;
-        }
-        uint8_t* row_ptr = smem + stage * Cfg::kStageBytes + r * 128;
+      for (int i = 0; i < 4 * BITS; ++i) cur[i] = nxt[i];
+      if (q + kExpandTeams < total_q) load_next();
+      if (!wait_barrier(empty(stage), phase ^ 1u, abort_flag)) {
+        timed_out = true;
+        where = (2 << 16) | stage;
+        break;
+      }
+      uint8_t* stage_ptr = smem + stage * Cfg::kStageBytes;
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          uint4 v = make_uint4(out[4 * c], out[4 * c + 1], out[4 * c + 2], out[4 * c + 3]);
-          *reinterpret_cast<uint4*>(row_ptr + ((c ^ (r & 7)) << 4)) = v;
-        }
-        ptx::fence_proxy_async_smem();
-        ptx::mbar_arrive(full_w(stage));
-        if (++stage == kStages) {
-          stage = 0;
-          phase ^= 1u;
-        }
+      for (int j = 0; j < 4; ++j) {
+        const int row = row0 + 32 * j;
+        uint32_t out[8];
+        expand_item<BITS>(cur + j * BITS, out);
+        // the item is 16-byte chunks 2*piece and 2*piece+1 of the row; 128-byte swizzle: chunk ^ (row % 8)
+        uint8_t* row_ptr = stage_ptr + row * 128;
+        *reinterpret_cast<uint4*>(row_ptr + (((2 * piece) ^ (row & 7)) << 4)) = make_uint4(out[0], out[1], out[2], out[3]);
+        *reinterpret_cast<uint4*>(row_ptr + (((2 * piece + 1) ^ (row & 7)) << 4)) = make_uint4(out[4], out[5], out[6], out[7]);
+      }
+      ptx::fence_proxy_async_smem();
+      ptx::mbar_arrive(full_w(stage));
+      stage += kExpandTeams;
+      if (stage >= kStages) {
+        stage -= kStages;
+        phase ^= 1u;
       }
     }
   } else {
@@ -350,6 +406,13 @@ qb_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p) {
         beta = __fmul_rn(s_a, zc);
         b = p.bias ? __ldg(p.bias + n) : 0.0f;
       }
+      // row sums of this tile's tokens -> shared memory (zero past M), visible to the four epilogue warps
+      {
+        const int e = threadIdx.x - kEpilogueThread0;
+        if (e < BT)
+          rs_tile[a * 256 + e] = (m0 + e < p.M) ? (float)__ldg(p.rowsum + m0 + e) : 0.0f;  // exact: |rowsum| < 2^24
+        asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpilogueWarps) : "memory");
+      }
       if (!wait_barrier(acc_full(a), aphase, abort_flag)) {
         timed_out = true;
         where = (3 << 16) | a;
@@ -357,33 +420,72 @@ qb_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p) {
       }
       ptx::tcgen05_fence_after_sync();
       const uint32_t t_base = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * BT);
-#pragma unroll 1
-      for (int ch = 0; ch < BT / 32; ++ch) {
+      const int n_chunks = min(BT / 32, (p.M - m0 + 31) / 32);  // chunks of 32 tokens, warp-uniform
+      // One chunk: dequantize 32 tokens x this lane's neuron and send them out.
+      auto process = [&](uint32_t (&v)[32], int ch) {
         const int mc = m0 + ch * 32;
-        if (mc >= p.M) break;  // warp-uniform
-        uint32_t v[32];
-        ptx::tmem_ld_32x32b_x32(t_base + (uint32_t)(ch * 32), v);
-        ptx::tmem_ld_wait();
-        float* yrow = p.y + (size_t)mc * p.N + n;
-        int32_t* arow = p.acc_out ? p.acc_out + (size_t)mc * p.N + n : nullptr;
+        const float4* rs4 = reinterpret_cast<const float4*>(rs_tile + a * 256 + ch * 32);
+        if (p.tma_store) {
+          // 32 tokens x 32 neurons of this warp -> shared memory [token][neuron] -> one TMA store.
+          // Lanes write consecutive words of a row: conflict-free.  Rows past M and neurons past N
+          // are clipped by the tensor map.
+          float* buf = out_stage + (warp - kFirstEpilogueWarp) * (32 * 32);
+          if (lane == 0) ptx::tma_store_wait_read0();  // this warp's previous store has read the buffer
+          __syncwarp();
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          if (mc + j < p.M) {
-            const int rs = __ldg(p.rowsum + mc + j);
-            const int ac = ((int)v[j]) >> (8 - BITS);
-            const float yv = __fmaf_rn(alpha, (float)ac, __fmaf_rn(beta, (float)rs, b));
-            if (nvalid) {
-              __stcs(yrow + (size_t)j * p.N, yv);
-              if (arow) arow[(size_t)j * p.N] = ac + c_code * rs;
+          for (int q = 0; q < 8; ++q) {
+            const float4 rv = rs4[q];  // same address in every lane: one broadcast read
+            const float rs[4] = {rv.x, rv.y, rv.z, rv.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const int j = 4 * q + i;
+              const int ac = ((int)v[j]) >> (8 - BITS);
+              buf[j * 32 + lane] = __fmaf_rn(alpha, (float)ac, __fmaf_rn(beta, rs[i], b));
+            }
+          }
+          ptx::fence_proxy_async_smem();
+          __syncwarp();
+          const int x0 = (t % p.n_tiles) * kTileN + quarter * 32;
+          if (lane == 0 && x0 < p.N) {
+            ptx::tma_store_2d(&tmap_y, ptx::smem_u32(buf), x0, mc);
+            ptx::tma_store_commit();
+          }
+        }
+        if (!p.tma_store || p.acc_out) {
+          float* yrow = p.y + (size_t)mc * p.N + n;
+          int32_t* arow = p.acc_out ? p.acc_out + (size_t)mc * p.N + n : nullptr;
+          const int rows = min(32, p.M - mc);  // warp-uniform
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            const float4 rv = rs4[q];
+            const float rs[4] = {rv.x, rv.y, rv.z, rv.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const int j = 4 * q + i;
+              const int ac = ((int)v[j]) >> (8 - BITS);
+              if (nvalid && j < rows) {
+                if (!p.tma_store) yrow[(size_t)j * p.N] = __fmaf_rn(alpha, (float)ac, __fmaf_rn(beta, rs[i], b));
+                if (arow) arow[(size_t)j * p.N] = ac + c_code * __float2int_rn(rs[i]);
+              }
             }
           }
         }
+      };
+      // the two warps of a lane quarter take alternate chunks
+#pragma unroll 1
+      for (int ch = (warp - kFirstEpilogueWarp) >> 2; ch < n_chunks; ch += kEpilogueWarps / 4) {
+        uint32_t v[32];
+        ptx::tmem_ld_32x32b_x32(t_base + (uint32_t)(ch * 32), v);
+        ptx::tmem_ld_wait();
+        ptx::tmem_ld_regs_ready(v);
+        process(v, ch);
       }
       ptx::tcgen05_fence_before_sync();
       ptx::mbar_arrive(acc_empty(a));
     }
   }
 
+  if (warp >= kFirstEpilogueWarp && lane == 0) ptx::tma_store_wait_read0();  // staging buffers still in use
   if (timed_out) {
     *abort_flag = 1;
     report_status(p.ws, QB_ERR_TIMEOUT, where);
@@ -439,34 +541,61 @@ static qb_status make_x_tensormap(CUtensorMap* tm, const int8_t* xq, int64_t M, 
   return QB_OK;
 }
 
+// fp32 outputs [M][N], N contiguous; box = 32 neurons x 32 tokens, no swizzle (plain row-major in smem).
+static qb_status make_y_tensormap(CUtensorMap* tm, float* y, int64_t M, int64_t N) {
+  EncodeTiledFn encode = nullptr;
+  qb_status st = get_encode_fn(&encode);
+  if (st != QB_OK) return st;
+  const cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
+  const cuuint64_t strides[1] = {(cuuint64_t)N * 4};
+  const cuuint32_t box[2] = {32, 32};
+  const cuuint32_t elem[2] = {1, 1};
+  CUresult r = encode(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, y, dims, strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                      CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    set_last_error("cuTensorMapEncodeTiled (outputs) failed with CUresult %d (M=%lld N=%lld)", (int)r, (long long)M,
+                   (long long)N);
+    return QB_ERR_CUDA;
+  }
+  return QB_OK;
+}
+
 template <int BT, int BITS>
-static qb_status launch_gemm_inst(const CUtensorMap& tm, const GemmParams& p, int grid, cudaStream_t stream) {
+static qb_status launch_gemm_inst(const CUtensorMap& tm, const CUtensorMap& tmy, const GemmParams& p, int grid, cudaStream_t stream) {
   using Cfg = GemmCfg<BT>;
   auto kernel = qb_gemm_kernel<BT, BITS>;
-  QB_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
-  kernel<<<grid, kGemmThreads, Cfg::kSmemBytes, stream>>>(tm, p);
+  static bool attr_set[64] = {};
+  int dev = 0;
+  QB_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+    QB_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
+    if (dev >= 0 && dev < 64) attr_set[dev] = true;
+  }
+  kernel<<<grid, kGemmThreads, Cfg::kSmemBytes, stream>>>(tm, tmy, p);
   QB_CUDA_TRY(cudaGetLastError());
   return QB_OK;
 }
 
 template <int BT>
-static qb_status launch_gemm_bits(int bits, const CUtensorMap& tm, const GemmParams& p, int grid,
+static qb_status launch_gemm_bits(int bits, const CUtensorMap& tm, const CUtensorMap& tmy, const GemmParams& p, int grid,
                                   cudaStream_t stream) {
   switch (bits) {
-    case 2: return launch_gemm_inst<BT, 2>(tm, p, grid, stream);
-    case 3: return launch_gemm_inst<BT, 3>(tm, p, grid, stream);
-    case 4: return launch_gemm_inst<BT, 4>(tm, p, grid, stream);
-    case 8: return launch_gemm_inst<BT, 8>(tm, p, grid, stream);
+    case 2: return launch_gemm_inst<BT, 2>(tm, tmy, p, grid, stream);
+    case 3: return launch_gemm_inst<BT, 3>(tm, tmy, p, grid, stream);
+    case 4: return launch_gemm_inst<BT, 4>(tm, tmy, p, grid, stream);
+    case 8: return launch_gemm_inst<BT, 8>(tm, tmy, p, grid, stream);
     default: return QB_ERR_INVALID;
   }
 }
 
-// Token-tile width: 256 tokens per tile when that still gives every SM at least two tiles.
+// Token-tile width: the one whose number of waves over the SMs times its width is smaller (ties: 256,
+// which expands each weight tile once for twice as many tokens).
 static int choose_token_tile(int64_t M, int64_t N, int sm_count) {
   if (M <= 128) return 128;
   const int64_t n_tiles = (N + kTileN - 1) / kTileN;
-  const int64_t tiles256 = n_tiles * ((M + 255) / 256);
-  return tiles256 >= 2 * (int64_t)sm_count ? 256 : 128;
+  const int64_t waves256 = (n_tiles * ((M + 255) / 256) + sm_count - 1) / sm_count;
+  const int64_t waves128 = (n_tiles * ((M + 127) / 128) + sm_count - 1) / sm_count;
+  return waves256 * 256 <= waves128 * 128 ? 256 : 128;
 }
 
 static qb_status validate_gemm(const int8_t* xq, const float* act_scale, const int32_t* rowsum,
@@ -497,7 +626,17 @@ static qb_status launch_gemm(const int8_t* xq, const float* act_scale, const int
   CUtensorMap tm;
   qb_status st = make_x_tensormap(&tm, xq, M, K, bt);
   if (st != QB_OK) return st;
+  // Y rows 16-byte aligned: the epilogue stages tiles in shared memory and stores them with TMA
+  const bool tma_store = (N % 4 == 0) && aligned16(y);
+  CUtensorMap tmy;
+  if (tma_store) {
+    st = make_y_tensormap(&tmy, y, M, N);
+    if (st != QB_OK) return st;
+  } else {
+    tmy = tm;  // unused by the kernel
+  }
   GemmParams p;
+  p.tma_store = tma_store ? 1 : 0;
   p.act_scale = act_scale;
   p.rowsum = rowsum;
   p.packed = packed;
@@ -515,8 +654,8 @@ static qb_status launch_gemm(const int8_t* xq, const float* act_scale, const int
   p.m_tiles = (int32_t)((M + bt - 1) / bt);
   const int64_t tiles = (int64_t)p.n_tiles * p.m_tiles;
   const int grid = (int)(tiles < sm_count ? tiles : sm_count);
-  return bt == 256 ? launch_gemm_bits<256>(bits, tm, p, grid, stream)
-                   : launch_gemm_bits<128>(bits, tm, p, grid, stream);
+  return bt == 256 ? launch_gemm_bits<256>(bits, tm, tmy, p, grid, stream)
+                   : launch_gemm_bits<128>(bits, tm, tmy, p, grid, stream);
 }
 
 }  // namespace qb
