@@ -111,6 +111,32 @@ qb_status qb_quantize_pack_weights(const float* w, int64_t N, int64_t K, int bit
                                    void* cuda_stream);
 
 /*
+ * The same quantizer and packer for callers that have no workspace to give.  (The paper has no
+ * counterpart; this entry point exists for the library's users.)
+ *
+ * Some callers cannot allocate device memory at the point where they need this call: a plug-in that
+ * receives tensors but no allocator, code running while its memory pool is frozen, a serving loop in
+ * which cudaMalloc is banned because it stalls the whole device.  For them the per-group min/max
+ * scratch that normally sits in the caller's workspace is a fixed array inside the library, held on
+ * every GPU that loads it until the process ends (256 + 8 * QB_NOALLOC_MAX_GROUPS bytes).  The call
+ * itself allocates and frees nothing.
+ *
+ *  - Arguments and results are those of qb_quantize_pack_weights, minus the workspace.  `groups` may
+ *    not exceed QB_NOALLOC_MAX_GROUPS; a larger value returns QB_ERR_WORKSPACE and launches nothing.
+ *  - status_out: dev int32 [1] or NULL.  When given, it receives this call's device status word
+ *    (QB_OK or QB_ERR_NONFINITE) by a 4-byte device-to-device copy enqueued after the kernels.
+ *  - The first call on each device looks up the array's device address.  Make that first call
+ *    outside any stream capture.
+ *  - Every call uses the same array and finds the previous call's contents in it; the call clears
+ *    what it needs to be zero.  Calls that may run on the GPU at the same time (two streams, two
+ *    host threads) race on the array: order them on one stream or with events.
+ */
+#define QB_NOALLOC_MAX_GROUPS 4096
+qb_status qb_quantize_pack_weights_noalloc(const float* w, int64_t N, int64_t K, int bits, int groups,
+                                           const float* range_lo, const float* range_hi, uint32_t* packed,
+                                           float* delta, float* q0, int32_t* status_out, void* cuda_stream);
+
+/*
  * Quantized linear layer (Appendix A: "integer arithmetic for the matrix multiplication with X^I,
  * and then followed by a gathered dequantization operation").
  *     acc[m][n] = sum_k xq[m][k] * code[n][k]                       (int32, exact)

@@ -29,8 +29,9 @@ QB_ERR_TIMEOUT = -6
 EXPORTS = (
     "qb_version", "qb_status_string", "qb_last_error", "qb_packed_words", "qb_workspace_bytes",
     "qb_workspace_init", "qb_read_status", "qb_quantize_act", "qb_quantize_pack_weights", "qb_gemm",
-    "qb_layer_linears",
+    "qb_layer_linears", "qb_quantize_pack_weights_noalloc",
 )
+NOALLOC_MAX_GROUPS = 4096
 
 
 class QbertError(RuntimeError):
@@ -80,6 +81,8 @@ def lib() -> ctypes.CDLL:
     L.qb_quantize_act.restype = i32
     L.qb_quantize_pack_weights.argtypes = [vp, i64, i64, ctypes.c_int, ctypes.c_int, vp, vp, vp, vp, vp, vp, sz, vp]
     L.qb_quantize_pack_weights.restype = i32
+    L.qb_quantize_pack_weights_noalloc.argtypes = [vp, i64, i64, ctypes.c_int, ctypes.c_int, vp, vp, vp, vp, vp, vp, vp]
+    L.qb_quantize_pack_weights_noalloc.restype = i32
     L.qb_gemm.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, ctypes.c_int, ctypes.c_int, vp, vp, vp, sz, vp]
     L.qb_gemm.restype = i32
     L.qb_layer_linears.argtypes = [ctypes.POINTER(LinearDescC), i32, vp, sz, vp]
@@ -155,6 +158,21 @@ def quantize_pack_weights(w: torch.Tensor, bits: int, groups: int, ws: torch.Ten
     _check(lib().qb_quantize_pack_weights(w.data_ptr(), N, K, bits, groups, _ptr(range_lo), _ptr(range_hi),
                                           packed.data_ptr(), delta.data_ptr(), q0.data_ptr(), ws.data_ptr(),
                                           ws.numel(), _stream()), "qb_quantize_pack_weights")
+    return packed, delta, q0
+
+
+def quantize_pack_weights_noalloc(w: torch.Tensor, bits: int, groups: int, packed: torch.Tensor,
+                                  delta: torch.Tensor, q0: torch.Tensor, status_out: Optional[torch.Tensor] = None,
+                                  range_lo: Optional[torch.Tensor] = None, range_hi: Optional[torch.Tensor] = None):
+    """``qb_quantize_pack_weights_noalloc``: same results as ``quantize_pack_weights`` for callers that
+    cannot allocate a workspace (the scratch is a fixed array inside the library, at most
+    ``NOALLOC_MAX_GROUPS`` groups).  Every buffer, outputs included, is the caller's: this wrapper
+    allocates nothing either.  ``status_out`` (int32 [1], optional) receives the device status word."""
+    assert w.is_cuda and w.dtype == torch.float32 and w.dim() == 2 and w.is_contiguous()
+    N, K = w.shape
+    _check(lib().qb_quantize_pack_weights_noalloc(w.data_ptr(), N, K, bits, groups, _ptr(range_lo), _ptr(range_hi),
+                                                  packed.data_ptr(), delta.data_ptr(), q0.data_ptr(),
+                                                  _ptr(status_out), _stream()), "qb_quantize_pack_weights_noalloc")
     return packed, delta, q0
 
 
