@@ -183,6 +183,19 @@ typedef struct {
 qb_status qb_layer_linears(const qb_linear_desc* descs /*host*/, int32_t count, void* ws,
                            size_t ws_bytes, void* cuda_stream);
 
+/*
+ * Diagnostic: the rate the tensor cores sustain for the GEMM's own instruction (tcgen05.mma kind::i8,
+ * s8 x s8 -> s32, 128 x `tokens` x 32) with both operands resident in shared memory, no global
+ * traffic, four K blocks in flight, one CTA per SM on the default stream.  (No counterpart in the
+ * paper; it gives the denominator for the tensor-bound shapes of qb_gemm.)
+ *   tokens    128 or 256 (the N of the instruction)
+ *   k_blocks  K blocks of 128 per CTA (8 .. 2^22); the run lasts about k_blocks * 0.3 us
+ *   tops_out  host, receives 1e-12 * 2*128*tokens*128*k_blocks*SMs / elapsed seconds
+ *   cycles_per_kblock_out  host or NULL, SM cycles per K block (four instructions) on the slowest SM
+ * Synchronizes the device.  Returns QB_ERR_TIMEOUT if a bounded wait expired.
+ */
+qb_status qb_probe_i8_mma(int32_t tokens, int32_t k_blocks, double* tops_out, double* cycles_per_kblock_out);
+
 #ifdef __cplusplus
 }
 #endif

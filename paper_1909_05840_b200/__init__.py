@@ -29,7 +29,7 @@ QB_ERR_TIMEOUT = -6
 EXPORTS = (
     "qb_version", "qb_status_string", "qb_last_error", "qb_packed_words", "qb_workspace_bytes",
     "qb_workspace_init", "qb_read_status", "qb_quantize_act", "qb_quantize_pack_weights", "qb_gemm",
-    "qb_layer_linears", "qb_quantize_pack_weights_noalloc",
+    "qb_layer_linears", "qb_quantize_pack_weights_noalloc", "qb_probe_i8_mma",
 )
 NOALLOC_MAX_GROUPS = 4096
 
@@ -83,6 +83,8 @@ def lib() -> ctypes.CDLL:
     L.qb_quantize_pack_weights.restype = i32
     L.qb_quantize_pack_weights_noalloc.argtypes = [vp, i64, i64, ctypes.c_int, ctypes.c_int, vp, vp, vp, vp, vp, vp, vp]
     L.qb_quantize_pack_weights_noalloc.restype = i32
+    L.qb_probe_i8_mma.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
+    L.qb_probe_i8_mma.restype = i32
     L.qb_gemm.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, ctypes.c_int, ctypes.c_int, vp, vp, vp, sz, vp]
     L.qb_gemm.restype = i32
     L.qb_layer_linears.argtypes = [ctypes.POINTER(LinearDescC), i32, vp, sz, vp]
@@ -174,6 +176,13 @@ def quantize_pack_weights_noalloc(w: torch.Tensor, bits: int, groups: int, packe
                                                   packed.data_ptr(), delta.data_ptr(), q0.data_ptr(),
                                                   _ptr(status_out), _stream()), "qb_quantize_pack_weights_noalloc")
     return packed, delta, q0
+
+
+def probe_i8_mma(tokens: int = 256, k_blocks: int = 20000):
+    """``qb_probe_i8_mma``: (TOPS, SM cycles per K block) the tensor cores sustain for the GEMM's MMA."""
+    tops, cyc = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    _check(lib().qb_probe_i8_mma(tokens, k_blocks, ctypes.byref(tops), ctypes.byref(cyc)), "qb_probe_i8_mma")
+    return tops.value, cyc.value
 
 
 def gemm(xq: torch.Tensor, act_scale: torch.Tensor, rowsum: torch.Tensor, packed: torch.Tensor,

@@ -22,11 +22,18 @@
 //                 running index is g mod 3, thread r of a team owns weight row r of the tile
 //   warps 14..21  epilogue: TMEM -> registers -> fp32 -> shared memory -> TMA store; two warps per
 //                 TMEM lane quarter, each taking every other chunk of 32 tokens
+// One launch serves up to kMaxProblems independent linears that share the bit width and the token
+// tile: their tiles form one list (longest K first) that the CTAs walk round-robin, so the start-up
+// and the drain of the pipeline are paid once per launch, not once per linear.
 // Shared-memory ring of STAGES stages (16 KB weights + BT*128 B tokens each, 128-byte swizzle, K
 // block of 128), two accumulator tiles in TMEM so the epilogue of tile i overlaps the MMAs of tile
 // i+1.  Every wait is bounded: on expiry the CTA records QB_ERR_TIMEOUT and leaves through the
 // normal exit path (TMEM freed).
 #include <cuda.h>
+
+#include <algorithm>
+#include <cstring>
+#include <vector>
 
 #include "common.cuh"
 #include "ptx.cuh"
@@ -43,7 +50,10 @@ constexpr int kBlockK = 128;         // K elements (= bytes) per pipeline stage
 constexpr int kWBytes = kTileN * kBlockK;
 constexpr long long kWaitLimitCycles = 4000000000ll;  // about 2 s at 2 GHz
 
-struct GemmParams {
+constexpr int kMaxProblems = 16;  // linears per launch (all in kernel-parameter space, no device table)
+
+// One linear of a launch.
+struct Problem {
   const float* act_scale;
   const int32_t* rowsum;
   const uint32_t* packed;
@@ -52,11 +62,20 @@ struct GemmParams {
   const float* bias;
   float* y;
   int32_t* acc_out;
-  void* ws;
   int32_t M, N, K;
   int32_t rows_per_group;
   int32_t n_tiles, m_tiles;
-  int32_t tma_store;  // 1: Y rows are 16-byte aligned, the epilogue stores through TMA
+  int32_t tile_begin;  // index of this problem's first tile in the launch's tile list
+  int32_t tma_store;   // 1: Y rows are 16-byte aligned, the epilogue stores through TMA
+};
+
+struct GroupedParams {
+  CUtensorMap tmx[kMaxProblems];  // int8 activations, box 128 B x BT tokens, 128-byte swizzle
+  CUtensorMap tmy[kMaxProblems];  // fp32 outputs, box 32 neurons x 32 tokens
+  Problem prob[kMaxProblems];
+  void* ws;
+  int32_t count;
+  int32_t total_tiles;
 };
 
 template <int BT>
@@ -175,10 +194,18 @@ __device__ __forceinline__ void load_item(const uint32_t* __restrict__ src, uint
   }
 }
 
+// Position of a role in the launch's tile list: global tile t -> problem, tile coordinates.
+struct TileCursor {
+  int t;   // global tile index (blockIdx.x, + gridDim.x, ...)
+  int pi;  // problem that owns tile t
+  __device__ __forceinline__ void seek(const GroupedParams& gp) {
+    while (pi + 1 < gp.count && t >= gp.prob[pi + 1].tile_begin) ++pi;
+  }
+};
+
 template <int BT, int BITS>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-qb_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_y,
-               const GemmParams p) {
+qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
   using Cfg = GemmCfg<BT>;
   constexpr int kStages = Cfg::kStages;
   // 128-byte swizzle patterns repeat every 1024 bytes: stage bases must be 1024-byte aligned.  The
@@ -186,7 +213,7 @@ qb_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
   extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t smem_base = ptx::smem_u32(smem);
   if ((smem_base & 1023u) != 0u) {  // never expected; leave without touching anything
-    if (threadIdx.x == 0) report_status(p.ws, QB_ERR_CUDA, (int)smem_base);
+    if (threadIdx.x == 0) report_status(gp.ws, QB_ERR_CUDA, (int)smem_base);
     return;
   }
   // after the ring: fp32 output staging for the TMA stores (1024-byte aligned), then barriers
@@ -221,8 +248,6 @@ qb_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
     ptx::mbar_init(drain_bar, 1);
     *abort_flag = 0;
     ptx::fence_mbar_init();
-    ptx::prefetch_tensormap(&tmap_x);
-    if (p.tma_store) ptx::prefetch_tensormap(&tmap_y);
   }
   if (warp == 1) {
     ptx::tmem_alloc(ptx::smem_u32(tmem_slot), Cfg::kTmemCols);
@@ -233,8 +258,7 @@ qb_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
   ptx::tcgen05_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
-  const int total_tiles = p.n_tiles * p.m_tiles;
-  const int k_blocks = p.K / kBlockK;
+  const int total_tiles = gp.total_tiles;
   bool timed_out = false;
   int where = 0;
 
@@ -243,16 +267,48 @@ qb_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
-      for (int t = blockIdx.x; t < total_tiles && !timed_out; t += gridDim.x) {
-        const int m0 = (t / p.n_tiles) * BT;
+      // The token tiles are first touched in DRAM by several CTAs at about the same time, and the
+      // ring holds only a few K blocks: L2 prefetches run kL2Ahead blocks ahead of the loads (into the
+      // CTA's next tile when the current one ends) so that the loads themselves hit L2.
+      constexpr int kL2Ahead = 8;
+      TileCursor c{(int)blockIdx.x, 0};
+      if (c.t < total_tiles) {
+        c.seek(gp);
+        const Problem& pr = gp.prob[c.pi];
+        const int m0 = ((c.t - pr.tile_begin) / pr.n_tiles) * BT;
+        for (int kb = 0; kb < kL2Ahead && kb < pr.K / kBlockK; ++kb) ptx::tma_prefetch_l2_2d(&gp.tmx[c.pi], kb * kBlockK, m0);
+      }
+      for (; c.t < total_tiles && !timed_out; c.t += gridDim.x) {
+        c.seek(gp);
+        const Problem& pr = gp.prob[c.pi];
+        const int m0 = ((c.t - pr.tile_begin) / pr.n_tiles) * BT;
+        const int k_blocks = pr.K / kBlockK;
+        const CUtensorMap* tm = &gp.tmx[c.pi];
+        // the CTA's next tile, for prefetches that run past the end of this one
+        TileCursor nx{c.t + (int)gridDim.x, c.pi};
+        const CUtensorMap* tm_nx = nullptr;
+        int m0_nx = 0, kblocks_nx = 0;
+        if (nx.t < total_tiles) {
+          nx.seek(gp);
+          const Problem& pn = gp.prob[nx.pi];
+          tm_nx = &gp.tmx[nx.pi];
+          m0_nx = ((nx.t - pn.tile_begin) / pn.n_tiles) * BT;
+          kblocks_nx = pn.K / kBlockK;
+        }
         for (int kb = 0; kb < k_blocks; ++kb) {
+          const int ahead = kb + kL2Ahead;
+          if (ahead < k_blocks) {
+            ptx::tma_prefetch_l2_2d(tm, ahead * kBlockK, m0);
+          } else if (tm_nx != nullptr && ahead - k_blocks < kblocks_nx && ahead - k_blocks < kL2Ahead) {
+            ptx::tma_prefetch_l2_2d(tm_nx, (ahead - k_blocks) * kBlockK, m0_nx);
+          }
           if (!wait_barrier(empty(stage), phase ^ 1u, abort_flag)) {
             timed_out = true;
             where = (0 << 16) | stage;
             break;
           }
           ptx::mbar_arrive_expect_tx(full_x(stage), Cfg::kXBytes);
-          ptx::tma_load_2d(stage_x(stage), &tmap_x, full_x(stage), kb * kBlockK, m0);
+          ptx::tma_load_2d(stage_x(stage), tm, full_x(stage), kb * kBlockK, m0);
           if (++stage == kStages) {
             stage = 0;
             phase ^= 1u;
@@ -273,7 +329,10 @@ qb_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
       int stage = 0;
       uint32_t phase = 0;
       int it = 0;
-      for (int t = blockIdx.x; t < total_tiles && !timed_out; t += gridDim.x, ++it) {
+      TileCursor c{(int)blockIdx.x, 0};
+      for (; c.t < total_tiles && !timed_out; c.t += gridDim.x, ++it) {
+        c.seek(gp);
+        const int k_blocks = gp.prob[c.pi].K / kBlockK;
         const int a = it & 1;
         const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
         if (!wait_barrier(acc_empty(a), aphase ^ 1u, abort_flag)) {
@@ -317,25 +376,52 @@ qb_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
     // A K block of the tile is 128 rows x 4 items of 32 codes.  Thread i of a team takes items
     // i, i+128, i+256, i+384: piece i%4 of rows i/4 + 32j.  Four neighbouring lanes read one row's
     // 16*BITS contiguous bytes, so a warp-wide load touches 8 rows instead of 32.
+    // The K blocks of all tiles of this CTA form one sequence; team g takes those with index g mod 3.
     const int team = (warp - 2) >> 2;
     const int i_team = (threadIdx.x - 64) & 127;
     const int piece = i_team & 3;
     const int row0 = i_team >> 2;
-    const int words_per_row = p.K / 32 * BITS;
-    const int my_tiles = (total_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
-    const int total_q = my_tiles * k_blocks;     // K blocks this CTA processes, in order
-    // position of the next block to fetch: tile iteration ld_ti, K block ld_kb, first weight row ld_n0
-    int ld_ti = team / k_blocks;
-    int ld_kb = team - ld_ti * k_blocks;
-    auto n0_of_tile = [&](int ti) { return (int)((blockIdx.x + ti * gridDim.x) % p.n_tiles) * kTileN; };
-    int ld_n0 = n0_of_tile(ld_ti);
-    uint32_t nxt[4 * BITS];
-    auto load_next = [&]() {
+    // fetch cursor: tile, K block inside it, and the tile's weight rows
+    TileCursor c{(int)blockIdx.x, 0};
+    int ld_kb = team;
+    int ld_kblocks = 0, ld_n0 = 0, ld_N = 0, ld_wpr = 0;
+    const uint32_t* ld_packed = nullptr;
+    bool ld_done = c.t >= total_tiles;
+    auto enter_tile = [&]() {  // fields of the tile the cursor stands on
+      c.seek(gp);
+      const Problem& pr = gp.prob[c.pi];
+      ld_kblocks = pr.K / kBlockK;
+      ld_n0 = ((c.t - pr.tile_begin) % pr.n_tiles) * kTileN;
+      ld_N = pr.N;
+      ld_wpr = pr.K / 32 * BITS;
+      ld_packed = pr.packed;
+    };
+    auto normalize = [&]() {  // carry ld_kb over tile ends
+      while (!ld_done && ld_kb >= ld_kblocks) {
+        ld_kb -= ld_kblocks;
+        c.t += gridDim.x;
+        if (c.t >= total_tiles) {
+          ld_done = true;
+        } else {
+          enter_tile();
+        }
+      }
+    };
+    if (!ld_done) {
+      enter_tile();
+      normalize();
+    }
+    // Register prefetch of the packed words, kPrefetch team-iterations ahead.
+    constexpr int kPrefetch = BITS == 8 ? 1 : 2;
+    uint32_t pre[kPrefetch][4 * BITS];
+    bool pre_valid[kPrefetch];
+    auto load_next = [&](uint32_t* nxt) -> bool {
+      if (ld_done) return false;
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const int n = ld_n0 + row0 + 32 * j;
-        if (n < p.N) {
-          load_item<BITS>(p.packed + (size_t)n * words_per_row + ld_kb * (4 * BITS) + piece * BITS, nxt + j * BITS);
+        if (n < ld_N) {
+          load_item<BITS>(ld_packed + (size_t)n * ld_wpr + ld_kb * (4 * BITS) + piece * BITS, nxt + j * BITS);
         } else {
           // rows past N: their accumulators are never stored, any operand value will do
 #pragma unroll
@@ -343,22 +429,24 @@ qb_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
         }
       }
       ld_kb += kExpandTeams;
-      if (ld_kb >= k_blocks) {  // next tile(s) of this CTA
-        do {
-          ld_kb -= k_blocks;
-          ++ld_ti;
-        } while (ld_kb >= k_blocks);
-        ld_n0 = n0_of_tile(ld_ti);
-      }
+      normalize();
+      return true;
     };
-    if (team < total_q) load_next();
+#pragma unroll
+    for (int d = 0; d < kPrefetch; ++d) pre_valid[d] = load_next(pre[d]);
     int stage = team % kStages;
     uint32_t phase = (uint32_t)(team / kStages) & 1u;
-    for (int q = team; q < total_q; q += kExpandTeams) {
+    while (pre_valid[0]) {
       uint32_t cur[4 * BITS];
 #pragma unroll
-      for (int i = 0; i < 4 * BITS; ++i) cur[i] = nxt[i];
-      if (q + kExpandTeams < total_q) load_next();
+      for (int i = 0; i < 4 * BITS; ++i) cur[i] = pre[0][i];
+#pragma unroll
+      for (int d = 0; d + 1 < kPrefetch; ++d) {
+        pre_valid[d] = pre_valid[d + 1];
+#pragma unroll
+        for (int i = 0; i < 4 * BITS; ++i) pre[d][i] = pre[d + 1][i];
+      }
+      pre_valid[kPrefetch - 1] = load_next(pre[kPrefetch - 1]);
       if (!wait_barrier(empty(stage), phase ^ 1u, abort_flag)) {
         timed_out = true;
         where = (2 << 16) | stage;
@@ -387,30 +475,40 @@ qb_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
     // ---------------- epilogue --------------------------------------------------------------------
     const int quarter = warp & 3;              // TMEM lanes this warp may access: 32*quarter ..
     const int r = quarter * 32 + lane;         // output neuron inside the tile
-    const float s_a = __ldg(p.act_scale);
     constexpr int c_code = 1 << (BITS - 1);
     int it = 0;
-    for (int t = blockIdx.x; t < total_tiles && !timed_out; t += gridDim.x, ++it) {
+    TileCursor c{(int)blockIdx.x, 0};
+    for (; c.t < total_tiles && !timed_out; c.t += gridDim.x, ++it) {
+      c.seek(gp);
+      const Problem& pr = gp.prob[c.pi];
+      const CUtensorMap* tmy = &gp.tmy[c.pi];
+      const int local = c.t - pr.tile_begin;
+      const int pM = pr.M, pN = pr.N;
       const int a = it & 1;
       const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
-      const int n = (t % p.n_tiles) * kTileN + r;
-      const int m0 = (t / p.n_tiles) * BT;
-      const bool nvalid = n < p.N;
+      const int n_base = (local % pr.n_tiles) * kTileN;
+      const int n = n_base + r;
+      const int m0 = (local / pr.n_tiles) * BT;
+      const bool nvalid = n < pN;
+      const bool tma_store = pr.tma_store != 0;
+      float* const y_ptr = pr.y;
+      int32_t* const acc_ptr = pr.acc_out;
       float alpha = 0.f, beta = 0.f, b = 0.f;
       if (nvalid) {
-        const int g = n / p.rows_per_group;
-        const float dlt = __ldg(p.delta + g);
-        const float z = __ldg(p.q0 + g);
+        const float s_a = __ldg(pr.act_scale);
+        const int g = n / pr.rows_per_group;
+        const float dlt = __ldg(pr.delta + g);
+        const float z = __ldg(pr.q0 + g);
         const float zc = __fmaf_rn(dlt, (float)c_code, z);
         alpha = __fmul_rn(s_a, dlt);
         beta = __fmul_rn(s_a, zc);
-        b = p.bias ? __ldg(p.bias + n) : 0.0f;
+        b = pr.bias ? __ldg(pr.bias + n) : 0.0f;
       }
-      // row sums of this tile's tokens -> shared memory (zero past M), visible to the four epilogue warps
+      // row sums of this tile's tokens -> shared memory (zero past M), visible to the epilogue warps
       {
         const int e = threadIdx.x - kEpilogueThread0;
         if (e < BT)
-          rs_tile[a * 256 + e] = (m0 + e < p.M) ? (float)__ldg(p.rowsum + m0 + e) : 0.0f;  // exact: |rowsum| < 2^24
+          rs_tile[a * 256 + e] = (m0 + e < pM) ? (float)__ldg(pr.rowsum + m0 + e) : 0.0f;  // exact: |rowsum| < 2^24
         asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpilogueWarps) : "memory");
       }
       if (!wait_barrier(acc_full(a), aphase, abort_flag)) {
@@ -420,41 +518,57 @@ qb_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
       }
       ptx::tcgen05_fence_after_sync();
       const uint32_t t_base = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * BT);
-      const int n_chunks = min(BT / 32, (p.M - m0 + 31) / 32);  // chunks of 32 tokens, warp-uniform
-      // One chunk: dequantize 32 tokens x this lane's neuron and send them out.
-      auto process = [&](uint32_t (&v)[32], int ch) {
+      const int n_chunks = min(BT / 32, (pM - m0 + 31) / 32);  // chunks of 32 tokens, warp-uniform
+      float* buf = out_stage + (warp - kFirstEpilogueWarp) * (32 * 32);
+      const int x0 = n_base + quarter * 32;
+      // the two warps of a lane quarter take alternate chunks
+#pragma unroll 1
+      for (int ch = (warp - kFirstEpilogueWarp) >> 2; ch < n_chunks; ch += kEpilogueWarps / 4) {
+        uint32_t v[32];
+        ptx::tmem_ld_32x32b_x32(t_base + (uint32_t)(ch * 32), v);
+        ptx::tmem_ld_wait();
+        ptx::tmem_ld_regs_ready(v);
         const int mc = m0 + ch * 32;
         const float4* rs4 = reinterpret_cast<const float4*>(rs_tile + a * 256 + ch * 32);
-        if (p.tma_store) {
+        if (tma_store) {
           // 32 tokens x 32 neurons of this warp -> shared memory [token][neuron] -> one TMA store.
           // Lanes write consecutive words of a row: conflict-free.  Rows past M and neurons past N
-          // are clipped by the tensor map.
-          float* buf = out_stage + (warp - kFirstEpilogueWarp) * (32 * 32);
-          if (lane == 0) ptx::tma_store_wait_read0();  // this warp's previous store has read the buffer
-          __syncwarp();
+          // are clipped by the tensor map.  Loads, then arithmetic, then stores, in halves of 16
+          // tokens; the wait for the warp's previous store comes as late as possible.
 #pragma unroll
-          for (int q = 0; q < 8; ++q) {
-            const float4 rv = rs4[q];  // same address in every lane: one broadcast read
-            const float rs[4] = {rv.x, rv.y, rv.z, rv.w};
+          for (int h = 0; h < 2; ++h) {
+            float rsv[16], yv[16];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const int j = 4 * q + i;
-              const int ac = ((int)v[j]) >> (8 - BITS);
-              buf[j * 32 + lane] = __fmaf_rn(alpha, (float)ac, __fmaf_rn(beta, rs[i], b));
+            for (int q = 0; q < 4; ++q) {
+              const float4 rv = rs4[4 * h + q];  // same address in every lane: one broadcast read
+              rsv[4 * q] = rv.x;
+              rsv[4 * q + 1] = rv.y;
+              rsv[4 * q + 2] = rv.z;
+              rsv[4 * q + 3] = rv.w;
             }
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const int ac = ((int)v[16 * h + j]) >> (8 - BITS);
+              yv[j] = __fmaf_rn(alpha, (float)ac, __fmaf_rn(beta, rsv[j], b));
+            }
+            if (h == 0) {
+              if (lane == 0) ptx::tma_store_wait_read0();  // this warp's previous store has read the buffer
+              __syncwarp();
+            }
+#pragma unroll
+            for (int j = 0; j < 16; ++j) buf[(16 * h + j) * 32 + lane] = yv[j];
           }
           ptx::fence_proxy_async_smem();
           __syncwarp();
-          const int x0 = (t % p.n_tiles) * kTileN + quarter * 32;
-          if (lane == 0 && x0 < p.N) {
-            ptx::tma_store_2d(&tmap_y, ptx::smem_u32(buf), x0, mc);
+          if (lane == 0 && x0 < pN) {
+            ptx::tma_store_2d(tmy, ptx::smem_u32(buf), x0, mc);
             ptx::tma_store_commit();
           }
         }
-        if (!p.tma_store || p.acc_out) {
-          float* yrow = p.y + (size_t)mc * p.N + n;
-          int32_t* arow = p.acc_out ? p.acc_out + (size_t)mc * p.N + n : nullptr;
-          const int rows = min(32, p.M - mc);  // warp-uniform
+        if (!tma_store || acc_ptr != nullptr) {
+          float* yrow = y_ptr + (size_t)mc * pN + n;
+          int32_t* arow = acc_ptr ? acc_ptr + (size_t)mc * pN + n : nullptr;
+          const int rows = min(32, pM - mc);  // warp-uniform
 #pragma unroll
           for (int q = 0; q < 8; ++q) {
             const float4 rv = rs4[q];
@@ -464,21 +578,12 @@ qb_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
               const int j = 4 * q + i;
               const int ac = ((int)v[j]) >> (8 - BITS);
               if (nvalid && j < rows) {
-                if (!p.tma_store) yrow[(size_t)j * p.N] = __fmaf_rn(alpha, (float)ac, __fmaf_rn(beta, rs[i], b));
-                if (arow) arow[(size_t)j * p.N] = ac + c_code * __float2int_rn(rs[i]);
+                if (!tma_store) yrow[(size_t)j * pN] = __fmaf_rn(alpha, (float)ac, __fmaf_rn(beta, rs[i], b));
+                if (arow) arow[(size_t)j * pN] = ac + c_code * __float2int_rn(rs[i]);
               }
             }
           }
         }
-      };
-      // the two warps of a lane quarter take alternate chunks
-#pragma unroll 1
-      for (int ch = (warp - kFirstEpilogueWarp) >> 2; ch < n_chunks; ch += kEpilogueWarps / 4) {
-        uint32_t v[32];
-        ptx::tmem_ld_32x32b_x32(t_base + (uint32_t)(ch * 32), v);
-        ptx::tmem_ld_wait();
-        ptx::tmem_ld_regs_ready(v);
-        process(v, ch);
       }
       ptx::tcgen05_fence_before_sync();
       ptx::mbar_arrive(acc_empty(a));
@@ -488,7 +593,7 @@ qb_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
   if (warp >= kFirstEpilogueWarp && lane == 0) ptx::tma_store_wait_read0();  // staging buffers still in use
   if (timed_out) {
     *abort_flag = 1;
-    report_status(p.ws, QB_ERR_TIMEOUT, where);
+    report_status(gp.ws, QB_ERR_TIMEOUT, where);
   }
   // ---------------- teardown ----------------------------------------------------------------------
   ptx::tcgen05_fence_before_sync();
@@ -561,7 +666,7 @@ static qb_status make_y_tensormap(CUtensorMap* tm, float* y, int64_t M, int64_t 
 }
 
 template <int BT, int BITS>
-static qb_status launch_gemm_inst(const CUtensorMap& tm, const CUtensorMap& tmy, const GemmParams& p, int grid, cudaStream_t stream) {
+static qb_status launch_group_inst(const GroupedParams& gp, int grid, cudaStream_t stream) {
   using Cfg = GemmCfg<BT>;
   auto kernel = qb_gemm_kernel<BT, BITS>;
   static bool attr_set[64] = {};
@@ -571,30 +676,38 @@ static qb_status launch_gemm_inst(const CUtensorMap& tm, const CUtensorMap& tmy,
     QB_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
-  kernel<<<grid, kGemmThreads, Cfg::kSmemBytes, stream>>>(tm, tmy, p);
+  kernel<<<grid, kGemmThreads, Cfg::kSmemBytes, stream>>>(gp);
   QB_CUDA_TRY(cudaGetLastError());
   return QB_OK;
 }
 
 template <int BT>
-static qb_status launch_gemm_bits(int bits, const CUtensorMap& tm, const CUtensorMap& tmy, const GemmParams& p, int grid,
-                                  cudaStream_t stream) {
+static qb_status launch_group_bits(int bits, const GroupedParams& gp, int grid, cudaStream_t stream) {
   switch (bits) {
-    case 2: return launch_gemm_inst<BT, 2>(tm, tmy, p, grid, stream);
-    case 3: return launch_gemm_inst<BT, 3>(tm, tmy, p, grid, stream);
-    case 4: return launch_gemm_inst<BT, 4>(tm, tmy, p, grid, stream);
-    case 8: return launch_gemm_inst<BT, 8>(tm, tmy, p, grid, stream);
+    case 2: return launch_group_inst<BT, 2>(gp, grid, stream);
+    case 3: return launch_group_inst<BT, 3>(gp, grid, stream);
+    case 4: return launch_group_inst<BT, 4>(gp, grid, stream);
+    case 8: return launch_group_inst<BT, 8>(gp, grid, stream);
     default: return QB_ERR_INVALID;
   }
 }
 
-// Token-tile width: the one whose number of waves over the SMs times its width is smaller (ties: 256,
-// which expands each weight tile once for twice as many tokens).
-static int choose_token_tile(int64_t M, int64_t N, int sm_count) {
-  if (M <= 128) return 128;
-  const int64_t n_tiles = (N + kTileN - 1) / kTileN;
-  const int64_t waves256 = (n_tiles * ((M + 255) / 256) + sm_count - 1) / sm_count;
-  const int64_t waves128 = (n_tiles * ((M + 127) / 128) + sm_count - 1) / sm_count;
+// Token-tile width for a launch: 256 tokens (each expanded weight tile serves twice as many tokens,
+// half the L2 traffic for weights) unless every problem is short or 128-token tiles need fewer
+// waves over the SMs.
+static int choose_token_tile(const qb_linear_desc* d, const int* idx, int count, int sm_count) {
+  int64_t tiles256 = 0, tiles128 = 0;
+  bool all_short = true;
+  for (int i = 0; i < count; ++i) {
+    const qb_linear_desc& q = d[idx[i]];
+    const int64_t n_tiles = (q.N + kTileN - 1) / kTileN;
+    tiles256 += n_tiles * ((q.M + 255) / 256);
+    tiles128 += n_tiles * ((q.M + 127) / 128);
+    all_short = all_short && q.M <= 128;
+  }
+  if (all_short) return 128;
+  const int64_t waves256 = (tiles256 + sm_count - 1) / sm_count;
+  const int64_t waves128 = (tiles128 + sm_count - 1) / sm_count;
   return waves256 * 256 <= waves128 * 128 ? 256 : 128;
 }
 
@@ -618,44 +731,76 @@ static qb_status validate_gemm(const int8_t* xq, const float* act_scale, const i
   return QB_OK;
 }
 
-static qb_status launch_gemm(const int8_t* xq, const float* act_scale, const int32_t* rowsum,
-                             const uint32_t* packed, const float* delta, const float* q0, const float* bias,
-                             int64_t M, int64_t N, int64_t K, int bits, int groups, float* y, int32_t* acc_out,
-                             void* ws, int sm_count, cudaStream_t stream) {
-  const int bt = choose_token_tile(M, N, sm_count);
-  CUtensorMap tm;
-  qb_status st = make_x_tensormap(&tm, xq, M, K, bt);
-  if (st != QB_OK) return st;
-  // Y rows 16-byte aligned: the epilogue stages tiles in shared memory and stores them with TMA
-  const bool tma_store = (N % 4 == 0) && aligned16(y);
-  CUtensorMap tmy;
-  if (tma_store) {
-    st = make_y_tensormap(&tmy, y, M, N);
+// One launch over descriptors d[idx[0..count)] (count <= kMaxProblems), all with the same bit width.
+static qb_status launch_group(const qb_linear_desc* d, const int* idx, int count, int32_t* acc_out, void* ws,
+                              int sm_count, cudaStream_t stream) {
+  const int bits = d[idx[0]].bits;
+  const int bt = choose_token_tile(d, idx, count, sm_count);
+  GroupedParams gp;
+  memset(&gp, 0, sizeof(gp));
+  gp.ws = ws;
+  gp.count = count;
+  int tile = 0;
+  for (int i = 0; i < count; ++i) {
+    const qb_linear_desc& q = d[idx[i]];
+    qb_status st = make_x_tensormap(&gp.tmx[i], q.xq, q.M, q.K, bt);
     if (st != QB_OK) return st;
-  } else {
-    tmy = tm;  // unused by the kernel
+    // Y rows 16-byte aligned: the epilogue stages tiles in shared memory and stores them with TMA
+    const bool tma_store = (q.N % 4 == 0) && aligned16(q.y);
+    if (tma_store) {
+      st = make_y_tensormap(&gp.tmy[i], q.y, q.M, q.N);
+      if (st != QB_OK) return st;
+    } else {
+      gp.tmy[i] = gp.tmx[i];  // unused by the kernel
+    }
+    Problem& p = gp.prob[i];
+    p.act_scale = q.act_scale;
+    p.rowsum = q.rowsum;
+    p.packed = q.packed;
+    p.delta = q.delta;
+    p.q0 = q.q0;
+    p.bias = q.bias;
+    p.y = q.y;
+    p.acc_out = acc_out;
+    p.M = (int32_t)q.M;
+    p.N = (int32_t)q.N;
+    p.K = (int32_t)q.K;
+    p.rows_per_group = (int32_t)(q.N / q.groups);
+    p.n_tiles = (int32_t)((q.N + kTileN - 1) / kTileN);
+    p.m_tiles = (int32_t)((q.M + bt - 1) / bt);
+    p.tile_begin = tile;
+    p.tma_store = tma_store ? 1 : 0;
+    tile += p.n_tiles * p.m_tiles;
   }
-  GemmParams p;
-  p.tma_store = tma_store ? 1 : 0;
-  p.act_scale = act_scale;
-  p.rowsum = rowsum;
-  p.packed = packed;
-  p.delta = delta;
-  p.q0 = q0;
-  p.bias = bias;
-  p.y = y;
-  p.acc_out = acc_out;
-  p.ws = ws;
-  p.M = (int32_t)M;
-  p.N = (int32_t)N;
-  p.K = (int32_t)K;
-  p.rows_per_group = (int32_t)(N / groups);
-  p.n_tiles = (int32_t)((N + kTileN - 1) / kTileN);
-  p.m_tiles = (int32_t)((M + bt - 1) / bt);
-  const int64_t tiles = (int64_t)p.n_tiles * p.m_tiles;
-  const int grid = (int)(tiles < sm_count ? tiles : sm_count);
-  return bt == 256 ? launch_gemm_bits<256>(bits, tm, tmy, p, grid, stream)
-                   : launch_gemm_bits<128>(bits, tm, tmy, p, grid, stream);
+  gp.total_tiles = tile;
+  const int grid = tile < sm_count ? tile : sm_count;
+  return bt == 256 ? launch_group_bits<256>(bits, gp, grid, stream) : launch_group_bits<128>(bits, gp, grid, stream);
+}
+
+// Split a stack into launches: same bit width per launch, longest K first (its tiles are the longest,
+// so they go out first in the round-robin), at most kMaxProblems problems and 2^30 tiles per launch.
+static qb_status launch_stack(const qb_linear_desc* d, int count, void* ws, int sm_count, cudaStream_t stream) {
+  std::vector<int> order(count);
+  for (int i = 0; i < count; ++i) order[i] = i;
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+    if (d[a].bits != d[b].bits) return d[a].bits < d[b].bits;
+    return d[a].K > d[b].K;
+  });
+  int i = 0;
+  while (i < count) {
+    int j = i;
+    int64_t tiles = 0;
+    while (j < count && j - i < kMaxProblems && d[order[j]].bits == d[order[i]].bits) {
+      const int64_t t = ((d[order[j]].N + kTileN - 1) / kTileN) * ((d[order[j]].M + 127) / 128);
+      if (j > i && tiles + t > (1 << 30)) break;
+      tiles += t;
+      ++j;
+    }
+    qb_status st = launch_group(d, order.data() + i, j - i, nullptr, ws, sm_count, stream);
+    if (st != QB_OK) return st;
+    i = j;
+  }
+  return QB_OK;
 }
 
 }  // namespace qb
@@ -669,8 +814,22 @@ extern "C" qb_status qb_gemm(const int8_t* xq, const float* act_scale, const int
   int sms = 0;
   st = qb::require_sm100(&sms);
   if (st != QB_OK) return st;
-  return qb::launch_gemm(xq, act_scale, rowsum, packed, delta, q0, bias, M, N, K, bits, groups, y, acc_out, ws, sms,
-                         (cudaStream_t)cuda_stream);
+  qb_linear_desc d;
+  d.xq = xq;
+  d.act_scale = act_scale;
+  d.rowsum = rowsum;
+  d.packed = packed;
+  d.delta = delta;
+  d.q0 = q0;
+  d.bias = bias;
+  d.M = M;
+  d.N = N;
+  d.K = K;
+  d.bits = bits;
+  d.groups = groups;
+  d.y = y;
+  const int idx = 0;
+  return qb::launch_group(&d, &idx, 1, acc_out, ws, sms, (cudaStream_t)cuda_stream);
 }
 
 extern "C" qb_status qb_layer_linears(const qb_linear_desc* descs, int32_t count, void* ws, size_t ws_bytes,
@@ -688,11 +847,5 @@ extern "C" qb_status qb_layer_linears(const qb_linear_desc* descs, int32_t count
   int sms = 0;
   qb_status st = qb::require_sm100(&sms);
   if (st != QB_OK) return st;
-  for (int i = 0; i < count; ++i) {
-    const qb_linear_desc& d = descs[i];
-    st = qb::launch_gemm(d.xq, d.act_scale, d.rowsum, d.packed, d.delta, d.q0, d.bias, d.M, d.N, d.K, d.bits,
-                         d.groups, d.y, nullptr, ws, sms, (cudaStream_t)cuda_stream);
-    if (st != QB_OK) return st;
-  }
-  return QB_OK;
+  return qb::launch_stack(descs, count, ws, sms, (cudaStream_t)cuda_stream);
 }

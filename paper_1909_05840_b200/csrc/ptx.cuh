@@ -70,6 +70,14 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst_smem, const void* tmap,
       : "memory");
 }
 
+// Ask L2 to fetch the box a later tma_load_2d will read (no shared memory involved, no completion).
+__device__ __forceinline__ void tma_prefetch_l2_2d(const void* tmap, int32_t x, int32_t y) {
+  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(
+                   reinterpret_cast<uint64_t>(tmap)),
+               "r"(x), "r"(y)
+               : "memory");
+}
+
 // 2-D tiled store shared -> global (bulk async group).  Rows / columns of the box that fall outside
 // the tensor are not written.  x * element size must be a multiple of 16 bytes; x, y >= 0.
 __device__ __forceinline__ void tma_store_2d(const void* tmap, uint32_t src_smem, int32_t x, int32_t y) {
