@@ -99,11 +99,21 @@ __device__ __forceinline__ bool wait_barrier(uint32_t bar, uint32_t parity, vola
   const long long t0 = clock64();
   for (uint32_t spin = 1;; ++spin) {
     if (ptx::mbar_try_wait(bar, parity)) return true;
+    __nanosleep(32);
     if ((spin & 255u) == 0u) {
       if (*abort_flag) return false;
       if (clock64() - t0 > kWaitLimitCycles) return false;
     }
   }
+}
+
+// Whole-warp wait: only lane 0 polls the barrier (hundreds of threads polling the same shared-memory
+// word would flood the shared-memory pipeline that the stores and the other roles' waits also use);
+// the outcome is broadcast, and the shuffle orders the other lanes' later accesses after the wait.
+__device__ __forceinline__ bool wait_barrier_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  int ok = 1;
+  if ((threadIdx.x & 31) == 0) ok = wait_barrier(bar, parity, abort_flag) ? 1 : 0;
+  return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 
 // Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes, groups of
@@ -238,12 +248,12 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       ptx::mbar_init(full_x(s), 1);
-      ptx::mbar_init(full_w(s), 128);
+      ptx::mbar_init(full_w(s), 4);  // one arrival per warp of the team that filled the stage
       ptx::mbar_init(empty(s), 1);
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(acc_full(a), 1);
-      ptx::mbar_init(acc_empty(a), 32 * kEpilogueWarps);
+      ptx::mbar_init(acc_empty(a), kEpilogueWarps);  // one arrival per epilogue warp
     }
     ptx::mbar_init(drain_bar, 1);
     *abort_flag = 0;
@@ -447,7 +457,7 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
         for (int i = 0; i < 4 * BITS; ++i) pre[d][i] = pre[d + 1][i];
       }
       pre_valid[kPrefetch - 1] = load_next(pre[kPrefetch - 1]);
-      if (!wait_barrier(empty(stage), phase ^ 1u, abort_flag)) {
+      if (!wait_barrier_warp(empty(stage), phase ^ 1u, abort_flag)) {
         timed_out = true;
         where = (2 << 16) | stage;
         break;
@@ -463,8 +473,9 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
         *reinterpret_cast<uint4*>(row_ptr + (((2 * piece) ^ (row & 7)) << 4)) = make_uint4(out[0], out[1], out[2], out[3]);
         *reinterpret_cast<uint4*>(row_ptr + (((2 * piece + 1) ^ (row & 7)) << 4)) = make_uint4(out[4], out[5], out[6], out[7]);
       }
-      ptx::fence_proxy_async_smem();
-      ptx::mbar_arrive(full_w(stage));
+      ptx::fence_proxy_async_smem();  // every lane: its own stores -> visible to the tensor cores
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(full_w(stage));
       stage += kExpandTeams;
       if (stage >= kStages) {
         stage -= kStages;
@@ -511,7 +522,7 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
           rs_tile[a * 256 + e] = (m0 + e < pM) ? (float)__ldg(pr.rowsum + m0 + e) : 0.0f;  // exact: |rowsum| < 2^24
         asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpilogueWarps) : "memory");
       }
-      if (!wait_barrier(acc_full(a), aphase, abort_flag)) {
+      if (!wait_barrier_warp(acc_full(a), aphase, abort_flag)) {
         timed_out = true;
         where = (3 << 16) | a;
         break;
@@ -586,7 +597,8 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
         }
       }
       ptx::tcgen05_fence_before_sync();
-      ptx::mbar_arrive(acc_empty(a));
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(acc_empty(a));
     }
   }
 
@@ -692,23 +704,14 @@ static qb_status launch_group_bits(int bits, const GroupedParams& gp, int grid, 
   }
 }
 
-// Token-tile width for a launch: 256 tokens (each expanded weight tile serves twice as many tokens,
-// half the L2 traffic for weights) unless every problem is short or 128-token tiles need fewer
-// waves over the SMs.
+// Token-tile width for a launch: 256 tokens unless every problem has at most 128.  The 128-wide
+// instruction takes as long as the 256-wide one (measured with qb_probe_i8_mma: 498 vs 512 cycles per
+// K block), so narrow tiles halve the tensor rate and double the weight expansion per token.
 static int choose_token_tile(const qb_linear_desc* d, const int* idx, int count, int sm_count) {
-  int64_t tiles256 = 0, tiles128 = 0;
-  bool all_short = true;
-  for (int i = 0; i < count; ++i) {
-    const qb_linear_desc& q = d[idx[i]];
-    const int64_t n_tiles = (q.N + kTileN - 1) / kTileN;
-    tiles256 += n_tiles * ((q.M + 255) / 256);
-    tiles128 += n_tiles * ((q.M + 127) / 128);
-    all_short = all_short && q.M <= 128;
-  }
-  if (all_short) return 128;
-  const int64_t waves256 = (tiles256 + sm_count - 1) / sm_count;
-  const int64_t waves128 = (tiles128 + sm_count - 1) / sm_count;
-  return waves256 * 256 <= waves128 * 128 ? 256 : 128;
+  (void)sm_count;
+  for (int i = 0; i < count; ++i)
+    if (d[idx[i]].M > 128) return 256;
+  return 128;
 }
 
 static qb_status validate_gemm(const int8_t* xq, const float* act_scale, const int32_t* rowsum,
