@@ -110,6 +110,41 @@ qb_status qb_quantize_pack_weights(const float* w, int64_t N, int64_t K, int bit
                                    float* delta, float* q0, void* ws, size_t ws_bytes,
                                    void* cuda_stream);
 
+/* One tensor of qb_quantize_act_batch: the arguments of qb_quantize_act. */
+typedef struct {
+  const float* x;
+  int64_t M, K;
+  int8_t* xq;
+  float* act_scale;
+  int32_t* rowsum;
+} qb_act_desc;
+
+/* One matrix of qb_quantize_pack_weights_batch: the arguments of qb_quantize_pack_weights. */
+typedef struct {
+  const float* w;
+  int64_t N, K;
+  int32_t bits, groups;
+  const float* range_lo; /* may be NULL (then range_hi too) */
+  const float* range_hi;
+  uint32_t* packed;
+  float* delta;
+  float* q0;
+} qb_weight_desc;
+
+/*
+ * The two quantizers over a whole stack of linears (the inputs and weight matrices of the encoder
+ * layers, Section 3.3 / Table 1 caption) in one pair of launches per call instead of one pair per
+ * tensor: BERT's matrices are a few MB each, so single launches are bound by launch latency, not by
+ * memory bandwidth.  `descs` is a HOST array; every element is validated before anything is launched;
+ * each result equals the single call on the same arguments bit for bit.  Each activation tensor keeps
+ * its own scale (per-tensor quantization).  Weight matrices of different bit widths may be mixed.
+ * Workspace: qb_workspace_bytes(0, 0, 0, 0, G) bytes with G = max(32, sum of `groups` over the batch).
+ */
+qb_status qb_quantize_act_batch(const qb_act_desc* descs /*host*/, int32_t count, void* ws, size_t ws_bytes,
+                                void* cuda_stream);
+qb_status qb_quantize_pack_weights_batch(const qb_weight_desc* descs /*host*/, int32_t count, void* ws,
+                                         size_t ws_bytes, void* cuda_stream);
+
 /*
  * The same quantizer and packer for callers that have no workspace to give.  (The paper has no
  * counterpart; this entry point exists for the library's users.)

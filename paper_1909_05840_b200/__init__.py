@@ -29,7 +29,8 @@ QB_ERR_TIMEOUT = -6
 EXPORTS = (
     "qb_version", "qb_status_string", "qb_last_error", "qb_packed_words", "qb_workspace_bytes",
     "qb_workspace_init", "qb_read_status", "qb_quantize_act", "qb_quantize_pack_weights", "qb_gemm",
-    "qb_layer_linears", "qb_quantize_pack_weights_noalloc", "qb_probe_i8_mma",
+    "qb_layer_linears", "qb_quantize_pack_weights_noalloc", "qb_probe_i8_mma", "qb_quantize_act_batch",
+    "qb_quantize_pack_weights_batch",
 )
 NOALLOC_MAX_GROUPS = 4096
 
@@ -50,6 +51,19 @@ class LinearDescC(ctypes.Structure):
         ("bits", ctypes.c_int32), ("groups", ctypes.c_int32),
         ("y", ctypes.c_void_p),
     ]
+
+
+class ActDescC(ctypes.Structure):
+    """Mirror of ``qb_act_desc``."""
+    _fields_ = [("x", ctypes.c_void_p), ("M", ctypes.c_int64), ("K", ctypes.c_int64), ("xq", ctypes.c_void_p),
+                ("act_scale", ctypes.c_void_p), ("rowsum", ctypes.c_void_p)]
+
+
+class WeightDescC(ctypes.Structure):
+    """Mirror of ``qb_weight_desc``."""
+    _fields_ = [("w", ctypes.c_void_p), ("N", ctypes.c_int64), ("K", ctypes.c_int64), ("bits", ctypes.c_int32),
+                ("groups", ctypes.c_int32), ("range_lo", ctypes.c_void_p), ("range_hi", ctypes.c_void_p),
+                ("packed", ctypes.c_void_p), ("delta", ctypes.c_void_p), ("q0", ctypes.c_void_p)]
 
 
 _lib: Optional[ctypes.CDLL] = None
@@ -85,6 +99,10 @@ def lib() -> ctypes.CDLL:
     L.qb_quantize_pack_weights_noalloc.restype = i32
     L.qb_probe_i8_mma.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
     L.qb_probe_i8_mma.restype = i32
+    L.qb_quantize_act_batch.argtypes = [ctypes.POINTER(ActDescC), i32, vp, sz, vp]
+    L.qb_quantize_act_batch.restype = i32
+    L.qb_quantize_pack_weights_batch.argtypes = [ctypes.POINTER(WeightDescC), i32, vp, sz, vp]
+    L.qb_quantize_pack_weights_batch.restype = i32
     L.qb_gemm.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, ctypes.c_int, ctypes.c_int, vp, vp, vp, sz, vp]
     L.qb_gemm.restype = i32
     L.qb_layer_linears.argtypes = [ctypes.POINTER(LinearDescC), i32, vp, sz, vp]
@@ -161,6 +179,38 @@ def quantize_pack_weights(w: torch.Tensor, bits: int, groups: int, ws: torch.Ten
                                           packed.data_ptr(), delta.data_ptr(), q0.data_ptr(), ws.data_ptr(),
                                           ws.numel(), _stream()), "qb_quantize_pack_weights")
     return packed, delta, q0
+
+
+def make_act_desc_array(items):
+    """``items``: sequence of ``(x, xq, act_scale, rowsum)`` tensors -> C array of ``qb_act_desc``."""
+    arr = (ActDescC * len(items))()
+    for i, (x, xq, sc, rs) in enumerate(items):
+        assert x.is_cuda and x.dtype == torch.float32 and x.dim() == 2 and x.is_contiguous()
+        arr[i] = ActDescC(x.data_ptr(), x.shape[0], x.shape[1], xq.data_ptr(), sc.data_ptr(), rs.data_ptr())
+    return arr
+
+
+def quantize_act_batch(items, ws: torch.Tensor) -> None:
+    """``qb_quantize_act_batch`` over ``(x, xq, act_scale, rowsum)`` tuples (or a prepared C array)."""
+    arr = items if isinstance(items, ctypes.Array) else make_act_desc_array(items)
+    _check(lib().qb_quantize_act_batch(arr, len(arr), ws.data_ptr(), ws.numel(), _stream()), "qb_quantize_act_batch")
+
+
+def make_weight_desc_array(items):
+    """``items``: sequence of ``(w, bits, groups, packed, delta, q0)`` -> C array of ``qb_weight_desc``."""
+    arr = (WeightDescC * len(items))()
+    for i, (w, bits, groups, packed, delta, q0) in enumerate(items):
+        assert w.is_cuda and w.dtype == torch.float32 and w.dim() == 2 and w.is_contiguous()
+        arr[i] = WeightDescC(w.data_ptr(), w.shape[0], w.shape[1], bits, groups, None, None, packed.data_ptr(),
+                             delta.data_ptr(), q0.data_ptr())
+    return arr
+
+
+def quantize_pack_weights_batch(items, ws: torch.Tensor) -> None:
+    """``qb_quantize_pack_weights_batch`` over ``(w, bits, groups, packed, delta, q0)`` tuples (or a C array)."""
+    arr = items if isinstance(items, ctypes.Array) else make_weight_desc_array(items)
+    _check(lib().qb_quantize_pack_weights_batch(arr, len(arr), ws.data_ptr(), ws.numel(), _stream()),
+           "qb_quantize_pack_weights_batch")
 
 
 def quantize_pack_weights_noalloc(w: torch.Tensor, bits: int, groups: int, packed: torch.Tensor,

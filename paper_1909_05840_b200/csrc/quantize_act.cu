@@ -1,33 +1,63 @@
-// qb_quantize_act: per-tensor 8-bit activation quantizer (Table 1 caption: 8-bit activations;
-// Appendix A's uniform quantizer on the symmetric range [-a, a], a = max|x|).
+// qb_quantize_act(_batch): per-tensor 8-bit activation quantizer (Table 1 caption: 8-bit activations;
+// Appendix A's uniform quantizer on the symmetric range [-a, a], a = max|x|), for one tensor or a
+// batch of tensors in one pair of launches.
 //
-// Kernel 1  act_absmax_kernel    grid-stride float4 loads, max of |x| bit patterns (monotone as
-//                                unsigned integers, and NaN/Inf sort above every finite value),
-//                                warp reduce + one atomicMax per block into the workspace.
-// Kernel 2  act_quantize_kernel  one warp per row: x * (127/a), round half to even, clamp, four
-//                                codes packed per 32-bit store, int32 row sum by warp reduction.
+// Kernel 1  act_absmax_kernel    each block belongs to one tensor; block-stride float4 loads, max of
+//                                |x| bit patterns (monotone as unsigned integers, and NaN/Inf sort
+//                                above every finite value), warp reduce + one atomicMax per block
+//                                into the tensor's slot of the workspace.
+// Kernel 2  act_quantize_kernel  one warp per row (rows of all tensors form one sequence):
+//                                x * (127/a), round half to even, clamp, four codes packed per 32-bit
+//                                store, int32 row sum by warp reduction.
 // Both kernels are HBM-bound: 4 B read per element in each, 1 B written in the second.
+#include <cstring>
+
 #include "common.cuh"
 
 namespace qb {
 
 constexpr int kActThreads = 256;
+constexpr int kMaxActBatch = 32;  // tensors per launch (descriptors travel as kernel parameters)
+
+struct ActItem {
+  const float* x;
+  int8_t* xq;
+  float* act_scale;
+  int32_t* rowsum;
+  int64_t M, K;
+  int64_t row_begin;    // index of the tensor's first row in the launch's row sequence
+  int32_t block_begin;  // first block of kernel 1 that works on this tensor
+  int32_t blocks;       // number of such blocks
+};
+
+struct ActBatch {
+  ActItem item[kMaxActBatch];
+  uint32_t* absmax_bits;  // [count] slots in the workspace
+  void* ws;
+  int64_t rows_total;
+  int32_t count;
+};
 
 __global__ void __launch_bounds__(kActThreads)
-act_absmax_kernel(const float4* __restrict__ x, int64_t n4, uint32_t* __restrict__ out_bits) {
+act_absmax_kernel(const __grid_constant__ ActBatch b) {
+  int it = 0;
+  while (it + 1 < b.count && (int)blockIdx.x >= b.item[it + 1].block_begin) ++it;
+  const ActItem& t = b.item[it];
+  const float4* __restrict__ x = reinterpret_cast<const float4*>(t.x);
+  const int64_t n4 = t.M * t.K / 4;
   uint32_t m = 0;
-  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-  int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t stride = (int64_t)t.blocks * blockDim.x;
+  int64_t i = (int64_t)((int)blockIdx.x - t.block_begin) * blockDim.x + threadIdx.x;
   // four independent 16-byte loads in flight per thread
   for (; i + 3 * stride < n4; i += 4 * stride) {
-    float4 a = __ldg(x + i), b = __ldg(x + i + stride), c = __ldg(x + i + 2 * stride),
+    float4 a = __ldg(x + i), bb = __ldg(x + i + stride), c = __ldg(x + i + 2 * stride),
            d = __ldg(x + i + 3 * stride);
 #define QB_ABSMAX4(v)                                            \
   m = max(m, __float_as_uint(v.x) & 0x7fffffffu);                \
   m = max(m, __float_as_uint(v.y) & 0x7fffffffu);                \
   m = max(m, __float_as_uint(v.z) & 0x7fffffffu);                \
   m = max(m, __float_as_uint(v.w) & 0x7fffffffu);
-    QB_ABSMAX4(a) QB_ABSMAX4(b) QB_ABSMAX4(c) QB_ABSMAX4(d)
+    QB_ABSMAX4(a) QB_ABSMAX4(bb) QB_ABSMAX4(c) QB_ABSMAX4(d)
   }
   for (; i < n4; i += stride) {
     float4 a = __ldg(x + i);
@@ -41,7 +71,7 @@ act_absmax_kernel(const float4* __restrict__ x, int64_t n4, uint32_t* __restrict
   if (threadIdx.x < 32) {
     uint32_t v = threadIdx.x < kActThreads / 32 ? warp_max[threadIdx.x] : 0u;
     v = __reduce_max_sync(0xffffffffu, v);
-    if (threadIdx.x == 0 && v != 0u) atomicMax(out_bits, v);
+    if (threadIdx.x == 0 && v != 0u) atomicMax(b.absmax_bits + it, v);
   }
 }
 
@@ -50,31 +80,44 @@ __device__ __forceinline__ int quant_code(float v, float inv) {
   return min(max(q, -127), 127);
 }
 
-__global__ void __launch_bounds__(kActThreads)
-act_quantize_kernel(const float* __restrict__ x, int64_t M, int64_t K, int8_t* __restrict__ xq,
-                    float* __restrict__ act_scale, int32_t* __restrict__ rowsum, void* ws,
-                    const uint32_t* __restrict__ absmax_bits) {
-  const uint32_t mb = *absmax_bits;
-  float s = 1.0f, inv = 0.0f;
-  if (mb >= 0x7f800000u) {  // NaN or Inf somewhere in the tensor
-    if (blockIdx.x == 0 && threadIdx.x == 0) report_status(ws, QB_ERR_NONFINITE);
-  } else {
-    const float a = __uint_as_float(mb);
-    const float s1 = __fdiv_rn(a, 127.0f);
-    const float inv1 = __fdiv_rn(127.0f, a);
-    if (a > 0.0f && inv1 <= 3.402823466e38f) {
-      s = s1;
-      inv = inv1;
-    }
+// scale and reciprocal of a tensor from the bit pattern of its max|x|; false if NaN/Inf was seen
+__device__ __forceinline__ bool act_scales(uint32_t mb, float* s, float* inv) {
+  *s = 1.0f;
+  *inv = 0.0f;
+  if (mb >= 0x7f800000u) return false;
+  const float a = __uint_as_float(mb);
+  const float s1 = __fdiv_rn(a, 127.0f);
+  const float inv1 = __fdiv_rn(127.0f, a);
+  if (a > 0.0f && inv1 <= 3.402823466e38f) {
+    *s = s1;
+    *inv = inv1;
   }
-  if (blockIdx.x == 0 && threadIdx.x == 0) *act_scale = s;
+  return true;
+}
 
+__global__ void __launch_bounds__(kActThreads)
+act_quantize_kernel(const __grid_constant__ ActBatch b) {
   const int lane = threadIdx.x & 31;
   const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
-  const int64_t k4 = K >> 2;  // float4 per row
-  for (int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); row < M; row += warps) {
-    const float4* src = reinterpret_cast<const float4*>(x + row * K);
-    uint32_t* dst = reinterpret_cast<uint32_t*>(xq + row * K);
+  int it = 0;
+  int cur = -1;
+  float inv = 0.0f;
+  for (int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); row < b.rows_total; row += warps) {
+    while (it + 1 < b.count && row >= b.item[it + 1].row_begin) ++it;
+    const ActItem& t = b.item[it];
+    if (it != cur) {  // warp-uniform: first row of this warp in tensor `it`
+      cur = it;
+      float s;
+      const bool finite = act_scales(b.absmax_bits[it], &s, &inv);
+      if (row == t.row_begin && lane == 0) {  // exactly one warp sees the tensor's first row
+        *t.act_scale = s;
+        if (!finite) report_status(b.ws, QB_ERR_NONFINITE);
+      }
+    }
+    const int64_t r = row - t.row_begin;
+    const int64_t k4 = t.K >> 2;  // float4 per row
+    const float4* src = reinterpret_cast<const float4*>(t.x + r * t.K);
+    uint32_t* dst = reinterpret_cast<uint32_t*>(t.xq + r * t.K);
     int sum = 0;
 #pragma unroll 4
     for (int64_t c = lane; c < k4; c += 32) {
@@ -86,28 +129,65 @@ act_quantize_kernel(const float* __restrict__ x, int64_t M, int64_t K, int8_t* _
                ((uint32_t)(q3 & 0xff) << 24);
     }
     sum = __reduce_add_sync(0xffffffffu, sum);
-    if (lane == 0) rowsum[row] = sum;
+    if (lane == 0) t.rowsum[r] = sum;
   }
 }
 
-qb_status launch_quantize_act(const float* x, int64_t M, int64_t K, int8_t* xq, float* act_scale,
-                              int32_t* rowsum, void* ws, uint32_t* absmax_slot, int sm_count,
-                              cudaStream_t stream) {
-  QB_CUDA_TRY(cudaMemsetAsync(absmax_slot, 0, sizeof(uint32_t), stream));
-  const int64_t n4 = M * K / 4;
-  int64_t blocks1 = (n4 + (int64_t)kActThreads * 4 - 1) / ((int64_t)kActThreads * 4);
+// One pair of launches over `count` tensors (<= kMaxActBatch).  `absmax_slots` has room for `count` words.
+static qb_status launch_act_batch(const qb_act_desc* d, int count, void* ws, uint32_t* absmax_slots, int sm_count,
+                                  cudaStream_t stream) {
+  ActBatch b;
+  memset(&b, 0, sizeof(b));
+  b.count = count;
+  b.ws = ws;
+  b.absmax_bits = absmax_slots;
   const int64_t cap = (int64_t)sm_count * 8;
-  if (blocks1 > cap) blocks1 = cap;
-  if (blocks1 < 1) blocks1 = 1;
-  act_absmax_kernel<<<(unsigned)blocks1, kActThreads, 0, stream>>>(reinterpret_cast<const float4*>(x), n4,
-                                                                   absmax_slot);
+  int64_t total4 = 0;
+  for (int i = 0; i < count; ++i) total4 += d[i].M * d[i].K / 4;
+  int64_t rows = 0;
+  int blocks1 = 0;
+  for (int i = 0; i < count; ++i) {
+    ActItem& t = b.item[i];
+    t.x = d[i].x;
+    t.xq = d[i].xq;
+    t.act_scale = d[i].act_scale;
+    t.rowsum = d[i].rowsum;
+    t.M = d[i].M;
+    t.K = d[i].K;
+    t.row_begin = rows;
+    rows += d[i].M;
+    // blocks of kernel 1 in proportion to the tensor's size, each thread >= 4 loads when possible
+    const int64_t n4 = d[i].M * d[i].K / 4;
+    int64_t want = (n4 + (int64_t)kActThreads * 4 - 1) / ((int64_t)kActThreads * 4);
+    const int64_t share = (cap * n4 + total4 - 1) / total4;
+    if (want > share) want = share;
+    if (want < 1) want = 1;
+    t.block_begin = blocks1;
+    t.blocks = (int32_t)want;
+    blocks1 += (int)want;
+  }
+  b.rows_total = rows;
+  QB_CUDA_TRY(cudaMemsetAsync(absmax_slots, 0, sizeof(uint32_t) * (size_t)count, stream));
+  act_absmax_kernel<<<(unsigned)blocks1, kActThreads, 0, stream>>>(b);
   QB_CUDA_TRY(cudaGetLastError());
   const int warps_per_block = kActThreads / 32;
-  int64_t blocks2 = (M + warps_per_block - 1) / warps_per_block;
+  int64_t blocks2 = (rows + warps_per_block - 1) / warps_per_block;
   if (blocks2 > cap) blocks2 = cap;
-  act_quantize_kernel<<<(unsigned)blocks2, kActThreads, 0, stream>>>(x, M, K, xq, act_scale, rowsum, ws,
-                                                                     absmax_slot);
+  act_quantize_kernel<<<(unsigned)blocks2, kActThreads, 0, stream>>>(b);
   QB_CUDA_TRY(cudaGetLastError());
+  return QB_OK;
+}
+
+static qb_status validate_act(const char* who, const float* x, int64_t M, int64_t K, const int8_t* xq,
+                              const float* act_scale, const int32_t* rowsum) {
+  if (!x || !xq || !act_scale || !rowsum || M <= 0 || K <= 0 || M > QB_MAX_MN || K > QB_MAX_K) {
+    set_last_error("%s: null pointer or size out of range (M=%lld K=%lld)", who, (long long)M, (long long)K);
+    return QB_ERR_INVALID;
+  }
+  if (K % 128 != 0 || !aligned16(x) || !aligned16(xq)) {
+    set_last_error("%s: K must be a multiple of 128 and x, xq 16-byte aligned", who);
+    return QB_ERR_ALIGN;
+  }
   return QB_OK;
 }
 
@@ -115,22 +195,45 @@ qb_status launch_quantize_act(const float* x, int64_t M, int64_t K, int8_t* xq, 
 
 extern "C" qb_status qb_quantize_act(const float* x, int64_t M, int64_t K, int8_t* xq, float* act_scale,
                                      int32_t* rowsum, void* ws, size_t ws_bytes, void* cuda_stream) {
-  if (!x || !xq || !act_scale || !rowsum || M <= 0 || K <= 0 || M > QB_MAX_MN || K > QB_MAX_K) {
-    qb::set_last_error("qb_quantize_act: null pointer or size out of range (M=%lld K=%lld)", (long long)M,
-                       (long long)K);
-    return QB_ERR_INVALID;
-  }
-  if (K % 128 != 0 || !qb::aligned16(x) || !qb::aligned16(xq)) {
-    qb::set_last_error("qb_quantize_act: K must be a multiple of 128 and x, xq 16-byte aligned");
-    return QB_ERR_ALIGN;
-  }
+  qb_status st = qb::validate_act("qb_quantize_act", x, M, K, xq, act_scale, rowsum);
+  if (st != QB_OK) return st;
   if (!ws || ws_bytes < qb::ws_bytes_needed(0)) {
     qb::set_last_error("qb_quantize_act: workspace null or too small");
     return QB_ERR_WORKSPACE;
   }
   int sms = 0;
-  qb_status st = qb::require_sm100(&sms);
+  st = qb::require_sm100(&sms);
   if (st != QB_OK) return st;
   uint32_t* slot = reinterpret_cast<uint32_t*>(static_cast<char*>(ws) + qb::kWsActMaxOff);
-  return qb::launch_quantize_act(x, M, K, xq, act_scale, rowsum, ws, slot, sms, (cudaStream_t)cuda_stream);
+  const qb_act_desc d{x, M, K, xq, act_scale, rowsum};
+  return qb::launch_act_batch(&d, 1, ws, slot, sms, (cudaStream_t)cuda_stream);
+}
+
+extern "C" qb_status qb_quantize_act_batch(const qb_act_desc* descs, int32_t count, void* ws, size_t ws_bytes,
+                                           void* cuda_stream) {
+  if (!descs || count <= 0) {
+    qb::set_last_error("qb_quantize_act_batch: descs null or count <= 0");
+    return QB_ERR_INVALID;
+  }
+  for (int i = 0; i < count; ++i) {
+    qb_status st = qb::validate_act("qb_quantize_act_batch", descs[i].x, descs[i].M, descs[i].K, descs[i].xq,
+                                    descs[i].act_scale, descs[i].rowsum);
+    if (st != QB_OK) return st;
+  }
+  // max-abs slots of a launch: the head of the range area of the workspace
+  if (!ws || ws_bytes < qb::kWsRangeOff + sizeof(uint32_t) * (size_t)qb::kMaxActBatch) {
+    qb::set_last_error("qb_quantize_act_batch: workspace null or smaller than %zu bytes",
+                       qb::kWsRangeOff + sizeof(uint32_t) * (size_t)qb::kMaxActBatch);
+    return QB_ERR_WORKSPACE;
+  }
+  int sms = 0;
+  qb_status st = qb::require_sm100(&sms);
+  if (st != QB_OK) return st;
+  uint32_t* slots = reinterpret_cast<uint32_t*>(static_cast<char*>(ws) + qb::kWsRangeOff);
+  for (int i = 0; i < count; i += qb::kMaxActBatch) {
+    const int n = count - i < qb::kMaxActBatch ? count - i : qb::kMaxActBatch;
+    st = qb::launch_act_batch(descs + i, n, ws, slots, sms, (cudaStream_t)cuda_stream);
+    if (st != QB_OK) return st;
+  }
+  return QB_OK;
 }

@@ -177,7 +177,7 @@ def test_config0_query_projection(ws):
 
 def _check_stack(ws, wl, layers, rows_per_tile=2):
     """quantize everything, run the stack through qb_layer_linears, compare with the oracle."""
-    descs, refs = [], []
+    descs, refs, acts, mats = [], [], [], []
     for layer in layers:
         bits = wl.bits[layer]
         for mi, s in enumerate(wl.linears):
@@ -185,11 +185,21 @@ def _check_stack(ws, wl, layers, rows_per_tile=2):
             x = synth.activations(wl.M, s.K, seed)
             w = synth.weights(s.N, s.K, seed)
             b = synth.bias(s.N, seed)
-            xq, sc, rs = gu.gpu_quantize_act(x, ws)
-            packed, delta, q0 = gu.gpu_quantize_weights(w, bits, s.groups, ws)
+            # outputs poisoned, then filled by the batched quantizers below
+            xq = gu.poison(torch.empty((wl.M, s.K), dtype=torch.int8, device="cuda"))
+            sc = gu.poison(torch.empty(1, dtype=torch.float32, device="cuda"))
+            rs = gu.poison(torch.empty(wl.M, dtype=torch.int32, device="cuda"))
+            packed = gu.poison(torch.empty((s.N, s.K * bits // 32), dtype=torch.int32, device="cuda"))
+            delta = gu.poison(torch.empty(s.groups, dtype=torch.float32, device="cuda"))
+            q0 = gu.poison(torch.empty(s.groups, dtype=torch.float32, device="cuda"))
+            acts.append((gu.dev(x), xq, sc, rs))
+            mats.append((gu.dev(w), bits, s.groups, packed, delta, q0))
             y = gu.poison(torch.empty((wl.M, s.N), dtype=torch.float32, device="cuda"))
             descs.append(qb.LinearDesc(xq, sc, rs, packed, delta, q0, gu.dev(b), s.N, bits, s.groups, y))
             refs.append((x, w, b, bits, s))
+    ws = qb.workspace(groups=max(32, sum(m[2] for m in mats)))
+    qb.quantize_act_batch(acts, ws)
+    qb.quantize_pack_weights_batch(mats, ws)
     qb.layer_linears(descs, ws)
     assert qb.read_status(ws) == qb.QB_OK
     for d, (x, w, b, bits, s) in zip(descs, refs):
@@ -208,6 +218,42 @@ def _check_stack(ws, wl, layers, rows_per_tile=2):
                            want_acc=True)
         assert torch.equal(y1, d.y)
         assert np.array_equal(acc1[torch.from_numpy(rows).cuda()].cpu().numpy(), o_acc)
+
+
+def test_batched_quantizers_equal_single_calls(ws):
+    # mixed bit widths and group counts, more tensors than one launch holds (32)
+    rng = np.random.default_rng(3)
+    acts, mats, single_a, single_w = [], [], [], []
+    shapes = [(5, 128), (129, 384), (64, 768), (300, 256)] * 9          # 36 activation tensors
+    for i, (M, K) in enumerate(shapes):
+        x = gu.dev(synth.activations(M, K, seed=700 + i))
+        single_a.append(qb.quantize_act(x, ws))
+        acts.append((x, gu.poison(torch.empty((M, K), dtype=torch.int8, device="cuda")),
+                     gu.poison(torch.empty(1, dtype=torch.float32, device="cuda")),
+                     gu.poison(torch.empty(M, dtype=torch.int32, device="cuda"))))
+    wshapes = [(24, 128, 4), (768, 768, 128), (264, 256, 11), (12, 384, 1), (96, 3072, 96)] * 8   # 40 matrices
+    for i, (N, K, G) in enumerate(wshapes):
+        bits = int(rng.choice(BITS))
+        w = gu.dev(synth.weights(N, K, seed=800 + i))
+        single_w.append(qb.quantize_pack_weights(w, bits, G, ws))
+        mats.append((w, bits, G, gu.poison(torch.empty((N, K * bits // 32), dtype=torch.int32, device="cuda")),
+                     gu.poison(torch.empty(G, dtype=torch.float32, device="cuda")),
+                     gu.poison(torch.empty(G, dtype=torch.float32, device="cuda"))))
+    ws2 = qb.workspace(groups=sum(m[2] for m in mats))
+    qb.quantize_act_batch(acts, ws2)
+    qb.quantize_pack_weights_batch(mats, ws2)
+    assert qb.read_status(ws2) == qb.QB_OK
+    for (x, xq, sc, rs), (xq1, sc1, rs1) in zip(acts, single_a):
+        assert torch.equal(xq, xq1) and torch.equal(sc, sc1) and torch.equal(rs, rs1)
+    for (w, bits, G, packed, delta, q0), (p1, d1, z1) in zip(mats, single_w):
+        assert torch.equal(packed, p1) and torch.equal(delta, d1) and torch.equal(q0, z1)
+    # a non-finite tensor in the middle of a batch is reported
+    bad = acts[7][0].clone()
+    bad[0, 3] = float("nan")
+    acts[7] = (bad,) + acts[7][1:]
+    ws3 = qb.workspace(groups=64)
+    qb.quantize_act_batch(acts, ws3)
+    assert qb.read_status(ws3) == qb.QB_ERR_NONFINITE
 
 
 def test_config1_encoder_layer_linears(ws):
