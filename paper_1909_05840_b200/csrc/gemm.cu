@@ -92,19 +92,31 @@ struct GemmCfg {
 // Bounded wait on an mbarrier phase.  Returns false if the wait expired or another role aborted.
 // The bound is counted in SM clock cycles (clock64 is a cheap register read; the global nanosecond
 // timer costs about a microsecond per read and would dominate short waits).
-__device__ __forceinline__ bool wait_barrier(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-#pragma unroll 1
-  for (int quick = 0; quick < 64; ++quick)
-    if (ptx::mbar_try_wait(bar, parity)) return true;
+// kSleep: the waiter is not on the critical path (it runs several stages ahead) and must not compete
+// for issue slots with the MMA issuer that shares its scheduler: it sleeps between polls.  A polling
+// warp is always "ready", so a handful of them starve the one thread that feeds the tensor cores.
+template <bool kSleep>
+__device__ __forceinline__ bool wait_barrier_t(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (ptx::mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
+  uint32_t ns = 32;
   for (uint32_t spin = 1;; ++spin) {
+    if (kSleep) {
+      __nanosleep(ns);
+      if (ns < 256) ns += ns;
+    }
     if (ptx::mbar_try_wait(bar, parity)) return true;
-    __nanosleep(32);
-    if ((spin & 255u) == 0u) {
+    if ((spin & 63u) == 0u) {
       if (*abort_flag) return false;
       if (clock64() - t0 > kWaitLimitCycles) return false;
     }
   }
+}
+__device__ __forceinline__ bool wait_barrier(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  return wait_barrier_t<false>(bar, parity, abort_flag);
+}
+__device__ __forceinline__ bool wait_barrier_relaxed(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  return wait_barrier_t<true>(bar, parity, abort_flag);
 }
 
 // Whole-warp wait: only lane 0 polls the barrier (hundreds of threads polling the same shared-memory
@@ -112,7 +124,7 @@ __device__ __forceinline__ bool wait_barrier(uint32_t bar, uint32_t parity, vola
 // the outcome is broadcast, and the shuffle orders the other lanes' later accesses after the wait.
 __device__ __forceinline__ bool wait_barrier_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   int ok = 1;
-  if ((threadIdx.x & 31) == 0) ok = wait_barrier(bar, parity, abort_flag) ? 1 : 0;
+  if ((threadIdx.x & 31) == 0) ok = wait_barrier_relaxed(bar, parity, abort_flag) ? 1 : 0;
   return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 
@@ -230,8 +242,9 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
   float* out_stage = reinterpret_cast<float*>(smem + kStages * Cfg::kStageBytes);
   const uint32_t bar_base = smem_base + kStages * Cfg::kStageBytes + Cfg::kOutStageBytes;
   uint8_t* bar_ptr = smem + kStages * Cfg::kStageBytes + Cfg::kOutStageBytes;
-  auto full_x = [&](int s) { return bar_base + 8u * s; };
-  auto full_w = [&](int s) { return bar_base + 8u * (kStages + s); };
+  // one "full" barrier per stage: the TMA producer's expect-tx arrival (+ the bytes) and one arrival per
+  // warp of the expander team that filled the weights; the issuer then needs a single wait per K block
+  auto full = [&](int s) { return bar_base + 8u * s; };
   auto empty = [&](int s) { return bar_base + 8u * (2 * kStages + s); };
   auto acc_full = [&](int a) { return bar_base + 8u * (3 * kStages + a); };
   auto acc_empty = [&](int a) { return bar_base + 8u * (3 * kStages + 2 + a); };
@@ -247,8 +260,7 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
-      ptx::mbar_init(full_x(s), 1);
-      ptx::mbar_init(full_w(s), 4);  // one arrival per warp of the team that filled the stage
+      ptx::mbar_init(full(s), 1 + 4);
       ptx::mbar_init(empty(s), 1);
     }
     for (int a = 0; a < 2; ++a) {
@@ -274,7 +286,7 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
 
   if (warp == 0) {
     // ---------------- TMA producer: token tiles -------------------------------------------------
-    if (lane == 0) {
+    if (ptx::elect_one()) {
       int stage = 0;
       uint32_t phase = 0;
       // The token tiles are first touched in DRAM by several CTAs at about the same time, and the
@@ -312,13 +324,13 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
           } else if (tm_nx != nullptr && ahead - k_blocks < kblocks_nx && ahead - k_blocks < kL2Ahead) {
             ptx::tma_prefetch_l2_2d(tm_nx, (ahead - k_blocks) * kBlockK, m0_nx);
           }
-          if (!wait_barrier(empty(stage), phase ^ 1u, abort_flag)) {
+          if (!wait_barrier_relaxed(empty(stage), phase ^ 1u, abort_flag)) {
             timed_out = true;
             where = (0 << 16) | stage;
             break;
           }
-          ptx::mbar_arrive_expect_tx(full_x(stage), Cfg::kXBytes);
-          ptx::tma_load_2d(stage_x(stage), tm, full_x(stage), kb * kBlockK, m0);
+          ptx::mbar_arrive_expect_tx(full(stage), Cfg::kXBytes);
+          ptx::tma_load_2d(stage_x(stage), tm, full(stage), kb * kBlockK, m0);
           if (++stage == kStages) {
             stage = 0;
             phase ^= 1u;
@@ -334,44 +346,60 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------------------------------------------------------
-    if (lane == 0) {
+    if (ptx::elect_one()) {
+      // This one thread must issue a K block's work in well under the 512 cycles the tensor cores need
+      // for it, and every instruction here is long-latency and serial.  So: one barrier wait per K
+      // block, and the loop is unrolled over the ring so that barrier addresses and both operand
+      // descriptors of a stage are compile-time offsets from loop-invariant values.
       constexpr uint32_t idesc = make_idesc_i8(kTileN, BT);
-      int stage = 0;
+      const uint64_t a_desc0 = make_kmajor_sw128_desc(stage_w(0));
+      const uint64_t b_desc0 = make_kmajor_sw128_desc(stage_x(0));
+      constexpr uint32_t kStageDescStep = Cfg::kStageBytes >> 4;  // start-address field counts 16-byte units
       uint32_t phase = 0;
-      int it = 0;
+      int it = 0, kb = 0, k_blocks = 0, a = 0;
+      uint32_t d_tmem = 0;
       TileCursor c{(int)blockIdx.x, 0};
-      for (; c.t < total_tiles && !timed_out; c.t += gridDim.x, ++it) {
-        c.seek(gp);
-        const int k_blocks = gp.prob[c.pi].K / kBlockK;
-        const int a = it & 1;
-        const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
-        if (!wait_barrier(acc_empty(a), aphase ^ 1u, abort_flag)) {
-          timed_out = true;
-          where = (1 << 16) | 0x100 | a;
-          break;
-        }
-        ptx::tcgen05_fence_after_sync();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(a * BT);
-        for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!wait_barrier(full_x(stage), phase, abort_flag) || !wait_barrier(full_w(stage), phase, abort_flag)) {
-            timed_out = true;
-            where = (1 << 16) | stage;
-            break;
-          }
-          ptx::tcgen05_fence_after_sync();
-          const uint64_t a_desc = make_kmajor_sw128_desc(stage_w(stage));
-          const uint64_t b_desc = make_kmajor_sw128_desc(stage_x(stage));
+      bool active = c.t < total_tiles;
+      while (active) {
 #pragma unroll
-          for (int j = 0; j < kBlockK / 32; ++j)  // 32 bytes of K per instruction: +2 in the address field
-            ptx::mma_i8_ss(d_tmem, a_desc + 2u * j, b_desc + 2u * j, idesc, (kb | j) != 0 ? 1u : 0u);
-          ptx::mma_commit(empty(stage));
-          if (++stage == kStages) {
-            stage = 0;
-            phase ^= 1u;
+        for (int stage = 0; stage < kStages; ++stage) {
+          if (active) {
+            if (kb == 0) {  // first K block of a tile: its problem, and a free accumulator
+              c.seek(gp);
+              k_blocks = gp.prob[c.pi].K / kBlockK;
+              a = it & 1;
+              const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
+              if (!wait_barrier(acc_empty(a), aphase ^ 1u, abort_flag)) {
+                timed_out = true;
+                where = (1 << 16) | 0x100 | a;
+                active = false;
+              }
+              d_tmem = tmem_base + (uint32_t)(a * BT);
+            }
+            if (active && !wait_barrier(full(stage), phase, abort_flag)) {
+              timed_out = true;
+              where = (1 << 16) | stage;
+              active = false;
+            }
+            if (active) {
+              ptx::tcgen05_fence_after_sync();
+              const uint64_t a_desc = a_desc0 + (uint64_t)(stage * kStageDescStep);
+              const uint64_t b_desc = b_desc0 + (uint64_t)(stage * kStageDescStep);
+#pragma unroll
+              for (int j = 0; j < kBlockK / 32; ++j)  // 32 bytes of K per instruction: +2 in the address field
+                ptx::mma_i8_ss(d_tmem, a_desc + 2u * j, b_desc + 2u * j, idesc, j != 0 ? 1u : (kb != 0 ? 1u : 0u));
+              ptx::mma_commit(empty(stage));
+              if (++kb == k_blocks) {  // tile done: hand the accumulator to the epilogue
+                ptx::mma_commit(acc_full(a));
+                kb = 0;
+                ++it;
+                c.t += gridDim.x;
+                active = c.t < total_tiles;
+              }
+            }
           }
         }
-        if (timed_out) break;
-        ptx::mma_commit(acc_full(a));
+        phase ^= 1u;
       }
       if (timed_out) {
         // wait (bounded) for the MMAs already issued before tensor memory is freed
@@ -475,7 +503,7 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
       }
       ptx::fence_proxy_async_smem();  // every lane: its own stores -> visible to the tensor cores
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(full_w(stage));
+      if (lane == 0) ptx::mbar_arrive(full(stage));
       stage += kExpandTeams;
       if (stage >= kStages) {
         stage -= kStages;
