@@ -82,10 +82,10 @@ template <int BT>
 struct GemmCfg {
   static constexpr int kXBytes = BT * kBlockK;
   static constexpr int kStageBytes = kWBytes + kXBytes;
-  static constexpr int kStages = (BT == 256) ? 4 : 6;
+  static constexpr int kStages = (BT == 256) ? 3 : 5;
   static constexpr int kTmemCols = 2 * BT;
   static constexpr int kBarBytes = 256 + 2 * 256 * 4;  // barriers + two row-sum tiles
-  static constexpr int kOutStageBytes = kEpilogueWarps * 32 * 32 * 4;  // per epilogue warp: 32 tokens x 32 neurons fp32
+  static constexpr int kOutStageBytes = kEpilogueWarps * 2 * 32 * 32 * 4;  // per epilogue warp: two buffers of 32 tokens x 32 neurons fp32
   static constexpr int kSmemBytes = kStages * kStageBytes + kOutStageBytes + kBarBytes;
 };
 
@@ -516,6 +516,7 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
     const int r = quarter * 32 + lane;         // output neuron inside the tile
     constexpr int c_code = 1 << (BITS - 1);
     int it = 0;
+    int out_flip = 0;
     TileCursor c{(int)blockIdx.x, 0};
     for (; c.t < total_tiles && !timed_out; c.t += gridDim.x, ++it) {
       c.seek(gp);
@@ -558,7 +559,7 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
       ptx::tcgen05_fence_after_sync();
       const uint32_t t_base = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * BT);
       const int n_chunks = min(BT / 32, (pM - m0 + 31) / 32);  // chunks of 32 tokens, warp-uniform
-      float* buf = out_stage + (warp - kFirstEpilogueWarp) * (32 * 32);
+      float* const warp_bufs = out_stage + (warp - kFirstEpilogueWarp) * (2 * 32 * 32);
       const int x0 = n_base + quarter * 32;
       // the two warps of a lane quarter take alternate chunks
 #pragma unroll 1
@@ -569,6 +570,8 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
         ptx::tmem_ld_regs_ready(v);
         const int mc = m0 + ch * 32;
         const float4* rs4 = reinterpret_cast<const float4*>(rs_tile + a * 256 + ch * 32);
+        float* buf = warp_bufs + (out_flip & 1) * (32 * 32);  // alternate between the warp's two staging buffers
+        ++out_flip;
         if (tma_store) {
           // 32 tokens x 32 neurons of this warp -> shared memory [token][neuron] -> one TMA store.
           // Lanes write consecutive words of a row: conflict-free.  Rows past M and neurons past N
@@ -591,7 +594,7 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
               yv[j] = __fmaf_rn(alpha, (float)ac, __fmaf_rn(beta, rsv[j], b));
             }
             if (h == 0) {
-              if (lane == 0) ptx::tma_store_wait_read0();  // this warp's previous store has read the buffer
+              if (lane == 0) ptx::tma_store_wait_read1();  // the store before last (same buffer) has read it
               __syncwarp();
             }
 #pragma unroll
