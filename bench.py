@@ -311,13 +311,8 @@ def run_ours(args, wl):
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
     sync_all()
     t_wall0 = time.time()
-    evf = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
     for i in range(args.steps):
-        if i == args.steps // 2:
-            evf[0].record()
         flush.fill_(i & 0xFF)                # untimed: evict the previous step's tensors from L2
-        if i == args.steps // 2:
-            evf[1].record()
         ev[i][0].record(); phase_act()
         ev[i][1].record(); phase_weights()
         ev[i][2].record(); phase_gemm()
@@ -356,7 +351,6 @@ def run_ours(args, wl):
     sync_all()
     ms_e2e = e0.elapsed_time(e1) / e2e_steps
 
-    write_stream_gbs = flush.numel() / (evf[0].elapsed_time(evf[1]) * 1e-3) / 1e9
     probe_tops, probe_cycles = qb.probe_i8_mma(256, 20000)
     ops = gemm_ops(wl)
     ms_job, ops_job = aggregate_over_ranks(ms_step, ops, world, dist, device)
@@ -393,8 +387,6 @@ def run_ours(args, wl):
         "linears_per_step": len(lin),
         "probed_int8_tops": probe_tops, "probed_cycles_per_k_block": probe_cycles,
         "frac_of_probed_int8": achieved_tops / probe_tops,
-        "write_stream_gbs": write_stream_gbs,
-        "write_stream_note": "a 512 MiB device fill timed in the same run: what a write-only stream sustains",
     })
 
     line = {
