@@ -443,12 +443,93 @@ def cpu_baseline(wl, args):
                       f"{reps} repetitions, {dt * 1e3:.1f} ms each"}
 
 
+def run_quantizer_sweep(args):
+    """Config 4: qb_quantize_pack_weights over a 109,117,440-parameter set of BERT-base-shaped matrices
+    for k in {2,3,4,8} x groups in {1,12,128,768}, and qb_quantize_act on a 24576 x 4096 tensor; GB/s of
+    algorithmic bytes against the measured HBM peak.  Single GPU; one JSON line."""
+    import torch
+    import paper_1909_05840_b200 as qb
+    from paper_1909_05840_b200 import build as qb_build
+    qb_build.build()
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    peaks, peak_kind = measured_peaks()
+    shapes = synth.quantizer_sweep_shapes()
+    params = sum(n * k for n, k in shapes)
+    distinct = {}
+    for i, (n, k) in enumerate(shapes):   # one host array per distinct shape, device copies per matrix
+        if (n, k) not in distinct:
+            distinct[(n, k)] = torch.from_numpy(synth.weights(n, k, synth.seed_for(4, 0, len(distinct))))
+    w_dev = [distinct[s].to(dev) for s in shapes]
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    steps = max(3, min(args.steps, 20))
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            fn()
+        ts = []
+        for i in range(steps):
+            flush.fill_(i & 0xFF)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); g.replay(); e1.record()
+            torch.cuda.synchronize(dev)
+            ts.append(e0.elapsed_time(e1))
+        return float(np.median(ts))
+
+    table = {}
+    launches = 0
+    for bits in synth.BITS_CHOICES:
+        for groups in (1, 12, 128, 768):
+            ws = qb.workspace(groups=max(32, groups * len(shapes)), device=dev)
+            items = [(w, bits, groups, torch.empty((w.shape[0], w.shape[1] * bits // 32), dtype=torch.int32, device=dev),
+                      torch.empty(groups, dtype=torch.float32, device=dev),
+                      torch.empty(groups, dtype=torch.float32, device=dev)) for w in w_dev]
+            arr = qb.make_weight_desc_array(items)
+            ms = timed(lambda: qb.quantize_pack_weights_batch(arr, ws))
+            assert qb.read_status(ws) == qb.QB_OK
+            gbs = params * (4.0 + bits / 8.0) / (ms * 1e-3) / 1e9
+            table[f"k{bits}_g{groups}"] = {"ms": ms, "GBps": gbs, "frac_hbm": gbs / peaks["hbm_gbs"]}
+            launches += 2 * -(-len(shapes) // 32) * (3 + steps)
+            del items, arr
+    M, K = synth.QUANTIZER_SWEEP_ACT
+    x = torch.from_numpy(synth.activations(M, K, synth.seed_for(4))).to(dev)
+    xq = torch.empty((M, K), dtype=torch.int8, device=dev)
+    sc = torch.empty(1, dtype=torch.float32, device=dev)
+    rs = torch.empty(M, dtype=torch.int32, device=dev)
+    ws = qb.workspace(groups=64, device=dev)
+    ms_act = timed(lambda: qb.quantize_act(x, ws, xq, sc, rs))
+    act_gbs = (9.0 * M * K + 4 * M) / (ms_act * 1e-3) / 1e9
+    best = max(table.values(), key=lambda r: r["frac_hbm"])
+    line = {
+        "metric": METRIC, "value": act_gbs, "unit": "GB/s", "n_gpus": 1, "steps": steps, "warmup": 3,
+        "ms_per_step": ms_act, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": "quantizer sweep: 109,117,440-parameter BERT-base-shaped weight set, k x groups; "
+                               "activations 24576 x 4096", "config_index": 4,
+                   "l2": "512 MiB flush write before every timed call (untimed)",
+                   "launch": "one C-ABI batch call captured in a CUDA graph, replayed"},
+        "gpu_launches": launches + 2 * (3 + steps),
+        "roofline": {"bound": "hbm", "achieved": act_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": act_gbs / peaks["hbm_gbs"], "traffic": None, "kernel": "act_absmax_kernel + act_quantize_kernel",
+                     "algorithmic_bytes_per_launch": 9.0 * M * K + 4 * M, "peak_source": peak_kind,
+                     "note": "9 B per element: the per-tensor maximum forces two reads of a 403 MB tensor"},
+        "quantize_act": {"ms": ms_act, "GBps": act_gbs, "frac_hbm": act_gbs / peaks["hbm_gbs"],
+                         "useful_5B_per_element_GBps": 5.0 * M * K / (ms_act * 1e-3) / 1e9},
+        "quantize_pack_weights": table,
+        "quantize_pack_weights_best_frac_hbm": best["frac_hbm"],
+    }
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--config", type=int, default=1, help="workload index 0-3 (see synth.workload)")
+    ap.add_argument("--config", type=int, default=1, help="workload index 0-3 (see synth.workload); 4 = quantizer sweep")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--ref-rows", type=int, default=256, help="token rows of the oracle's bounded sample")
     ap.add_argument("--ref-steps", type=int, default=5)
@@ -458,6 +539,13 @@ def main():
     ap.add_argument("--busy-ms", type=float, default=300.0,
                     help="untimed load before the timed steps so that clocks are sampled under load")
     args = ap.parse_args()
+    if args.config == 4:
+        if args.impl == "reference" or int(os.environ.get("RANK", "0")) != 0:
+            if int(os.environ.get("RANK", "0")) == 0:
+                print(json.dumps({"impl": "reference", "unavailable": "the quantizer sweep has no reference arm; use --config 0..3"}))
+            return
+        run_quantizer_sweep(args)
+        return
     wl = synth.workload(args.config)
     if args.impl == "reference":
         run_reference(args, wl)
