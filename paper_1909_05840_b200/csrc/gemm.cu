@@ -50,7 +50,9 @@ constexpr int kBlockK = 128;         // K elements (= bytes) per pipeline stage
 constexpr int kWBytes = kTileN * kBlockK;
 constexpr long long kWaitLimitCycles = 4000000000ll;  // about 2 s at 2 GHz
 
-constexpr int kMaxProblems = 16;  // linears per launch (all in kernel-parameter space, no device table)
+constexpr int kMaxProblems = 16;
+constexpr int kMaxOrder = 4096;   // entries of the explicit tile visiting order (when it is used)
+constexpr uint16_t kNoTile = 0xFFFF;  // linears per launch (all in kernel-parameter space, no device table)
 
 // One linear of a launch.
 struct Problem {
@@ -76,6 +78,12 @@ struct GroupedParams {
   void* ws;
   int32_t count;
   int32_t total_tiles;
+  // Visiting order.  Position p is visited by CTA p % gridDim.x.  Without `use_order` position p is tile
+  // p; with it, order[p] is the tile (or kNoTile): the host balances tiles of unequal length (K) over
+  // the CTAs instead of dealing them round-robin.
+  int32_t total_positions;
+  int32_t use_order;
+  uint16_t order[kMaxOrder];
 };
 
 template <int BT>
@@ -216,12 +224,34 @@ __device__ __forceinline__ void load_item(const uint32_t* __restrict__ src, uint
   }
 }
 
-// Position of a role in the launch's tile list: global tile t -> problem, tile coordinates.
+// A role's walk over the tiles of its CTA: positions blockIdx.x, + gridDim.x, ... of the visiting order.
 struct TileCursor {
-  int t;   // global tile index (blockIdx.x, + gridDim.x, ...)
+  int p;   // position
+  int t;   // tile at that position
   int pi;  // problem that owns tile t
-  __device__ __forceinline__ void seek(const GroupedParams& gp) {
+  __device__ __forceinline__ void start() {
+    p = (int)blockIdx.x - (int)gridDim.x;
+    t = 0;
+    pi = 0;
+  }
+  // move to the CTA's next tile; false when there is none
+  __device__ __forceinline__ bool next(const GroupedParams& gp) {
+    for (;;) {
+      p += (int)gridDim.x;
+      if (p >= gp.total_positions) return false;
+      if (!gp.use_order) {
+        t = p;
+        break;
+      }
+      const uint16_t e = gp.order[p];
+      if (e != kNoTile) {
+        t = (int)e;
+        break;
+      }
+    }
+    pi = 0;
     while (pi + 1 < gp.count && t >= gp.prob[pi + 1].tile_begin) ++pi;
+    return true;
   }
 };
 
@@ -280,7 +310,6 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
   ptx::tcgen05_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
-  const int total_tiles = gp.total_tiles;
   bool timed_out = false;
   int where = 0;
 
@@ -293,25 +322,25 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
       // ring holds only a few K blocks: L2 prefetches run kL2Ahead blocks ahead of the loads (into the
       // CTA's next tile when the current one ends) so that the loads themselves hit L2.
       constexpr int kL2Ahead = 8;
-      TileCursor c{(int)blockIdx.x, 0};
-      if (c.t < total_tiles) {
-        c.seek(gp);
+      TileCursor c;
+      c.start();
+      bool have = c.next(gp);
+      if (have) {
         const Problem& pr = gp.prob[c.pi];
         const int m0 = ((c.t - pr.tile_begin) / pr.n_tiles) * BT;
         for (int kb = 0; kb < kL2Ahead && kb < pr.K / kBlockK; ++kb) ptx::tma_prefetch_l2_2d(&gp.tmx[c.pi], kb * kBlockK, m0);
       }
-      for (; c.t < total_tiles && !timed_out; c.t += gridDim.x) {
-        c.seek(gp);
+      while (have && !timed_out) {
         const Problem& pr = gp.prob[c.pi];
         const int m0 = ((c.t - pr.tile_begin) / pr.n_tiles) * BT;
         const int k_blocks = pr.K / kBlockK;
         const CUtensorMap* tm = &gp.tmx[c.pi];
         // the CTA's next tile, for prefetches that run past the end of this one
-        TileCursor nx{c.t + (int)gridDim.x, c.pi};
+        TileCursor nx = c;
+        const bool have_nx = nx.next(gp);
         const CUtensorMap* tm_nx = nullptr;
         int m0_nx = 0, kblocks_nx = 0;
-        if (nx.t < total_tiles) {
-          nx.seek(gp);
+        if (have_nx) {
           const Problem& pn = gp.prob[nx.pi];
           tm_nx = &gp.tmx[nx.pi];
           m0_nx = ((nx.t - pn.tile_begin) / pn.n_tiles) * BT;
@@ -336,6 +365,8 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
             phase ^= 1u;
           }
         }
+        c = nx;
+        have = have_nx;
       }
       if (timed_out) {
         // let copies already in flight land before the CTA's shared memory is released
@@ -358,14 +389,14 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
       uint32_t phase = 0;
       int it = 0, kb = 0, k_blocks = 0, a = 0;
       uint32_t d_tmem = 0;
-      TileCursor c{(int)blockIdx.x, 0};
-      bool active = c.t < total_tiles;
+      TileCursor c;
+      c.start();
+      bool active = c.next(gp);
       while (active) {
 #pragma unroll
         for (int stage = 0; stage < kStages; ++stage) {
           if (active) {
             if (kb == 0) {  // first K block of a tile: its problem, and a free accumulator
-              c.seek(gp);
               k_blocks = gp.prob[c.pi].K / kBlockK;
               a = it & 1;
               const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
@@ -393,8 +424,7 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
                 ptx::mma_commit(acc_full(a));
                 kb = 0;
                 ++it;
-                c.t += gridDim.x;
-                active = c.t < total_tiles;
+                active = c.next(gp);
               }
             }
           }
@@ -420,13 +450,13 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
     const int piece = i_team & 3;
     const int row0 = i_team >> 2;
     // fetch cursor: tile, K block inside it, and the tile's weight rows
-    TileCursor c{(int)blockIdx.x, 0};
+    TileCursor c;
+    c.start();
     int ld_kb = team;
     int ld_kblocks = 0, ld_n0 = 0, ld_N = 0, ld_wpr = 0;
     const uint32_t* ld_packed = nullptr;
-    bool ld_done = c.t >= total_tiles;
+    bool ld_done = !c.next(gp);
     auto enter_tile = [&]() {  // fields of the tile the cursor stands on
-      c.seek(gp);
       const Problem& pr = gp.prob[c.pi];
       ld_kblocks = pr.K / kBlockK;
       ld_n0 = ((c.t - pr.tile_begin) % pr.n_tiles) * kTileN;
@@ -437,8 +467,7 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
     auto normalize = [&]() {  // carry ld_kb over tile ends
       while (!ld_done && ld_kb >= ld_kblocks) {
         ld_kb -= ld_kblocks;
-        c.t += gridDim.x;
-        if (c.t >= total_tiles) {
+        if (!c.next(gp)) {
           ld_done = true;
         } else {
           enter_tile();
@@ -517,9 +546,9 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
     constexpr int c_code = 1 << (BITS - 1);
     int it = 0;
     int out_flip = 0;
-    TileCursor c{(int)blockIdx.x, 0};
-    for (; c.t < total_tiles && !timed_out; c.t += gridDim.x, ++it) {
-      c.seek(gp);
+    TileCursor c;
+    c.start();
+    for (; !timed_out && c.next(gp); ++it) {
       const Problem& pr = gp.prob[c.pi];
       const CUtensorMap* tmy = &gp.tmy[c.pi];
       const int local = c.t - pr.tile_begin;
@@ -808,6 +837,42 @@ static qb_status launch_group(const qb_linear_desc* d, const int* idx, int count
   }
   gp.total_tiles = tile;
   const int grid = tile < sm_count ? tile : sm_count;
+  gp.total_positions = tile;
+  gp.use_order = 0;
+  // Tiles of different problems differ in length (K blocks).  When the launch is small enough for the
+  // table, deal the tiles longest first to the least loaded CTA instead of round-robin.
+  {
+    bool uniform = true;
+    for (int i = 1; i < count; ++i) uniform = uniform && gp.prob[i].K == gp.prob[0].K;
+    if (!uniform && tile <= kMaxOrder && tile < (int)kNoTile) {
+      constexpr int kEpilogueCost = 5;  // a tile's fixed cost in units of one K block
+      std::vector<int> ids(tile), cost(tile);
+      for (int i = 0, t = 0; i < count; ++i)
+        for (int j = 0; j < gp.prob[i].n_tiles * gp.prob[i].m_tiles; ++j, ++t) {
+          ids[t] = t;
+          cost[t] = gp.prob[i].K / kBlockK + kEpilogueCost;
+        }
+      std::stable_sort(ids.begin(), ids.end(), [&](int a, int b) { return cost[a] > cost[b]; });
+      std::vector<std::vector<int>> lists(grid);
+      std::vector<long long> load(grid, 0);
+      size_t max_len = 0;
+      for (int t : ids) {
+        int best = 0;
+        for (int c = 1; c < grid; ++c)
+          if (load[c] < load[best]) best = c;
+        lists[best].push_back(t);
+        load[best] += cost[t];
+        if (lists[best].size() > max_len) max_len = lists[best].size();
+      }
+      if (max_len * (size_t)grid <= (size_t)kMaxOrder) {
+        for (size_t i = 0; i < max_len; ++i)
+          for (int c = 0; c < grid; ++c)
+            gp.order[i * grid + c] = i < lists[c].size() ? (uint16_t)lists[c][i] : kNoTile;
+        gp.total_positions = (int32_t)(max_len * grid);
+        gp.use_order = 1;
+      }
+    }
+  }
   return bt == 256 ? launch_group_bits<256>(bits, gp, grid, stream) : launch_group_bits<128>(bits, gp, grid, stream);
 }
 
