@@ -17,6 +17,12 @@
 #include <vector>
 
 #include "common.cuh"
+#include "ptx.cuh"
+
+#ifndef FUSED_WARPS
+#define FUSED_WARPS 16
+#define FUSED_RING_KB 192
+#endif
 
 namespace qb {
 
@@ -180,25 +186,21 @@ struct GroupParams {
   float lo, hi, inv;
 };
 
-// Range of group g -> (q0, qmax, 1/Delta); lane-uniform.  Also publishes Delta and q0 once.
-__device__ __forceinline__ GroupParams load_group(int g, int bits_levels, const uint32_t* __restrict__ hi_enc,
-                                                  const uint32_t* __restrict__ lo_inv,
-                                                  const float* __restrict__ range_lo,
-                                                  const float* __restrict__ range_hi, float* __restrict__ delta,
-                                                  float* __restrict__ q0, bool publish, void* ws) {
+// Range [lo, hi] of group g -> (q0, qmax, 1/Delta); lane-uniform.  Publishes Delta and q0 if asked.
+// A caller-supplied range must be finite and ordered; a constant group gets Delta = 1, all codes 0.
+__device__ __forceinline__ GroupParams finish_group(float lo, float hi, bool from_caller, int bits_levels, int g,
+                                                    float* __restrict__ delta, float* __restrict__ q0,
+                                                    bool publish, void* ws) {
   GroupParams p;
-  if (range_lo != nullptr) {
-    p.lo = __ldg(range_lo + g);
-    p.hi = __ldg(range_hi + g);
+  p.lo = lo;
+  p.hi = hi;
+  if (from_caller) {
     const bool bad = !(fabsf(p.lo) <= 3.402823466e38f) || !(fabsf(p.hi) <= 3.402823466e38f) || p.hi < p.lo;
     if (bad) {
       if (publish) report_status(ws, QB_ERR_NONFINITE);
       p.lo = 0.0f;
       p.hi = 0.0f;
     }
-  } else {
-    p.hi = ordered_to_float(hi_enc[g]);
-    p.lo = ordered_to_float(~lo_inv[g]);
   }
   float d = __fdiv_rn(__fsub_rn(p.hi, p.lo), (float)bits_levels);
   float inv = __fdiv_rn(1.0f, d);
@@ -215,13 +217,57 @@ __device__ __forceinline__ GroupParams load_group(int g, int bits_levels, const 
   return p;
 }
 
+// Group g of a matrix: range from the caller's tables or from the reduced encodings in the workspace.
+__device__ __forceinline__ GroupParams load_group(int g, int bits_levels, const uint32_t* __restrict__ hi_enc,
+                                                  const uint32_t* __restrict__ lo_inv,
+                                                  const float* __restrict__ range_lo,
+                                                  const float* __restrict__ range_hi, float* __restrict__ delta,
+                                                  float* __restrict__ q0, bool publish, void* ws) {
+  if (range_lo != nullptr)
+    return finish_group(__ldg(range_lo + g), __ldg(range_hi + g), true, bits_levels, g, delta, q0, publish, ws);
+  return finish_group(ordered_to_float(~lo_inv[g]), ordered_to_float(hi_enc[g]), false, bits_levels, g, delta, q0,
+                      publish, ws);
+}
+
+// Four codes of this lane (Appendix A's Q: clamp, subtract q0, scale by 1/Delta, round half to even)
+// and the output word `lane` of the unit of 128 codes, gathered from the lanes whose 4k-bit fields
+// overlap stream bits [32*lane, 32*lane + 32).  Lanes >= 4k return a word nobody stores.
+template <int BITS>
+__device__ __forceinline__ uint32_t pack_unit(const float4 v, const GroupParams& gp, int lane, int first_src) {
+  constexpr int L = (1 << BITS) - 1;
+  constexpr int F = 4 * BITS;
+  constexpr int NSRC = BITS == 8 ? 1 : (BITS == 4 ? 2 : 4);
+  const float e[4] = {v.x, v.y, v.z, v.w};
+  uint32_t field = 0;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float xc = fminf(fmaxf(e[i], gp.lo), gp.hi);        // Clamp(X, q0, qmax)
+    const float t = __fmul_rn(__fsub_rn(xc, gp.lo), gp.inv);  // (X' - q0) * (1/Delta)
+    int c = __float2int_rn(t);                                // round half to even
+    c = min(max(c, 0), L);
+    field |= (uint32_t)c << (BITS * i);
+  }
+  uint32_t word = 0;
+#pragma unroll
+  for (int s = 0; s < NSRC; ++s) {
+    const int src = first_src + s;
+    const uint32_t f = __shfl_sync(0xffffffffu, field, src & 31);
+    const int off = src * F - 32 * lane;  // position of that field relative to the word
+    if (off >= 0) {
+      if (off < 32) word |= f << off;
+    } else {
+      word |= f >> (-off);
+    }
+  }
+  return word;
+}
+
 template <int BITS>
 __global__ void __launch_bounds__(kWqThreads)
 weight_pack_kernel(const __grid_constant__ WeightBatch b) {
   constexpr int L = (1 << BITS) - 1;
   constexpr int F = 4 * BITS;          // bits contributed by one lane (four codes)
   constexpr int WORDS = 4 * BITS;      // output words per unit of 128 codes
-  constexpr int NSRC = BITS == 8 ? 1 : (BITS == 4 ? 2 : 4);
   const int lane = threadIdx.x & 31;
   const int64_t gwarp = (int64_t)blockIdx.x * kWqWarps + (threadIdx.x >> 5);
   int64_t u = gwarp * b.units_per_warp;
@@ -260,34 +306,377 @@ weight_pack_kernel(const __grid_constant__ WeightBatch b) {
           const int gl = cur_g - group_begin;
           gp = load_group(gl, L, b.hi_enc + group_begin, b.lo_inv + group_begin, rlo, rhi, dl, qz, publish, b.ws);
         }
-        const float e[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
-        uint32_t field = 0;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float xc = fminf(fmaxf(e[i], gp.lo), gp.hi);            // Clamp(X, q0, qmax)
-          const float t = __fmul_rn(__fsub_rn(xc, gp.lo), gp.inv);      // (X' - q0) * (1/Delta)
-          int c = __float2int_rn(t);                                    // round half to even
-          c = min(max(c, 0), L);
-          field |= (uint32_t)c << (BITS * i);
-        }
-        // word `lane` of this unit collects the fields that overlap its 32 bits
-        uint32_t word = 0;
-#pragma unroll
-        for (int s = 0; s < NSRC; ++s) {
-          const int src = first_src + s;
-          const uint32_t f = __shfl_sync(0xffffffffu, field, src & 31);
-          const int off = src * F - 32 * lane;  // position of that field relative to the word
-          if (off >= 0) {
-            if (off < 32) word |= f << off;
-          } else {
-            word |= f >> (-off);
-          }
-        }
+        const uint32_t word = pack_unit<BITS>(v[j], gp, lane, first_src);
         if (lane < WORDS) out_base[j * WORDS + lane] = word;
         pos.advance(b);
       }
     }
     u += nload;
+  }
+}
+
+// ---- single-read path ------------------------------------------------------------------------------
+// When a whole group fits in shared memory the matrix is read from HBM once.  A persistent CTA per SM
+// takes groups round-robin.  Four producer lanes (in warps of their own) stream the CTA's groups as bulk
+// copies into a ring of shared-memory slots, running ahead into the next groups.  The sixteen consumer warps form teams of
+// 1, 2, 4, 8 or 16 warps (small groups: many small teams); the CTA's groups go to the teams in turn, so
+// one team reduces a range while another packs.  A team takes the range of its group from shared
+// memory as the chunks land, agrees on it through its named barrier, then quantizes the group from
+// shared memory in blocks of 8 units: the 4k-bit fields of a block are laid down in element order in
+// the warp's staging area, which for k = 2, 4, 8 is already the packed stream (copied out with 16-byte
+// stores) and for k = 3 is regrouped (eight 12-bit fields -> three words) on the way out.
+constexpr int kFusedConsumerWarps = FUSED_WARPS;
+constexpr int kFusedProducers = 4;                              // producer warps (one lane each issues copies)
+constexpr int kFusedThreads = 32 * (kFusedConsumerWarps + kFusedProducers);
+constexpr int kRingBytes = FUSED_RING_KB * 1024;
+constexpr int kMaxRingSlots = kRingBytes / 4096;               // 4 KB slots, or a quarter as many of 16 KB
+constexpr int kFusedMaxGroupUnits = kRingBytes / 512;           // 384 units = 49,152 weights per group
+constexpr int kStagingBytes = kFusedConsumerWarps * 1024;       // per consumer warp: fields of one block
+constexpr int kTailBarriers = 0;                                // full[kMaxRingSlots], empty[kMaxRingSlots]
+constexpr int kTailScratch = 16 * kMaxRingSlots;                // s_hi, s_lo: [2][kFusedConsumerWarps] each
+constexpr int kTailFlags = kTailScratch + 16 * kFusedConsumerWarps;  // abort flag, then issued[kMaxRingSlots]
+constexpr int kFusedTailBytes = (kTailFlags + 8 + 4 * kMaxRingSlots + 127) / 128 * 128;
+constexpr int kFusedSmemBytes = kRingBytes + kStagingBytes + kFusedTailBytes;
+constexpr long long kFusedWaitLimit = 4000000000ll;             // SM cycles, about 2 s
+
+struct FusedBatch {
+  WeightItem item[kMaxWeightBatch];
+  void* ws;
+  int32_t total_groups;
+  int32_t count;
+  int32_t team_warps;   // 1, 2, 4, 8 or 16
+  int32_t chunk_units;  // units of 128 weights per ring slot: 8 or 32
+  int32_t n_slots;      // kRingBytes / (chunk_units * 512)
+};
+
+// Bounded wait on an mbarrier phase; false when it expired (or, if asked, when another role gave up).
+__device__ __forceinline__ bool fused_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (ptx::mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (uint32_t spin = 1;; ++spin) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    if ((spin & 1023u) == 0u) {
+      if (abort_flag != nullptr && *abort_flag) return false;
+      if (clock64() - t0 > kFusedWaitLimit) return false;
+    }
+  }
+}
+
+// Bounded wait until a slot has been issued more than `index` times (`issued` is the slot's counter).
+__device__ __forceinline__ bool wait_issued(volatile int* issued, int index, volatile int* abort_flag) {
+  if (*issued > index) {
+    __threadfence_block();
+    return true;
+  }
+  const long long t0 = clock64();
+  for (uint32_t spin = 1;; ++spin) {
+    if (*issued > index) {
+      __threadfence_block();
+      return true;
+    }
+    if ((spin & 1023u) == 0u && (*abort_flag || clock64() - t0 > kFusedWaitLimit)) return false;
+  }
+}
+
+// Barrier over the threads of a team that also ORs a predicate over them: every thread gets the same
+// answer, so all of them leave the group loop together.  A one-warp team needs no named barrier.
+__device__ __forceinline__ bool team_sync_or(bool pred, int team_warps, int bar_id) {
+  if (team_warps == 1) return __any_sync(0xffffffffu, pred) != 0;
+  uint32_t res;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.or.pred p, %2, %3, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(res)
+      : "r"((uint32_t)pred), "r"(bar_id), "r"(32 * team_warps)
+      : "memory");
+  return res != 0;
+}
+
+// min / max that return NaN when an input is NaN, so a single NaN survives to the group's range
+__device__ __forceinline__ float min_nan(float a, float b) {
+  float d;
+  asm("min.NaN.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+  return d;
+}
+__device__ __forceinline__ float max_nan(float a, float b) {
+  float d;
+  asm("max.NaN.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+  return d;
+}
+
+// Four codes of one float4 as a 4k-bit field (code i at bits [k*i, k*i + k)).  Adding 1.5 * 2^23 rounds
+// (X' - q0) * (1/Delta) to an integer, half to even, and leaves it in the low mantissa bits; the four bit
+// patterns are combined with integer multiply-adds and the constant they carry is taken off once.
+// With a range that covers the data no clamp is needed: 0 <= t <= L (1 + 3 * 2^-24) rounds into [0, L].
+template <int BITS, bool kClamp>
+__device__ __forceinline__ uint32_t quant_field(const float4 v, const GroupParams& gp) {
+  constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23, bit pattern 0x4B400000
+  constexpr uint32_t kCarry = 0x4B400000u * (1u + (1u << BITS) + (1u << (2 * BITS)) + (1u << (3 * BITS)));
+  const float e[4] = {v.x, v.y, v.z, v.w};
+  uint32_t bits[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float x = e[i];
+    if (kClamp) x = fminf(fmaxf(x, gp.lo), gp.hi);                    // Clamp(X, q0, qmax)
+    const float t = __fmul_rn(__fsub_rn(x, gp.lo), gp.inv);          // (X' - q0) * (1/Delta)
+    bits[i] = __float_as_uint(__fadd_rn(t, kMagic));                  // round half to even
+  }
+  uint32_t f = bits[0] + (bits[1] << BITS) + (bits[2] << (2 * BITS)) + (bits[3] << (3 * BITS)) - kCarry;
+  if constexpr (BITS < 8) f &= (1u << (4 * BITS)) - 1u;
+  return f;
+}
+
+// A block of `nu` <= 8 units (1024 weights) that starts at `blk` in shared memory: quantize it and
+// write its packed words to `out` (the words of the block's first unit).  One warp; `stg` is the
+// warp's own 1 KB staging area, where the 4k-bit fields are laid down in element order.
+template <int BITS, bool kClamp>
+__device__ __forceinline__ void pack_block(const uint8_t* blk, uint8_t* stg, int nu, const GroupParams& gp,
+                                           uint32_t* __restrict__ out, int lane) {
+  const float4* src = reinterpret_cast<const float4*>(blk);
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    float4 v[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      if (4 * h + j < nu) v[j] = src[(4 * h + j) * 32 + lane];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (4 * h + j < nu) {
+        const uint32_t f = quant_field<BITS, kClamp>(v[j], gp);
+        const int fi = (4 * h + j) * 32 + lane;  // field index = element index / 4
+        if (BITS == 8) reinterpret_cast<uint32_t*>(stg)[fi] = f;
+        if (BITS == 4 || BITS == 3) reinterpret_cast<uint16_t*>(stg)[fi] = (uint16_t)f;
+        if (BITS == 2) stg[fi] = (uint8_t)f;
+      }
+    }
+  }
+  __syncwarp();
+  if (BITS == 3) {
+    // item = 32 codes = eight 12-bit fields held in 16-bit cells -> three words
+    if (lane < 4 * nu) {
+      const uint4 q = reinterpret_cast<const uint4*>(stg)[lane];
+      const uint32_t f0 = q.x & 0xffffu, f1 = q.x >> 16, f2 = q.y & 0xffffu, f3 = q.y >> 16;
+      const uint32_t f4 = q.z & 0xffffu, f5 = q.z >> 16, f6 = q.w & 0xffffu, f7 = q.w >> 16;
+      uint32_t* o = out + lane * 3;
+      o[0] = f0 | (f1 << 12) | (f2 << 24);
+      o[1] = (f2 >> 8) | (f3 << 4) | (f4 << 16) | (f5 << 28);
+      o[2] = (f5 >> 4) | (f6 << 8) | (f7 << 20);
+    }
+  } else {
+    const int n16 = nu * BITS;  // 16 * BITS bytes per unit
+    const uint4* pk = reinterpret_cast<const uint4*>(stg);
+    uint4* o = reinterpret_cast<uint4*>(out);
+    for (int i = lane; i < n16; i += 32) o[i] = pk[i];
+  }
+  __syncwarp();  // the staging area is free again
+}
+
+template <int BITS>
+__global__ void __launch_bounds__(kFusedThreads, 1)
+weight_fused_kernel(const __grid_constant__ FusedBatch b) {
+  constexpr int L = (1 << BITS) - 1;
+  constexpr int WORDS = 4 * BITS;
+  extern __shared__ __align__(1024) uint8_t fused_smem[];
+  const uint32_t ring = ptx::smem_u32(fused_smem);
+  uint8_t* const staging = fused_smem + kRingBytes + (threadIdx.x >> 5) * 1024;  // consumer warps only
+  uint8_t* tail = fused_smem + kRingBytes + kStagingBytes;
+  const uint32_t bar0 = ring + kRingBytes + kStagingBytes;
+  auto full = [&](int s) { return bar0 + 8u * (uint32_t)s; };
+  auto empty = [&](int s) { return bar0 + 8u * (uint32_t)(kMaxRingSlots + s); };
+  uint32_t* s_hi = reinterpret_cast<uint32_t*>(tail + kTailScratch);  // [2][kFusedConsumerWarps]
+  uint32_t* s_lo = s_hi + 2 * kFusedConsumerWarps;
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + kTailFlags);
+  volatile int* issued = reinterpret_cast<volatile int*>(tail + kTailFlags + 8);  // [kMaxRingSlots] copies issued into each slot
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int W = b.team_warps;
+  const int chunk_units = b.chunk_units;
+  const int chunk_bytes = chunk_units * 512;
+  const int n_slots = b.n_slots;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < n_slots; ++s) {
+      ptx::mbar_init(full(s), 1);
+      ptx::mbar_init(empty(s), (uint32_t)W);
+    }
+    *abort_flag = 0;
+    for (int s = 0; s < kMaxRingSlots; ++s) issued[s] = 0;
+    ptx::fence_mbar_init();
+  }
+  __syncthreads();
+
+  if (warp >= kFusedConsumerWarps) {
+    // ---------------- producers ---------------------------------------------------------------------
+    // One lane issues a copy every few hundred cycles, too slow for small chunks: several producer
+    // warps share the CTA's chunk sequence, producer p taking the chunks whose index is p modulo the
+    // number of producers.
+    if (lane == 0) {
+      const int me = warp - kFusedConsumerWarps;
+      int slot = 0, it = 0, use = 0, turn = 0;  // use: how often `slot` has been filled so far
+      bool ok = true;
+      for (int g = blockIdx.x; ok && g < b.total_groups; g += gridDim.x) {
+        while (it + 1 < b.count && g >= b.item[it + 1].group_begin) ++it;
+        const WeightItem& m = b.item[it];
+        const int ug = m.rows_per_group * m.units_per_row;
+        const char* src = reinterpret_cast<const char*>(m.w) + (int64_t)(g - m.group_begin) * ug * 512;
+        for (int u0 = 0; u0 < ug; u0 += chunk_units) {
+          if (turn == me) {
+            // the slot's previous copy may be another producer's: it must have been issued before the
+            // parity of its release can be waited for
+            if (!((use == 0 || wait_issued(issued + slot, use - 1, abort_flag)) &&
+                  fused_wait(empty(slot), (uint32_t)(use & 1) ^ 1u, abort_flag))) {
+              ok = false;
+              break;
+            }
+            const uint32_t bytes = (uint32_t)min(chunk_units, ug - u0) * 512u;
+            ptx::mbar_arrive_expect_tx(full(slot), bytes);
+            ptx::bulk_load_1d(ring + (uint32_t)(slot * chunk_bytes), src + (int64_t)u0 * 512, bytes, full(slot));
+            __threadfence_block();
+            issued[slot] = use + 1;  // consumers wait on a slot's barrier only once its copy has been issued
+          }
+          if (++turn == kFusedProducers) turn = 0;
+          if (++slot == n_slots) {
+            slot = 0;
+            ++use;
+          }
+        }
+      }
+      if (!ok) {
+        *abort_flag = 1;
+        report_status(b.ws, QB_ERR_TIMEOUT, 0x40000);
+      }
+    }
+  } else {
+    // ---------------- consumer teams ----------------------------------------------------------------
+    const float kInf = __int_as_float(0x7f800000);
+    const int n_teams = kFusedConsumerWarps / W;
+    const int team = warp / W;
+    const int tw = warp - team * W;     // warp inside the team
+    const int tthread = tw * 32 + lane;  // thread inside the team
+    const int tthreads = 32 * W;
+    int slot = 0, it = 0, flip = 0, turn = 0;
+    int use = 0;  // how often `slot` has been filled before the current chunk
+    uint32_t phase = 0;
+    bool ok = true;
+    for (int g = blockIdx.x; g < b.total_groups; g += gridDim.x) {
+      while (it + 1 < b.count && g >= b.item[it + 1].group_begin) ++it;
+      const WeightItem& m = b.item[it];
+      const int gl = g - m.group_begin;
+      const int ug = m.rows_per_group * m.units_per_row;
+      const int n_chunks = (ug + chunk_units - 1) / chunk_units;
+      const bool mine = turn == team;
+      if (++turn == n_teams) turn = 0;
+      if (!mine) {  // another team's group: step over its slots
+        slot += n_chunks;
+        if (slot >= n_slots) {
+          slot -= n_slots;
+          phase ^= 1u;
+          ++use;
+        }
+        continue;
+      }
+      // pass 1: range of the group as the chunks arrive (NaN propagates; Inf shows in the range)
+      float lo = kInf, hi = -kInf;
+      {
+        int s = slot, us = use;
+        uint32_t ph = phase;
+        for (int c = 0; c < n_chunks; ++c) {
+          // A team does not see the phases of the slots it steps over, and a parity wait cannot tell
+          // phase n from phase n - 2: wait for the copy to have been issued (the slot's previous phase
+          // is then complete), and only then for its bytes.
+          bool got = true;
+          if (lane == 0) got = wait_issued(issued + s, us, abort_flag) && fused_wait(full(s), ph, abort_flag);
+          got = __shfl_sync(0xffffffffu, got, 0);
+          if (!got) {
+            ok = false;
+            break;
+          }
+          (void)ptx::mbar_try_wait(full(s), ph);  // every lane observes the completed phase itself
+          const int n4 = min(chunk_units, ug - c * chunk_units) * 32;
+          const float4* src = reinterpret_cast<const float4*>(fused_smem + s * chunk_bytes);
+#pragma unroll 4
+          for (int i = tthread; i < n4; i += tthreads) {
+            const float4 v = src[i];
+            lo = min_nan(min_nan(lo, v.x), min_nan(v.y, min_nan(v.z, v.w)));
+            hi = max_nan(max_nan(hi, v.x), max_nan(v.y, max_nan(v.z, v.w)));
+          }
+          if (++s == n_slots) {
+            s = 0;
+            ph ^= 1u;
+            ++us;
+          }
+        }
+      }
+      // NaN anywhere makes hi NaN (encoded above every number); Inf shows as hi = +Inf or lo = -Inf
+      uint32_t e_hi = __reduce_max_sync(0xffffffffu, float_to_ordered(hi));
+      uint32_t e_lo = __reduce_max_sync(0xffffffffu, ~float_to_ordered(lo));
+      if (W > 1) {
+        if (lane == 0) {
+          s_hi[flip * kFusedConsumerWarps + warp] = e_hi;
+          s_lo[flip * kFusedConsumerWarps + warp] = e_lo;
+        }
+      }
+      // every warp of the team reaches this barrier for every group of the team, whatever happened
+      if (team_sync_or(!ok || *abort_flag != 0, W, 1 + team)) {
+        ok = false;
+        break;
+      }
+      if (W > 1) {
+        const uint32_t vh = lane < W ? s_hi[flip * kFusedConsumerWarps + team * W + lane] : 0u;
+        const uint32_t vl = lane < W ? s_lo[flip * kFusedConsumerWarps + team * W + lane] : 0u;
+        e_hi = __reduce_max_sync(0xffffffffu, vh);
+        e_lo = __reduce_max_sync(0xffffffffu, vl);
+        flip ^= 1;
+      }
+      const float g_hi = ordered_to_float(e_hi);
+      const float g_lo = ordered_to_float(~e_lo);
+      const bool publish = tthread == 0;
+      if (publish && !(fabsf(g_hi) <= 3.402823466e38f && fabsf(g_lo) <= 3.402823466e38f))
+        report_status(b.ws, QB_ERR_NONFINITE);
+      const bool from_caller = m.range_lo != nullptr;
+      GroupParams gp;
+      if (from_caller)
+        gp = finish_group(__ldg(m.range_lo + gl), __ldg(m.range_hi + gl), true, L, gl, m.delta, m.q0, publish, b.ws);
+      else
+        gp = finish_group(g_lo, g_hi, false, L, gl, m.delta, m.q0, publish, b.ws);
+      // pass 2: codes and packed words from shared memory; each slot is released behind the warp
+      uint32_t* const out = m.packed + (int64_t)gl * ug * WORDS;
+      const int blocks_per_chunk = chunk_units >> 3;
+      for (int c = 0; c < n_chunks; ++c) {
+        const int units_here = min(chunk_units, ug - c * chunk_units);
+        const uint8_t* const base = fused_smem + slot * chunk_bytes;
+        // blocks of 8 units, numbered through the whole group, go to the team's warps in turn
+        for (int bb = 0; bb * 8 < units_here; ++bb) {
+          if (((c * blocks_per_chunk + bb) & (W - 1)) != tw) continue;
+          const int u0 = bb * 8;
+          const int nu = min(8, units_here - u0);
+          uint32_t* const o = out + (int64_t)(c * chunk_units + u0) * WORDS;
+          if (from_caller)
+            pack_block<BITS, true>(base + u0 * 512, staging, nu, gp, o, lane);
+          else
+            pack_block<BITS, false>(base + u0 * 512, staging, nu, gp, o, lane);
+        }
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(empty(slot));
+        if (++slot == n_slots) {
+          slot = 0;
+          phase ^= 1u;
+          ++use;
+        }
+      }
+    }
+    if (!ok && lane == 0) {
+      *abort_flag = 1;
+      report_status(b.ws, QB_ERR_TIMEOUT, 0x50000);
+    }
+  }
+
+  // ---------------- teardown: after a failed wait, let the copies already issued land ------------------
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) {
+    for (int s = 0; s < n_slots; ++s) {
+      const int n = issued[s];  // the last copy issued into slot s completes phase n - 1 of its barrier
+      if (n > 0) (void)fused_wait(full(s), (uint32_t)(n - 1) & 1u, nullptr);
+    }
   }
 }
 
@@ -302,10 +691,11 @@ struct HostWeight {
   float* q0;
 };
 
-// One pair of launches over `count` matrices (<= kMaxWeightBatch) of the same bit width.  Their range
-// tables sit back to back in the workspace: maxima at ws + kWsRangeOff, inverted minima after them.
-static qb_status launch_weight_batch(const HostWeight* m, int count, int bits, void* ws, int sm_count,
-                                     cudaStream_t stream) {
+// Two-pass path: one pair of launches over `count` matrices (<= kMaxWeightBatch) of the same bit width.
+// Their range tables sit back to back in the workspace: maxima at ws + kWsRangeOff, inverted minima
+// after them.
+static qb_status launch_two_pass(const HostWeight* m, int count, int bits, void* ws, int sm_count,
+                                 cudaStream_t stream) {
   WeightBatch b;
   memset(&b, 0, sizeof(b));
   int total_groups = 0;
@@ -350,6 +740,107 @@ static qb_status launch_weight_batch(const HostWeight* m, int count, int bits, v
     default: return QB_ERR_INVALID;
   }
   QB_CUDA_TRY(cudaGetLastError());
+  return QB_OK;
+}
+
+static inline int64_t group_units(const HostWeight& h) { return (h.N / h.groups) * (h.K / 128); }
+
+// Single-read path over `count` matrices (<= kMaxWeightBatch) whose groups all fit the ring.
+static qb_status launch_fused(const HostWeight* m, int count, int bits, void* ws, int sm_count,
+                              cudaStream_t stream) {
+  FusedBatch b;
+  memset(&b, 0, sizeof(b));
+  int total_groups = 0;
+  for (int i = 0; i < count; ++i) {
+    WeightItem& it = b.item[i];
+    it.w = reinterpret_cast<const float4*>(m[i].w);
+    it.packed = m[i].packed;
+    it.delta = m[i].delta;
+    it.q0 = m[i].q0;
+    it.range_lo = m[i].range_lo;
+    it.range_hi = m[i].range_hi;
+    it.units = m[i].N * m[i].K / 128;
+    it.units_per_row = (int32_t)(m[i].K / 128);
+    it.rows_per_group = (int32_t)(m[i].N / m[i].groups);
+    it.group_begin = total_groups;
+    total_groups += m[i].groups;
+  }
+  b.count = count;
+  b.ws = ws;
+  b.total_groups = total_groups;
+  // small groups: 4 KB slots and small teams (many groups in flight); large groups: 16 KB slots
+  int64_t ug_max = 1;
+  for (int i = 0; i < count; ++i) ug_max = std::max(ug_max, group_units(m[i]));
+  b.chunk_units = ug_max <= 64 ? 8 : 32;
+  b.n_slots = kRingBytes / (b.chunk_units * 512);
+  b.team_warps = ug_max <= 16 ? 1 : (ug_max <= 64 ? 2 : (ug_max <= 160 ? 4 : 8));
+  const unsigned grid = (unsigned)(total_groups < sm_count ? total_groups : sm_count);
+#define QB_LAUNCH_FUSED(B)                                                                                  \
+  do {                                                                                                      \
+    QB_CUDA_TRY(cudaFuncSetAttribute(weight_fused_kernel<B>, cudaFuncAttributeMaxDynamicSharedMemorySize,  \
+                                     kFusedSmemBytes));                                                     \
+    weight_fused_kernel<B><<<grid, kFusedThreads, kFusedSmemBytes, stream>>>(b);                           \
+  } while (0)
+  switch (bits) {
+    case 2: QB_LAUNCH_FUSED(2); break;
+    case 3: QB_LAUNCH_FUSED(3); break;
+    case 4: QB_LAUNCH_FUSED(4); break;
+    case 8: QB_LAUNCH_FUSED(8); break;
+    default: return QB_ERR_INVALID;
+  }
+#undef QB_LAUNCH_FUSED
+  QB_CUDA_TRY(cudaGetLastError());
+  return QB_OK;
+}
+
+// Size class of a matrix for the single-read path (team size and slot size are per launch).
+static inline int fused_class(int64_t ug) { return ug <= 16 ? 0 : (ug <= 64 ? 1 : (ug <= 160 ? 2 : 3)); }
+
+// Matrices of one bit width (<= kMaxWeightBatch).  Those whose groups fit in shared memory take the
+// single-read path when together they have enough groups to occupy the GPU, one launch per size class
+// of groups (a class too small to be worth a launch joins the next larger one); the others take the
+// two-pass path.
+static qb_status launch_weight_batch(const HostWeight* m, int count, int bits, void* ws, int sm_count,
+                                     cudaStream_t stream) {
+  constexpr int64_t kClassWorthALaunch = 32ll << 20;  // bytes of fp32 weights
+  HostWeight fused[kMaxWeightBatch], rest[kMaxWeightBatch];
+  int cls[kMaxWeightBatch];
+  int nf = 0, nr = 0;
+  int64_t fused_groups = 0;
+  for (int i = 0; i < count; ++i) {
+    if (group_units(m[i]) <= kFusedMaxGroupUnits) {
+      cls[nf] = fused_class(group_units(m[i]));
+      fused[nf++] = m[i];
+      fused_groups += m[i].groups;
+    } else {
+      rest[nr++] = m[i];
+    }
+  }
+  if (fused_groups * 2 < sm_count) {  // too few groups to spread over the SMs
+    for (int i = 0; i < nf; ++i) rest[nr++] = fused[i];
+    nf = 0;
+  }
+  if (nf > 0) {
+    HostWeight batch[kMaxWeightBatch];
+    int nb = 0;
+    int64_t bytes = 0;
+    for (int c = 0; c < 4; ++c) {
+      for (int i = 0; i < nf; ++i)
+        if (cls[i] == c) {
+          batch[nb++] = fused[i];
+          bytes += fused[i].N * fused[i].K * 4;
+        }
+      bool later = false;  // does a larger class still have matrices?
+      for (int i = 0; i < nf; ++i) later = later || cls[i] > c;
+      if (nb > 0 && (bytes >= kClassWorthALaunch || !later)) {
+        qb_status st = launch_fused(batch, nb, bits, ws, sm_count, stream);
+        if (st != QB_OK) return st;
+        nb = 0;
+        bytes = 0;
+      }
+    }
+  }
+  if (nr > 0) return launch_two_pass(rest, nr, bits, ws, sm_count, stream);
   return QB_OK;
 }
 

@@ -74,6 +74,82 @@ def test_quantize_pack_weights_matches_oracle(ws, bits, N, K, groups):
     assert torch.equal(packed, packed2) and torch.equal(delta, delta2) and torch.equal(q0, q02)
 
 
+@pytest.mark.parametrize("bits", BITS)
+@pytest.mark.parametrize("N,K,groups", [
+    (2304, 768, 384),    # more groups than SMs, 36 units per group: one full chunk + a ragged one
+    (2560, 1536, 80),    # 384 units per group: the largest group the shared-memory ring holds
+    (2640, 1536, 80),    # 396 units per group: too large, two-pass path
+    (2048, 9600, 512),   # 300 units per group, several groups per CTA: the ring wraps
+    (296, 128, 148),     # two units per group
+])
+def test_quantize_weights_single_read_path(bits, N, K, groups):
+    ws_big = qb.workspace(groups=1024)
+    w = synth.weights(N, K, seed=7 * N + K + groups + bits)
+    packed, delta, q0 = gu.gpu_quantize_weights(w, bits, groups, ws_big)
+    assert qb.read_status(ws_big) == qb.QB_OK
+    st, codes, o_delta, o_q0 = oracle.quantize_weights(w, bits, groups)
+    assert np.array_equal(gu.words_np(packed), oracle.pack(codes, bits))
+    assert np.array_equal(delta.cpu().numpy(), o_delta)
+    assert np.array_equal(q0.cpu().numpy(), o_q0)
+
+
+@pytest.mark.parametrize("bits,shapes", [
+    # thirteen matrices whose groups each fill the whole ring; some CTAs take two groups
+    (4, [(768, 768, 12)] * 13),
+    # group sizes from 6 to 240 units in one launch, hundreds of groups per CTA
+    (3, [(768, 768, 768), (768, 7680, 768), (3072, 768, 768), (768, 768, 128), (768, 3072, 768)]),
+    (2, [(768, 768, 128), (3072, 768, 128), (768, 3072, 128), (2304, 768, 384)] * 3),
+])
+def test_quantize_weights_single_read_path_batches(bits, shapes):
+    ws_big = qb.workspace(groups=8192)
+    items, host = [], []
+    for i, (N, K, G) in enumerate(shapes):
+        w = synth.weights(N, K, seed=31 * i + N + K + G)
+        packed = gu.poison(torch.empty((N, K * bits // 32), dtype=torch.int32, device="cuda"))
+        delta = gu.poison(torch.empty(G, dtype=torch.float32, device="cuda"))
+        q0 = gu.poison(torch.empty(G, dtype=torch.float32, device="cuda"))
+        items.append((gu.dev(w), bits, G, packed, delta, q0))
+        host.append(w)
+    for _ in range(3):  # repeated: a race between teams would not show every time
+        qb.quantize_pack_weights_batch(items, ws_big)
+    assert qb.read_status(ws_big) == qb.QB_OK
+    for (wd, _, G, packed, delta, q0), w in zip(items, host):
+        st, codes, o_delta, o_q0 = oracle.quantize_weights(w, bits, G)
+        assert np.array_equal(gu.words_np(packed), oracle.pack(codes, bits))
+        assert np.array_equal(delta.cpu().numpy(), o_delta)
+        assert np.array_equal(q0.cpu().numpy(), o_q0)
+
+
+def test_quantize_weights_single_read_path_edge_cases():
+    # enough small groups for the single-read path: constant groups, caller ranges, non-finite input
+    N, K, G = 256, 128, 128
+    w = synth.weights(N, K, seed=11)
+    w[:2] = -0.25
+    w[4, :8] = [0.0, 0.5, 1.5, 2.5, 3.0, 1.0, 2.0, 0.25]
+    w[4, 8:] = 1.0
+    w[5] = w[4]
+    ws1 = qb.workspace(groups=G)
+    for bits in BITS:
+        packed, delta, q0 = gu.gpu_quantize_weights(w, bits, G, ws1)
+        st, codes, o_delta, o_q0 = oracle.quantize_weights(w, bits, G)
+        assert np.array_equal(gu.words_np(packed), oracle.pack(codes, bits))
+        assert np.array_equal(delta.cpu().numpy(), o_delta) and np.array_equal(q0.cpu().numpy(), o_q0)
+        assert delta.cpu().numpy()[0] == 1.0
+        lo = np.linspace(-0.05, -0.01, G).astype(np.float32)
+        hi = np.linspace(0.02, 0.06, G).astype(np.float32)
+        packed, delta, q0 = gu.gpu_quantize_weights(w, bits, G, ws1, lo, hi)
+        st, codes, o_delta, o_q0 = oracle.quantize_weights(w, bits, G, lo, hi)
+        assert st == oracle.OK
+        assert np.array_equal(gu.words_np(packed), oracle.pack(codes, bits))
+        assert np.array_equal(delta.cpu().numpy(), o_delta) and np.array_equal(q0.cpu().numpy(), o_q0)
+    assert qb.read_status(ws1) == qb.QB_OK
+    ws2 = qb.workspace(groups=G)
+    w[200, 77] = np.inf
+    gu.gpu_quantize_weights(w, 3, G, ws2)
+    assert qb.read_status(ws2) == qb.QB_ERR_NONFINITE
+    assert oracle.quantize_weights(w, 3, G)[0] == oracle.ERR_NONFINITE
+
+
 def test_quantize_weights_edge_cases(ws):
     # constant group, exact ties, caller-supplied (clipping) ranges, non-finite input
     w = synth.weights(8, 128, seed=1)
