@@ -101,19 +101,21 @@ struct GemmCfg {
 // The bound is counted in SM clock cycles (clock64 is a cheap register read; the global nanosecond
 // timer costs about a microsecond per read and would dominate short waits).
 // kSleep: the waiter is not on the critical path (it runs several stages ahead) and must not compete
-// for issue slots with the MMA issuer that shares its scheduler: it sleeps between polls.  A polling
-// warp is always "ready", so a handful of them starve the one thread that feeds the tensor cores.
+// for issue slots with the MMA issuer that shares its scheduler: it uses the form of try_wait that
+// takes a suspend-time hint.  A warp that polls in a tight loop is always "ready", and a handful of
+// them starve the one thread that feeds the tensor cores.
 template <bool kSleep>
 __device__ __forceinline__ bool wait_barrier_t(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   if (ptx::mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
-  uint32_t ns = 32;
   for (uint32_t spin = 1;; ++spin) {
     if (kSleep) {
-      __nanosleep(ns);
-      if (ns < 256) ns += ns;
+      // suspended by the hardware until the phase completes or about a microsecond has passed: no issue
+      // slots are spent while waiting and the wake-up does not wait for a sleep interval to end
+      if (ptx::mbar_try_wait_suspend(bar, parity, 1000u)) return true;
+    } else {
+      if (ptx::mbar_try_wait(bar, parity)) return true;
     }
-    if (ptx::mbar_try_wait(bar, parity)) return true;
     if ((spin & 63u) == 0u) {
       if (*abort_flag) return false;
       if (clock64() - t0 > kWaitLimitCycles) return false;
@@ -794,9 +796,11 @@ static qb_status validate_gemm(const int8_t* xq, const float* act_scale, const i
   return QB_OK;
 }
 
-// One launch over descriptors d[idx[0..count)] (count <= kMaxProblems), all with the same bit width.
+// One launch over descriptors d[idx[0..count)] (count <= kMaxProblems), all with the same bit width, on at
+// most `max_ctas` CTAs.
 static qb_status launch_group(const qb_linear_desc* d, const int* idx, int count, int32_t* acc_out, void* ws,
-                              int sm_count, cudaStream_t stream) {
+                              int max_ctas, cudaStream_t stream) {
+  const int sm_count = max_ctas;
   const int bits = d[idx[0]].bits;
   const int bt = choose_token_tile(d, idx, count, sm_count);
   GroupedParams gp;
@@ -876,8 +880,42 @@ static qb_status launch_group(const qb_linear_desc* d, const int* idx, int count
   return bt == 256 ? launch_group_bits<256>(bits, gp, grid, stream) : launch_group_bits<128>(bits, gp, grid, stream);
 }
 
+// Side streams and events for launches of one stack that run side by side (host objects, created once per
+// device on first use; no device memory).
+constexpr int kMaxSide = 7;
+struct SideStreams {
+  cudaStream_t stream[kMaxSide];
+  cudaEvent_t done[kMaxSide];
+  cudaEvent_t fork;
+  bool ready;
+};
+static qb_status side_streams(SideStreams** out) {
+  static SideStreams per_dev[64];
+  int dev = 0;
+  QB_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) {
+    set_last_error("device ordinal %d out of range", dev);
+    return QB_ERR_CUDA;
+  }
+  SideStreams& s = per_dev[dev];
+  if (!s.ready) {
+    for (int i = 0; i < kMaxSide; ++i) {
+      QB_CUDA_TRY(cudaStreamCreateWithFlags(&s.stream[i], cudaStreamNonBlocking));
+      QB_CUDA_TRY(cudaEventCreateWithFlags(&s.done[i], cudaEventDisableTiming));
+    }
+    QB_CUDA_TRY(cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming));
+    s.ready = true;
+  }
+  *out = &s;
+  return QB_OK;
+}
+
 // Split a stack into launches: same bit width per launch, longest K first (its tiles are the longest,
 // so they go out first in the round-robin), at most kMaxProblems problems and 2^30 tiles per launch.
+// A stack whose launches are all short (a mixed-precision stack at small M: a few tiles per SM in
+// total) runs its launches side by side, each on a share of the SMs in proportion to its work, so that
+// the start-up and the drain of the pipelines overlap instead of adding up; the launches join the
+// caller's stream before the call returns.  Large stacks keep one launch after the other on all SMs.
 static qb_status launch_stack(const qb_linear_desc* d, int count, void* ws, int sm_count, cudaStream_t stream) {
   std::vector<int> order(count);
   for (int i = 0; i < count; ++i) order[i] = i;
@@ -885,21 +923,83 @@ static qb_status launch_stack(const qb_linear_desc* d, int count, void* ws, int 
     if (d[a].bits != d[b].bits) return d[a].bits < d[b].bits;
     return d[a].K > d[b].K;
   });
+  struct Group {
+    int begin, count;
+    int64_t tiles, cost;
+  };
+  std::vector<Group> groups;
+  int64_t all_tiles = 0, all_cost = 0;
   int i = 0;
   while (i < count) {
     int j = i;
-    int64_t tiles = 0;
+    int64_t tiles = 0, cost = 0;
     while (j < count && j - i < kMaxProblems && d[order[j]].bits == d[order[i]].bits) {
       const int64_t t = ((d[order[j]].N + kTileN - 1) / kTileN) * ((d[order[j]].M + 127) / 128);
       if (j > i && tiles + t > (1 << 30)) break;
       tiles += t;
+      cost += t * (d[order[j]].K / kBlockK + 5);  // K blocks plus a tile's fixed cost, as in the tile order
       ++j;
     }
-    qb_status st = launch_group(d, order.data() + i, j - i, nullptr, ws, sm_count, stream);
-    if (st != QB_OK) return st;
+    groups.push_back({i, j - i, tiles, cost});
+    all_tiles += tiles;
+    all_cost += cost;
     i = j;
   }
-  return QB_OK;
+  const int n_groups = (int)groups.size();
+  const bool side_by_side = n_groups > 1 && n_groups <= kMaxSide + 1 && n_groups <= sm_count &&
+                            all_tiles < (int64_t)16 * sm_count;
+  if (!side_by_side) {
+    for (const Group& g : groups) {
+      qb_status st = launch_group(d, order.data() + g.begin, g.count, nullptr, ws, sm_count, stream);
+      if (st != QB_OK) return st;
+    }
+    return QB_OK;
+  }
+  // SM shares in proportion to cost (at least one CTA each, no more than the launch has tiles); what
+  // rounding leaves over goes to the launches with the most work per CTA.
+  std::vector<int> share(n_groups);
+  int used = 0;
+  for (int g = 0; g < n_groups; ++g) {
+    int64_t sh = (int64_t)sm_count * groups[g].cost / all_cost;
+    if (sh < 1) sh = 1;
+    if (sh > groups[g].tiles) sh = groups[g].tiles;
+    share[g] = (int)sh;
+    used += share[g];
+  }
+  while (used > sm_count) {  // the minimum of one CTA per launch can overshoot: take from the largest share
+    int big = 0;
+    for (int g = 1; g < n_groups; ++g)
+      if (share[g] > share[big]) big = g;
+    --share[big];
+    --used;
+  }
+  while (used < sm_count) {
+    int best = -1;
+    for (int g = 0; g < n_groups; ++g)
+      if (share[g] < groups[g].tiles &&
+          (best < 0 || groups[g].cost * share[best] > groups[best].cost * share[g]))
+        best = g;
+    if (best < 0) break;
+    ++share[best];
+    ++used;
+  }
+  SideStreams* side = nullptr;
+  qb_status st = side_streams(&side);
+  if (st != QB_OK) return st;
+  QB_CUDA_TRY(cudaEventRecord(side->fork, stream));
+  for (int g = 1; g < n_groups; ++g) QB_CUDA_TRY(cudaStreamWaitEvent(side->stream[g - 1], side->fork, 0));
+  qb_status first_error = QB_OK;
+  for (int g = 0; g < n_groups; ++g) {
+    cudaStream_t sg = g == 0 ? stream : side->stream[g - 1];
+    st = launch_group(d, order.data() + groups[g].begin, groups[g].count, nullptr, ws, share[g], sg);
+    if (st != QB_OK && first_error == QB_OK) first_error = st;
+  }
+  // always join, also after an error: the caller's stream must not run ahead of the side streams
+  for (int g = 1; g < n_groups; ++g) {
+    QB_CUDA_TRY(cudaEventRecord(side->done[g - 1], side->stream[g - 1]));
+    QB_CUDA_TRY(cudaStreamWaitEvent(stream, side->done[g - 1], 0));
+  }
+  return first_error;
 }
 
 }  // namespace qb
