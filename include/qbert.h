@@ -214,6 +214,12 @@ typedef struct {
  * descriptors, e.g. four per encoder layer in the order QKV, attention output, FFN1, FFN2; each is
  * an independent problem with its own input, and the result of each equals qb_gemm on the same
  * arguments bit for bit.  All descriptors are validated before anything is launched.
+ * Descriptors of equal bit width share a launch; a stack that mixes bit widths and is small (a few
+ * tiles per SM in total) runs its launches side by side on streams the library creates once per
+ * device (host objects only, no device memory).  They fork from and join `cuda_stream` inside the
+ * call, so to the caller the work is ordered on `cuda_stream` as for every other call, and the call may
+ * be captured into a CUDA graph.  The first such call on a device creates the streams and is not
+ * safe to issue from two host threads at once.
  */
 qb_status qb_layer_linears(const qb_linear_desc* descs /*host*/, int32_t count, void* ws,
                            size_t ws_bytes, void* cuda_stream);
