@@ -10,6 +10,7 @@
 //                                x * (127/a), round half to even, clamp, four codes packed per 32-bit
 //                                store, int32 row sum by warp reduction.
 // Both kernels are HBM-bound: 4 B read per element in each, 1 B written in the second.
+#include <algorithm>
 #include <cstring>
 
 #include "common.cuh"
@@ -95,7 +96,7 @@ __device__ __forceinline__ bool act_scales(uint32_t mb, float* s, float* inv) {
   return true;
 }
 
-__global__ void __launch_bounds__(kActThreads)
+__global__ void __launch_bounds__(kActThreads, 8)  // eight blocks per SM resident: the grid is one full wave
 act_quantize_kernel(const __grid_constant__ ActBatch b) {
   const int lane = threadIdx.x & 31;
   const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
@@ -141,25 +142,35 @@ static qb_status launch_act_batch(const qb_act_desc* d, int count, void* ws, uin
   b.count = count;
   b.ws = ws;
   b.absmax_bits = absmax_slots;
-  const int64_t cap = (int64_t)sm_count * 8;
+  const int64_t cap = (int64_t)sm_count * 8;  // one full wave of either kernel (eight blocks per SM)
   int64_t total4 = 0;
   for (int i = 0; i < count; ++i) total4 += d[i].M * d[i].K / 4;
+  // Tensors with the longest rows first: kernel 2 hands rows to warps round-robin, and a long row met
+  // at the end of a warp's list would be the launch's tail.  Slot i of `absmax_slots` stays with the
+  // i-th tensor of this order; nothing outside the two kernels reads the slots.
+  int ord[kMaxActBatch];
+  for (int i = 0; i < count; ++i) ord[i] = i;
+  std::stable_sort(ord, ord + count, [&](int a, int c) { return d[a].K > d[c].K; });
   int64_t rows = 0;
   int blocks1 = 0;
   for (int i = 0; i < count; ++i) {
+    const qb_act_desc& q = d[ord[i]];
     ActItem& t = b.item[i];
-    t.x = d[i].x;
-    t.xq = d[i].xq;
-    t.act_scale = d[i].act_scale;
-    t.rowsum = d[i].rowsum;
-    t.M = d[i].M;
-    t.K = d[i].K;
+    t.x = q.x;
+    t.xq = q.xq;
+    t.act_scale = q.act_scale;
+    t.rowsum = q.rowsum;
+    t.M = q.M;
+    t.K = q.K;
     t.row_begin = rows;
-    rows += d[i].M;
-    // blocks of kernel 1 in proportion to the tensor's size, each thread >= 4 loads when possible
-    const int64_t n4 = d[i].M * d[i].K / 4;
+    rows += q.M;
+    // blocks of kernel 1 in proportion to the tensor's size (rounded down, so that the launch never
+    // exceeds one wave: a block of a second wave would run alone for as long as the whole first wave),
+    // each thread >= 4 loads when possible
+    const int64_t n4 = q.M * q.K / 4;
     int64_t want = (n4 + (int64_t)kActThreads * 4 - 1) / ((int64_t)kActThreads * 4);
-    const int64_t share = (cap * n4 + total4 - 1) / total4;
+    const int64_t avail = cap - count > 0 ? cap - count : 0;  // one block per tensor is set aside
+    const int64_t share = 1 + avail * n4 / total4;
     if (want > share) want = share;
     if (want < 1) want = 1;
     t.block_begin = blocks1;
