@@ -940,6 +940,10 @@ static qb_status launch_stack(const qb_linear_desc* d, int count, void* ws, int 
       cost += t * (d[order[j]].K / kBlockK + 5);  // K blocks plus a tile's fixed cost, as in the tile order
       ++j;
     }
+    // measured at M = 128: a K block of 3-bit weights takes about 1.2 times, of 8-bit weights about 1.4 times
+    // as long as one of 2- or 4-bit weights (expansion work; bytes fetched per block with few CTAs pulling)
+    const int b = d[order[i]].bits;
+    cost *= b == 3 ? 12 : (b == 8 ? 14 : 10);
     groups.push_back({i, j - i, tiles, cost});
     all_tiles += tiles;
     all_cost += cost;
