@@ -342,6 +342,43 @@ def test_config2_mixed_precision_stack(ws):
     _check_stack(ws, wl, layers=range(wl.layers), rows_per_tile=8)
 
 
+def test_mixed_stack_side_by_side_in_a_graph(ws):
+    # A small stack that mixes bit widths runs its launches side by side on the library's own streams.
+    # Captured into a CUDA graph on a non-default stream and replayed, it must still equal the single
+    # calls bit for bit (the side streams fork from and join the capturing stream inside the call).
+    M = 128
+    shapes = [(256, 256, 2, 4), (384, 512, 4, 6), (128, 1024, 8, 2), (256, 256, 3, 1), (256, 768, 2, 8)]
+    descs, singles = [], []
+    for i, (N, K, bits, G) in enumerate(shapes):
+        x = synth.activations(M, K, seed=900 + i)
+        w = synth.weights(N, K, seed=950 + i)
+        b = synth.bias(N, seed=990 + i)
+        xq, sc, rs = qb.quantize_act(gu.dev(x), ws)
+        packed, delta, q0 = qb.quantize_pack_weights(gu.dev(w), bits, G, ws)
+        y = gu.poison(torch.empty((M, N), dtype=torch.float32, device="cuda"))
+        descs.append(qb.LinearDesc(xq, sc, rs, packed, delta, q0, gu.dev(b), N, bits, G, y))
+        singles.append(qb.gemm(xq, sc, rs, packed, delta, q0, gu.dev(b), N, bits, G, ws).clone())
+    arr = qb.make_desc_array(descs)
+    qb.layer_linears(arr, ws)  # first call on the device creates the side streams: before any capture
+    torch.cuda.synchronize()
+    for d, y1 in zip(descs, singles):
+        assert torch.equal(d.y, y1)
+        gu.poison(d.y)
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            qb.layer_linears(arr, ws)
+        for _ in range(2):
+            graph.replay()
+    stream.synchronize()
+    torch.cuda.synchronize()
+    assert qb.read_status(ws) == qb.QB_OK
+    for d, y1 in zip(descs, singles):
+        assert torch.equal(d.y, y1)
+
+
 @pytest.mark.parametrize("preset", ["2/3-MP SST-2", "2/4-MP SST-2"])
 def test_paper_bit_presets_stack(ws, preset):
     # the per-layer bit widths printed in the paper's appendix tables, first four layers' worth of bits
