@@ -57,6 +57,8 @@ def _lib(omp: bool = False) -> ctypes.CDLL:
         lib.qo_pack.restype = i32
         lib.qo_unpack.argtypes = [vp, i64, i64, i32, vp]
         lib.qo_unpack.restype = i32
+        lib.qo_round_bf16.argtypes = [vp, i64, vp]
+        lib.qo_round_bf16.restype = None
         lib.qo_quantize_act.argtypes = [vp, i64, i64, vp, vp, vp]
         lib.qo_quantize_act.restype = i32
         lib.qo_int_gemm.argtypes = [vp, vp, i64, i64, i64, vp, vp]
@@ -198,3 +200,11 @@ def linear(x, w, bias, bits: int, groups: int, omp: bool = False):
     y = dequant_epilogue(acc, rowsum, s_a, delta, q0, bias, bits, groups, omp=omp)
     return dict(status_act=st_a, status_w=st_w, xq=xq, act_scale=s_a, rowsum=rowsum, codes=codes,
                 delta=delta, q0=q0, words=words, acc=acc, y=y)
+
+
+def round_bf16(y) -> np.ndarray:
+    """fp32 -> bfloat16 bit patterns (uint16), round to nearest, ties to even; same shape as ``y``."""
+    y = _c(np.asarray(y), np.float32)
+    out = np.empty(y.shape, dtype=np.uint16)
+    _lib().qo_round_bf16(_p(y), y.size, _p(out))
+    return out

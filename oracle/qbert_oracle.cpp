@@ -279,4 +279,35 @@ void qo_linear_fp64(const int8_t* xq, float act_scale, const uint8_t* codes, con
     }
 }
 
+// Narrow output (the paper keeps the activations between layers at 8 bits, Table 1 caption, so a
+// linear's fp32 result is an intermediate that the next operation narrows): the fp32 result of the
+// dequantizing epilogue rounded to bfloat16 (8 significant bits, the exponent range of fp32), round to
+// nearest, ties to the value whose last kept bit is 0.  Written as the definition: the two neighbours
+// of y that bfloat16 can represent are found by dropping the 16 low bits (towards zero) and by one
+// step of the kept field away from zero; the nearer one in exact arithmetic (double holds both
+// differences exactly) is taken.  Inputs must be finite; a result that would overflow becomes
+// infinity, as the step away from zero yields that bit pattern.
+void qo_round_bf16(const float* y, int64_t n, uint16_t* out) {
+  for (int64_t i = 0; i < n; ++i) {
+    uint32_t u;
+    std::memcpy(&u, &y[i], 4);
+    const uint32_t lo_bits = u & 0xFFFF0000u;    // towards zero
+    const uint32_t hi_bits = lo_bits + 0x10000u;  // one step away from zero (same sign bit)
+    float lo, hi;
+    std::memcpy(&lo, &lo_bits, 4);
+    std::memcpy(&hi, &hi_bits, 4);
+    const double d_lo = std::fabs((double)y[i] - (double)lo);
+    const bool hi_finite = ((hi_bits >> 23) & 0xFFu) != 0xFFu;
+    // distance to the upper neighbour; when that neighbour is infinity the value it stands for is
+    // 2^128 (the next step of the same grid)
+    const double hi_val = hi_finite ? (double)hi : std::ldexp((u >> 31) ? -1.0 : 1.0, 128);
+    const double d_hi = std::fabs(hi_val - (double)y[i]);
+    uint32_t r;
+    if (d_lo < d_hi) r = lo_bits;
+    else if (d_hi < d_lo) r = hi_bits;
+    else r = ((lo_bits >> 16) & 1u) == 0u ? lo_bits : hi_bits;  // tie: last kept bit 0
+    out[i] = (uint16_t)(r >> 16);
+  }
+}
+
 }  // extern "C"
