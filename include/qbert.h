@@ -225,6 +225,26 @@ qb_status qb_layer_linears(const qb_linear_desc* descs /*host*/, int32_t count, 
                            size_t ws_bytes, void* cuda_stream);
 
 /*
+ * Narrow-output forms of qb_gemm and qb_layer_linears.  The paper keeps the activations between
+ * layers at 8 bits (Table 1 caption: every quantized model uses 8-bit activations), so the fp32
+ * result of a linear is an intermediate that the next operation narrows again; writing it as
+ * bfloat16 halves the bytes of the write that bounds the K <= 1024 linears.
+ *     y[m][n] = bf16( the fp32 value qb_gemm writes for the same arguments )
+ * with round to nearest, ties to even, on the finished fp32 value (one extra rounding, after the
+ * epilogue of Appendix A has been evaluated exactly as in qb_gemm).
+ *   y   dev bfloat16 [M][N], as 16-bit patterns                     (written)
+ * Everything else as for qb_gemm; there is no accumulator export.  In qb_layer_linears_bf16 the
+ * `y` field of every descriptor points to such a bfloat16 array (cast to float*); each result equals
+ * qb_gemm_bf16 on the same arguments bit for bit.
+ */
+qb_status qb_gemm_bf16(const int8_t* xq, const float* act_scale, const int32_t* rowsum,
+                       const uint32_t* packed, const float* delta, const float* q0, const float* bias,
+                       int64_t M, int64_t N, int64_t K, int bits, int groups, uint16_t* y, void* ws,
+                       size_t ws_bytes, void* cuda_stream);
+qb_status qb_layer_linears_bf16(const qb_linear_desc* descs /*host*/, int32_t count, void* ws,
+                                size_t ws_bytes, void* cuda_stream);
+
+/*
  * Diagnostic: the rate the tensor cores sustain for the GEMM's own instruction (tcgen05.mma kind::i8,
  * s8 x s8 -> s32, 128 x `tokens` x 32) with both operands resident in shared memory, no global
  * traffic, four K blocks in flight, one CTA per SM on the default stream.  (No counterpart in the

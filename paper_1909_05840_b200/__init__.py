@@ -30,7 +30,7 @@ EXPORTS = (
     "qb_version", "qb_status_string", "qb_last_error", "qb_packed_words", "qb_workspace_bytes",
     "qb_workspace_init", "qb_read_status", "qb_quantize_act", "qb_quantize_pack_weights", "qb_gemm",
     "qb_layer_linears", "qb_quantize_pack_weights_noalloc", "qb_probe_i8_mma", "qb_quantize_act_batch",
-    "qb_quantize_pack_weights_batch",
+    "qb_quantize_pack_weights_batch", "qb_gemm_bf16", "qb_layer_linears_bf16",
 )
 NOALLOC_MAX_GROUPS = 4096
 
@@ -107,6 +107,10 @@ def lib() -> ctypes.CDLL:
     L.qb_gemm.restype = i32
     L.qb_layer_linears.argtypes = [ctypes.POINTER(LinearDescC), i32, vp, sz, vp]
     L.qb_layer_linears.restype = i32
+    L.qb_gemm_bf16.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, ctypes.c_int, ctypes.c_int, vp, vp, sz, vp]
+    L.qb_gemm_bf16.restype = i32
+    L.qb_layer_linears_bf16.argtypes = [ctypes.POINTER(LinearDescC), i32, vp, sz, vp]
+    L.qb_layer_linears_bf16.restype = i32
     _lib = L
     return L
 
@@ -251,6 +255,20 @@ def gemm(xq: torch.Tensor, act_scale: torch.Tensor, rowsum: torch.Tensor, packed
     return (y, acc_out) if (want_acc or acc_out is not None) else y
 
 
+def gemm_bf16(xq: torch.Tensor, act_scale: torch.Tensor, rowsum: torch.Tensor, packed: torch.Tensor,
+              delta: torch.Tensor, q0: torch.Tensor, bias: Optional[torch.Tensor], N: int, bits: int, groups: int,
+              ws: torch.Tensor, y: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """``qb_gemm_bf16``: returns ``y`` bfloat16 [M,N]."""
+    assert xq.is_cuda and xq.dtype == torch.int8 and xq.is_contiguous()
+    M, K = xq.shape
+    y = torch.empty((M, N), dtype=torch.bfloat16, device=xq.device) if y is None else y
+    assert y.dtype == torch.bfloat16 and y.is_contiguous()
+    _check(lib().qb_gemm_bf16(xq.data_ptr(), act_scale.data_ptr(), rowsum.data_ptr(), packed.data_ptr(),
+                              delta.data_ptr(), q0.data_ptr(), _ptr(bias), M, N, K, bits, groups, y.data_ptr(),
+                              ws.data_ptr(), ws.numel(), _stream()), "qb_gemm_bf16")
+    return y
+
+
 @dataclass
 class LinearDesc:
     """One linear of a stack: tensors as produced by ``quantize_act`` / ``quantize_pack_weights``."""
@@ -282,3 +300,11 @@ def layer_linears(descs, ws: torch.Tensor) -> None:
     """``qb_layer_linears`` over a list of ``LinearDesc`` (or an array from ``make_desc_array``)."""
     arr = descs if isinstance(descs, ctypes.Array) else make_desc_array(descs)
     _check(lib().qb_layer_linears(arr, len(arr), ws.data_ptr(), ws.numel(), _stream()), "qb_layer_linears")
+
+
+def layer_linears_bf16(descs, ws: torch.Tensor) -> None:
+    """``qb_layer_linears_bf16``: as ``layer_linears``, every ``y`` a bfloat16 [M,N] tensor."""
+    if not isinstance(descs, ctypes.Array):
+        assert all(d.y.dtype == torch.bfloat16 for d in descs)
+    arr = descs if isinstance(descs, ctypes.Array) else make_desc_array(descs)
+    _check(lib().qb_layer_linears_bf16(arr, len(arr), ws.data_ptr(), ws.numel(), _stream()), "qb_layer_linears_bf16")

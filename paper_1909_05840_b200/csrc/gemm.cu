@@ -30,6 +30,7 @@
 // i+1.  Every wait is bounded: on expiry the CTA records QB_ERR_TIMEOUT and leaves through the
 // normal exit path (TMEM freed).
 #include <cuda.h>
+#include <cuda_bf16.h>
 
 #include <algorithm>
 #include <cstring>
@@ -62,7 +63,7 @@ struct Problem {
   const float* delta;
   const float* q0;
   const float* bias;
-  float* y;
+  void* y;           // fp32 [M][N], or bfloat16 [M][N] in the narrow-output kernels
   int32_t* acc_out;
   int32_t M, N, K;
   int32_t rows_per_group;
@@ -73,7 +74,7 @@ struct Problem {
 
 struct GroupedParams {
   CUtensorMap tmx[kMaxProblems];  // int8 activations, box 128 B x BT tokens, 128-byte swizzle
-  CUtensorMap tmy[kMaxProblems];  // fp32 outputs, box 32 neurons x 32 tokens
+  CUtensorMap tmy[kMaxProblems];  // outputs (fp32 or bfloat16), box 32 neurons x 32 tokens
   Problem prob[kMaxProblems];
   void* ws;
   int32_t count;
@@ -257,7 +258,8 @@ struct TileCursor {
   }
 };
 
-template <int BT, int BITS>
+// BF16: the epilogue rounds its fp32 result to bfloat16 (round to nearest even) and Y is bfloat16 [M][N].
+template <int BT, int BITS, bool BF16>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
   using Cfg = GemmCfg<BT>;
@@ -562,7 +564,8 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
       const int m0 = (local / pr.n_tiles) * BT;
       const bool nvalid = n < pN;
       const bool tma_store = pr.tma_store != 0;
-      float* const y_ptr = pr.y;
+      float* const y_ptr = reinterpret_cast<float*>(pr.y);
+      uint16_t* const y16_ptr = reinterpret_cast<uint16_t*>(pr.y);
       int32_t* const acc_ptr = pr.acc_out;
       float alpha = 0.f, beta = 0.f, b = 0.f;
       if (nvalid) {
@@ -628,8 +631,15 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
               if (lane == 0) ptx::tma_store_wait_read1();  // the store before last (same buffer) has read it
               __syncwarp();
             }
+            if constexpr (BF16) {  // rows of 32 bfloat16 (64 bytes): the first half of the fp32 buffer
+              uint16_t* buf16 = reinterpret_cast<uint16_t*>(buf);
 #pragma unroll
-            for (int j = 0; j < 16; ++j) buf[(16 * h + j) * 32 + lane] = yv[j];
+              for (int j = 0; j < 16; ++j)
+                buf16[(16 * h + j) * 32 + lane] = __bfloat16_as_ushort(__float2bfloat16_rn(yv[j]));
+            } else {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) buf[(16 * h + j) * 32 + lane] = yv[j];
+            }
           }
           ptx::fence_proxy_async_smem();
           __syncwarp();
@@ -640,6 +650,7 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
         }
         if (!tma_store || acc_ptr != nullptr) {
           float* yrow = y_ptr + (size_t)mc * pN + n;
+          uint16_t* yrow16 = y16_ptr + (size_t)mc * pN + n;
           int32_t* arow = acc_ptr ? acc_ptr + (size_t)mc * pN + n : nullptr;
           const int rows = min(32, pM - mc);  // warp-uniform
 #pragma unroll
@@ -651,7 +662,13 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
               const int j = 4 * q + i;
               const int ac = ((int)v[j]) >> (8 - BITS);
               if (nvalid && j < rows) {
-                if (!tma_store) yrow[(size_t)j * pN] = __fmaf_rn(alpha, (float)ac, __fmaf_rn(beta, rs[i], b));
+                if (!tma_store) {
+                  const float yv = __fmaf_rn(alpha, (float)ac, __fmaf_rn(beta, rs[i], b));
+                  if constexpr (BF16)
+                    yrow16[(size_t)j * pN] = __bfloat16_as_ushort(__float2bfloat16_rn(yv));
+                  else
+                    yrow[(size_t)j * pN] = yv;
+                }
                 if (arow) arow[(size_t)j * pN] = ac + c_code * __float2int_rn(rs[i]);
               }
             }
@@ -720,16 +737,18 @@ static qb_status make_x_tensormap(CUtensorMap* tm, const int8_t* xq, int64_t M, 
   return QB_OK;
 }
 
-// fp32 outputs [M][N], N contiguous; box = 32 neurons x 32 tokens, no swizzle (plain row-major in smem).
-static qb_status make_y_tensormap(CUtensorMap* tm, float* y, int64_t M, int64_t N) {
+// Outputs [M][N] (fp32 or bfloat16), N contiguous; box = 32 neurons x 32 tokens, no swizzle (plain row-major
+// in smem).
+static qb_status make_y_tensormap(CUtensorMap* tm, void* y, int64_t M, int64_t N, bool bf16) {
   EncodeTiledFn encode = nullptr;
   qb_status st = get_encode_fn(&encode);
   if (st != QB_OK) return st;
   const cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
-  const cuuint64_t strides[1] = {(cuuint64_t)N * 4};
+  const cuuint64_t strides[1] = {(cuuint64_t)N * (bf16 ? 2 : 4)};
   const cuuint32_t box[2] = {32, 32};
   const cuuint32_t elem[2] = {1, 1};
-  CUresult r = encode(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, y, dims, strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE,
+  CUresult r = encode(tm, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, y, dims, strides,
+                      box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE,
                       CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
     set_last_error("cuTensorMapEncodeTiled (outputs) failed with CUresult %d (M=%lld N=%lld)", (int)r, (long long)M,
@@ -739,10 +758,10 @@ static qb_status make_y_tensormap(CUtensorMap* tm, float* y, int64_t M, int64_t 
   return QB_OK;
 }
 
-template <int BT, int BITS>
+template <int BT, int BITS, bool BF16>
 static qb_status launch_group_inst(const GroupedParams& gp, int grid, cudaStream_t stream) {
   using Cfg = GemmCfg<BT>;
-  auto kernel = qb_gemm_kernel<BT, BITS>;
+  auto kernel = qb_gemm_kernel<BT, BITS, BF16>;
   static bool attr_set[64] = {};
   int dev = 0;
   QB_CUDA_TRY(cudaGetDevice(&dev));
@@ -755,13 +774,13 @@ static qb_status launch_group_inst(const GroupedParams& gp, int grid, cudaStream
   return QB_OK;
 }
 
-template <int BT>
+template <int BT, bool BF16>
 static qb_status launch_group_bits(int bits, const GroupedParams& gp, int grid, cudaStream_t stream) {
   switch (bits) {
-    case 2: return launch_group_inst<BT, 2>(gp, grid, stream);
-    case 3: return launch_group_inst<BT, 3>(gp, grid, stream);
-    case 4: return launch_group_inst<BT, 4>(gp, grid, stream);
-    case 8: return launch_group_inst<BT, 8>(gp, grid, stream);
+    case 2: return launch_group_inst<BT, 2, BF16>(gp, grid, stream);
+    case 3: return launch_group_inst<BT, 3, BF16>(gp, grid, stream);
+    case 4: return launch_group_inst<BT, 4, BF16>(gp, grid, stream);
+    case 8: return launch_group_inst<BT, 8, BF16>(gp, grid, stream);
     default: return QB_ERR_INVALID;
   }
 }
@@ -778,7 +797,7 @@ static int choose_token_tile(const qb_linear_desc* d, const int* idx, int count,
 
 static qb_status validate_gemm(const int8_t* xq, const float* act_scale, const int32_t* rowsum,
                                const uint32_t* packed, const float* delta, const float* q0, int64_t M, int64_t N,
-                               int64_t K, int bits, int groups, const float* y, const void* ws, size_t ws_bytes) {
+                               int64_t K, int bits, int groups, const void* y, const void* ws, size_t ws_bytes) {
   if (!xq || !act_scale || !rowsum || !packed || !delta || !q0 || !y || M <= 0 || N <= 0 || K <= 0 ||
       M > QB_MAX_MN || N > QB_MAX_MN || K > QB_MAX_K || !valid_bits(bits) || groups < 1 || N % groups != 0) {
     set_last_error("qb_gemm: invalid argument (M=%lld N=%lld K=%lld bits=%d groups=%d)", (long long)M,
@@ -799,7 +818,7 @@ static qb_status validate_gemm(const int8_t* xq, const float* act_scale, const i
 // One launch over descriptors d[idx[0..count)] (count <= kMaxProblems), all with the same bit width, on at
 // most `max_ctas` CTAs.
 static qb_status launch_group(const qb_linear_desc* d, const int* idx, int count, int32_t* acc_out, void* ws,
-                              int max_ctas, cudaStream_t stream) {
+                              int max_ctas, cudaStream_t stream, bool bf16) {
   const int sm_count = max_ctas;
   const int bits = d[idx[0]].bits;
   const int bt = choose_token_tile(d, idx, count, sm_count);
@@ -813,9 +832,9 @@ static qb_status launch_group(const qb_linear_desc* d, const int* idx, int count
     qb_status st = make_x_tensormap(&gp.tmx[i], q.xq, q.M, q.K, bt);
     if (st != QB_OK) return st;
     // Y rows 16-byte aligned: the epilogue stages tiles in shared memory and stores them with TMA
-    const bool tma_store = (q.N % 4 == 0) && aligned16(q.y);
+    const bool tma_store = (q.N % (bf16 ? 8 : 4) == 0) && aligned16(q.y);
     if (tma_store) {
-      st = make_y_tensormap(&gp.tmy[i], q.y, q.M, q.N);
+      st = make_y_tensormap(&gp.tmy[i], q.y, q.M, q.N, bf16);
       if (st != QB_OK) return st;
     } else {
       gp.tmy[i] = gp.tmx[i];  // unused by the kernel
@@ -877,7 +896,11 @@ static qb_status launch_group(const qb_linear_desc* d, const int* idx, int count
       }
     }
   }
-  return bt == 256 ? launch_group_bits<256>(bits, gp, grid, stream) : launch_group_bits<128>(bits, gp, grid, stream);
+  if (bf16)
+    return bt == 256 ? launch_group_bits<256, true>(bits, gp, grid, stream)
+                     : launch_group_bits<128, true>(bits, gp, grid, stream);
+  return bt == 256 ? launch_group_bits<256, false>(bits, gp, grid, stream)
+                   : launch_group_bits<128, false>(bits, gp, grid, stream);
 }
 
 // Side streams and events for launches of one stack that run side by side (host objects, created once per
@@ -916,7 +939,8 @@ static qb_status side_streams(SideStreams** out) {
 // total) runs its launches side by side, each on a share of the SMs in proportion to its work, so that
 // the start-up and the drain of the pipelines overlap instead of adding up; the launches join the
 // caller's stream before the call returns.  Large stacks keep one launch after the other on all SMs.
-static qb_status launch_stack(const qb_linear_desc* d, int count, void* ws, int sm_count, cudaStream_t stream) {
+static qb_status launch_stack(const qb_linear_desc* d, int count, void* ws, int sm_count, cudaStream_t stream,
+                              bool bf16) {
   std::vector<int> order(count);
   for (int i = 0; i < count; ++i) order[i] = i;
   std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
@@ -954,7 +978,7 @@ static qb_status launch_stack(const qb_linear_desc* d, int count, void* ws, int 
                             all_tiles < (int64_t)16 * sm_count;
   if (!side_by_side) {
     for (const Group& g : groups) {
-      qb_status st = launch_group(d, order.data() + g.begin, g.count, nullptr, ws, sm_count, stream);
+      qb_status st = launch_group(d, order.data() + g.begin, g.count, nullptr, ws, sm_count, stream, bf16);
       if (st != QB_OK) return st;
     }
     return QB_OK;
@@ -995,7 +1019,7 @@ static qb_status launch_stack(const qb_linear_desc* d, int count, void* ws, int 
   qb_status first_error = QB_OK;
   for (int g = 0; g < n_groups; ++g) {
     cudaStream_t sg = g == 0 ? stream : side->stream[g - 1];
-    st = launch_group(d, order.data() + groups[g].begin, groups[g].count, nullptr, ws, share[g], sg);
+    st = launch_group(d, order.data() + groups[g].begin, groups[g].count, nullptr, ws, share[g], sg, bf16);
     if (st != QB_OK && first_error == QB_OK) first_error = st;
   }
   // always join, also after an error: the caller's stream must not run ahead of the side streams
@@ -1008,10 +1032,11 @@ static qb_status launch_stack(const qb_linear_desc* d, int count, void* ws, int 
 
 }  // namespace qb
 
-extern "C" qb_status qb_gemm(const int8_t* xq, const float* act_scale, const int32_t* rowsum,
-                             const uint32_t* packed, const float* delta, const float* q0, const float* bias,
-                             int64_t M, int64_t N, int64_t K, int bits, int groups, float* y, int32_t* acc_out,
-                             void* ws, size_t ws_bytes, void* cuda_stream) {
+// fp32 or bfloat16 output: `y` is float* or uint16_t* (bfloat16 bit patterns) accordingly
+static qb_status gemm_entry(const int8_t* xq, const float* act_scale, const int32_t* rowsum, const uint32_t* packed,
+                            const float* delta, const float* q0, const float* bias, int64_t M, int64_t N, int64_t K,
+                            int bits, int groups, void* y, int32_t* acc_out, void* ws, size_t ws_bytes,
+                            void* cuda_stream, bool bf16) {
   qb_status st = qb::validate_gemm(xq, act_scale, rowsum, packed, delta, q0, M, N, K, bits, groups, y, ws, ws_bytes);
   if (st != QB_OK) return st;
   int sms = 0;
@@ -1030,15 +1055,15 @@ extern "C" qb_status qb_gemm(const int8_t* xq, const float* act_scale, const int
   d.K = K;
   d.bits = bits;
   d.groups = groups;
-  d.y = y;
+  d.y = static_cast<float*>(y);
   const int idx = 0;
-  return qb::launch_group(&d, &idx, 1, acc_out, ws, sms, (cudaStream_t)cuda_stream);
+  return qb::launch_group(&d, &idx, 1, acc_out, ws, sms, (cudaStream_t)cuda_stream, bf16);
 }
 
-extern "C" qb_status qb_layer_linears(const qb_linear_desc* descs, int32_t count, void* ws, size_t ws_bytes,
-                                      void* cuda_stream) {
+static qb_status stack_entry(const char* who, const qb_linear_desc* descs, int32_t count, void* ws, size_t ws_bytes,
+                             void* cuda_stream, bool bf16) {
   if (!descs || count <= 0) {
-    qb::set_last_error("qb_layer_linears: descs null or count <= 0");
+    qb::set_last_error("%s: descs null or count <= 0", who);
     return QB_ERR_INVALID;
   }
   for (int i = 0; i < count; ++i) {
@@ -1050,5 +1075,31 @@ extern "C" qb_status qb_layer_linears(const qb_linear_desc* descs, int32_t count
   int sms = 0;
   qb_status st = qb::require_sm100(&sms);
   if (st != QB_OK) return st;
-  return qb::launch_stack(descs, count, ws, sms, (cudaStream_t)cuda_stream);
+  return qb::launch_stack(descs, count, ws, sms, (cudaStream_t)cuda_stream, bf16);
+}
+
+extern "C" qb_status qb_gemm(const int8_t* xq, const float* act_scale, const int32_t* rowsum,
+                             const uint32_t* packed, const float* delta, const float* q0, const float* bias,
+                             int64_t M, int64_t N, int64_t K, int bits, int groups, float* y, int32_t* acc_out,
+                             void* ws, size_t ws_bytes, void* cuda_stream) {
+  return gemm_entry(xq, act_scale, rowsum, packed, delta, q0, bias, M, N, K, bits, groups, y, acc_out, ws, ws_bytes,
+                    cuda_stream, false);
+}
+
+extern "C" qb_status qb_gemm_bf16(const int8_t* xq, const float* act_scale, const int32_t* rowsum,
+                                  const uint32_t* packed, const float* delta, const float* q0, const float* bias,
+                                  int64_t M, int64_t N, int64_t K, int bits, int groups, uint16_t* y, void* ws,
+                                  size_t ws_bytes, void* cuda_stream) {
+  return gemm_entry(xq, act_scale, rowsum, packed, delta, q0, bias, M, N, K, bits, groups, y, nullptr, ws, ws_bytes,
+                    cuda_stream, true);
+}
+
+extern "C" qb_status qb_layer_linears(const qb_linear_desc* descs, int32_t count, void* ws, size_t ws_bytes,
+                                      void* cuda_stream) {
+  return stack_entry("qb_layer_linears", descs, count, ws, ws_bytes, cuda_stream, false);
+}
+
+extern "C" qb_status qb_layer_linears_bf16(const qb_linear_desc* descs, int32_t count, void* ws, size_t ws_bytes,
+                                           void* cuda_stream) {
+  return stack_entry("qb_layer_linears_bf16", descs, count, ws, ws_bytes, cuda_stream, true);
 }

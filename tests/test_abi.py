@@ -77,12 +77,18 @@ def test_argument_errors_are_returned_before_any_launch(lib):
     assert lib.qb_gemm(A, A, A, A, A, A, None, 8, 12, 128, 4, 3, None, None, A, ws_bytes, None) == qb.QB_ERR_INVALID
     assert lib.qb_gemm(A, A, A, A, A, A, None, 8, 12, 1 << 20, 4, 3, A, None, A, ws_bytes, None) == qb.QB_ERR_INVALID
     assert b"qb_gemm" in lib.qb_last_error()
+    # narrow-output forms: same validation
+    assert lib.qb_gemm_bf16(A, A, A, A, A, A, None, 8, 12, 128, 4, 5, A, A, ws_bytes, None) == qb.QB_ERR_INVALID
+    assert lib.qb_gemm_bf16(A, A, A, A, A, A, None, 8, 12, 192, 4, 3, A, A, ws_bytes, None) == qb.QB_ERR_ALIGN
+    assert lib.qb_gemm_bf16(A, A, A, A, A, A, None, 8, 12, 128, 4, 3, None, A, ws_bytes, None) == qb.QB_ERR_INVALID
     # stack: every descriptor is validated before the first launch
     good = qb.LinearDescC(A, A, A, A, A, A, None, 8, 12, 128, 4, 3, A)
     bad = qb.LinearDescC(A, A, A, A, A, A, None, 8, 12, 128, 7, 3, A)
     arr = (qb.LinearDescC * 2)(good, bad)
     assert lib.qb_layer_linears(arr, 2, A, ws_bytes, None) == qb.QB_ERR_INVALID
     assert lib.qb_layer_linears(None, 2, A, ws_bytes, None) == qb.QB_ERR_INVALID
+    assert lib.qb_layer_linears_bf16(arr, 2, A, ws_bytes, None) == qb.QB_ERR_INVALID
+    assert b"qb_layer_linears_bf16" in lib.qb_last_error() or b"qb_gemm" in lib.qb_last_error()
 
 
 def test_no_cpu_fallback_without_a_device(lib):
