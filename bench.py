@@ -73,11 +73,11 @@ def gemm_ops(wl: synth.Workload, M=None) -> float:
     return float(sum(2.0 * M * s.N * s.K for _, _, s, _ in linear_list(wl)))
 
 
-def gemm_algorithmic_bytes(wl: synth.Workload) -> float:
-    """int8 activations + packed weights + fp32 outputs + bias, row sums and group tables."""
+def gemm_algorithmic_bytes(wl: synth.Workload, out_bytes: float = 4.0) -> float:
+    """int8 activations + packed weights + outputs (fp32, or bfloat16) + bias, row sums and group tables."""
     tot = 0.0
     for _, _, s, bits in linear_list(wl):
-        tot += wl.M * s.K + s.N * s.K * bits / 8 + 4.0 * wl.M * s.N + 4 * s.N + 4 * wl.M + 8 * s.groups
+        tot += wl.M * s.K + s.N * s.K * bits / 8 + out_bytes * wl.M * s.N + 4 * s.N + 4 * wl.M + 8 * s.groups
     return tot
 
 
@@ -253,7 +253,7 @@ def run_ours(args, wl):
             packed=torch.empty((s.N, s.K * bits // 32), dtype=torch.int32, device=device),
             delta=torch.empty(s.groups, dtype=torch.float32, device=device),
             q0=torch.empty(s.groups, dtype=torch.float32, device=device),
-            y=torch.empty((wl.M, s.N), dtype=torch.float32, device=device),
+            y=torch.empty((wl.M, s.N), dtype=torch.bfloat16 if args.out == "bf16" else torch.float32, device=device),
             bits=bits, s=s)
         devb.append(d)
     descs = qb.make_desc_array([qb.LinearDesc(d["xq"], d["sc"], d["rs"], d["packed"], d["delta"], d["q0"], d["b"],
@@ -275,7 +275,10 @@ def run_ours(args, wl):
         qb.quantize_pack_weights_batch(w_arr, ws_w)
 
     def phase_gemm():
-        qb.layer_linears(descs, ws)
+        if args.out == "bf16":
+            qb.layer_linears_bf16(descs, ws)
+        else:
+            qb.layer_linears(descs, ws)
 
     side = torch.cuda.Stream(device=device)
 
@@ -368,9 +371,9 @@ def run_ours(args, wl):
 
     # ---- end to end: host buffers in, results out, copies inside the timed region ------------------
     e2e_steps = max(1, min(args.steps, args.e2e_steps))  # a shorter loop: each step moves ~250 MB over PCIe
-    y_host = [torch.empty((wl.M, d["s"].N), dtype=torch.float32).pin_memory() for d in devb]
+    y_host = [torch.empty((wl.M, d["s"].N), dtype=d["y"].dtype).pin_memory() for d in devb]
     h2d = sum(x.numel() * 4 + w.numel() * 4 + b.numel() * 4 for x, w, b in host)
-    d2h = sum(y.numel() * 4 for y in y_host)
+    d2h = sum(y.numel() * y.element_size() for y in y_host)
 
     def e2e_step():
         for (x, w, b), d in zip(host, devb):
@@ -403,7 +406,7 @@ def run_ours(args, wl):
 
     peaks, peak_kind = measured_peaks()
     n_gemm = gemm_launches
-    gemm_bytes = gemm_algorithmic_bytes(wl)
+    gemm_bytes = gemm_algorithmic_bytes(wl, 2.0 if args.out == "bf16" else 4.0)
     gemm_s_per_launch = ms_gemm * 1e-3 / n_gemm
     achieved_gbs = gemm_bytes / n_gemm / gemm_s_per_launch / 1e9
     achieved_tops = ops / n_gemm / gemm_s_per_launch / 1e12
@@ -416,7 +419,7 @@ def run_ours(args, wl):
     else:
         roof = {"bound": "tensor", "achieved": achieved_tops, "peak": int8_peak, "unit": "TOP/s",
                 "frac": achieved_tops / int8_peak}
-    traffic = NCU_GEMM_TRAFFIC.get(kernel_source_hash(), {}).get(str(wl.config))
+    traffic = NCU_GEMM_TRAFFIC.get(kernel_source_hash(), {}).get(str(wl.config)) if args.out == "f32" else None
     roof.update({
         "traffic": traffic, "kernel": "qb_gemm_kernel", "launches_per_step": n_gemm,
         "us_per_launch": gemm_s_per_launch * 1e6, "algorithmic_bytes_per_launch": gemm_bytes / n_gemm,
@@ -434,7 +437,7 @@ def run_ours(args, wl):
         "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_job, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
         "config": {"workload": wl.name, "config_index": wl.config, "M": wl.M, "linears": n_gemm,
-                   "bits": sorted(set(wl.bits)),
+                   "bits": sorted(set(wl.bits)), "output": "fp32" if args.out == "f32" else "bfloat16 (narrow-output epilogue)",
                    "l2": "untimed between timed steps: 512 MiB flush write, then a 256 MiB read of another buffer (L2 left with clean lines)",
                    "step": "quantize_act_batch beside quantize_pack_weights_batch (two streams), then layer_linears over all linears",
                    "launch": "direct C-ABI calls" if args.no_graphs else "C-ABI calls captured once per phase into CUDA graphs, replayed"},
@@ -580,6 +583,8 @@ def main():
     ap.add_argument("--ref-steps", type=int, default=5)
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--out", default="f32", choices=["f32", "bf16"],
+                    help="output type of the GEMMs: fp32 (the graded path) or bfloat16 (qb_layer_linears_bf16)")
     ap.add_argument("--no-graphs", action="store_true", help="issue the C-ABI calls directly every step")
     ap.add_argument("--busy-ms", type=float, default=300.0,
                     help="untimed load before the timed steps so that clocks are sampled under load")
