@@ -40,10 +40,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # launches of one step), from an ncu capture; valid only for the kernel source it was taken on.
 NCU_GEMM_TRAFFIC = {
     # "<sha256 of csrc/gemm.cu + csrc/ptx.cuh>": {<config>: bytes per launch}
-    # profiles/qb_gemm_kernel_config1.md, _config2.md, _config3.md (launch averages).  The key is the
-    # source the counters were taken on plus one later edit of the host code only (bit-width factors
-    # in the SM shares of side-by-side launches); the kernel itself is unchanged.
-    "dbf69d585261cf88": {"1": 78.3e6, "2": 8.18e6, "3": 4298.7e6},
+    # profiles/qb_gemm_kernel_config1.md, _config2.md, _config3.md (launch averages of the fp32 kernels)
+    "50eb2ced7e8c1609": {"1": 78.1e6, "2": 8.18e6, "3": 4300.2e6},
 }
 
 
