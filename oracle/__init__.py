@@ -57,6 +57,8 @@ def _lib(omp: bool = False) -> ctypes.CDLL:
         lib.qo_pack.restype = i32
         lib.qo_unpack.argtypes = [vp, i64, i64, i32, vp]
         lib.qo_unpack.restype = i32
+        lib.qo_ste_backward.argtypes = [vp, vp, i64, i64, i32, vp, vp, vp]
+        lib.qo_ste_backward.restype = None
         lib.qo_round_bf16.argtypes = [vp, i64, vp]
         lib.qo_round_bf16.restype = None
         lib.qo_quantize_act.argtypes = [vp, i64, i64, vp, vp, vp]
@@ -207,4 +209,22 @@ def round_bf16(y) -> np.ndarray:
     y = _c(np.asarray(y), np.float32)
     out = np.empty(y.shape, dtype=np.uint16)
     _lib().qo_round_bf16(_p(y), y.size, _p(out))
+    return out
+
+
+def fake_quantize_weights(w, bits: int, groups: int, range_lo=None, range_hi=None, omp: bool = False):
+    """Q(W) of Appendix A in fp32: (status, Q(w) [N,K], delta [G], q0 [G]); quantize, then Delta * code + q0."""
+    st, codes, delta, q0 = quantize_weights(w, bits, groups, range_lo, range_hi, omp=omp)
+    return st, dequantize_weights(codes, groups, delta, q0), delta, q0
+
+
+def ste_backward(grad_q, w, groups: int, lo, hi) -> np.ndarray:
+    """Straight-through gradient of the quantizer: grad_q where lo_g <= w <= hi_g, else 0."""
+    grad_q = _c(grad_q, np.float32)
+    w = _c(w, np.float32)
+    lo = _c(lo, np.float32)
+    hi = _c(hi, np.float32)
+    N, K = w.shape
+    out = np.empty((N, K), dtype=np.float32)
+    _lib().qo_ste_backward(_p(grad_q), _p(w), N, K, groups, _p(lo), _p(hi), _p(out))
     return out

@@ -310,4 +310,23 @@ void qo_round_bf16(const float* y, int64_t n, uint16_t* out) {
   }
 }
 
+// Backward pass of the quantizer for quantization-aware fine-tuning (Section 3.1 and Appendix A: the
+// straight-through estimator is used for the gradient of X).  Q is Clamp followed by rounding onto the
+// grid; the estimator treats the rounding as the identity, so the gradient of the loss with respect
+// to X is the gradient with respect to Q(X) where Clamp passes X through (q0 <= X <= qmax of its
+// group, both ends included) and zero where Clamp holds X at an end of the range.  With the default
+// range [min, max] of the group every element is inside and the gradient passes unchanged.
+// lo, hi: per group, [G]; rows of W are grouped as in qo_quantize_weights.
+void qo_ste_backward(const float* grad_q, const float* w, int64_t N, int64_t K, int groups, const float* lo,
+                     const float* hi, float* grad_w) {
+  const int64_t R = N / groups;
+  for (int64_t n = 0; n < N; ++n) {
+    const int64_t g = n / R;
+    for (int64_t k = 0; k < K; ++k) {
+      const float x = w[n * K + k];
+      grad_w[n * K + k] = (x >= lo[g] && x <= hi[g]) ? grad_q[n * K + k] : 0.0f;
+    }
+  }
+}
+
 }  // extern "C"
