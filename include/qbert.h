@@ -245,6 +245,34 @@ qb_status qb_layer_linears_bf16(const qb_linear_desc* descs /*host*/, int32_t co
                                 size_t ws_bytes, void* cuda_stream);
 
 /*
+ * Quantization-aware fine-tuning (Section 3.1: gradients pass through Q by the straight-through
+ * estimator; Appendix A: forward and backward of the quantization process).
+ *
+ * Forward ("fake quantization"): the quantizer of qb_quantize_pack_weights, but the result is the
+ * dequantized tensor Q(W) = Delta_g * code + q0_g in fp32 (one fused multiply-add per element, on the
+ * codes and the Delta, q0 that qb_quantize_pack_weights computes for the same arguments).
+ *   w        dev fp32 [N][K], 16-byte aligned                     (read)
+ *   wq       dev fp32 [N][K], 16-byte aligned                     (written)
+ *   delta,q0 dev fp32 [G]                                         (written)
+ *   range_lo, range_hi: dev fp32 [G] or both NULL, as for qb_quantize_pack_weights.
+ * Two kernels: per-group min/max reduction into the workspace, then round/clamp/dequantize.
+ *
+ * Backward: grad_w = grad_wq where Clamp passes the weight through (range_lo[g] <= w <= range_hi[g],
+ * both ends included), 0 where Clamp holds it at an end of the range; the rounding is treated as the
+ * identity.  With range_lo = range_hi = NULL (the group's own [min, max]) every weight is inside
+ * and the call copies grad_wq to grad_w (nothing is done if they are the same buffer).
+ *   grad_wq  dev fp32 [N][K], gradient with respect to Q(W)       (read)
+ *   w        dev fp32 [N][K], the weights that were quantized     (read)
+ *   grad_w   dev fp32 [N][K]                                      (written; may alias grad_wq)
+ * All three 16-byte aligned.  No workspace, no device-side status.
+ */
+qb_status qb_fake_quantize_weights(const float* w, int64_t N, int64_t K, int bits, int groups,
+                                   const float* range_lo, const float* range_hi, float* wq, float* delta,
+                                   float* q0, void* ws, size_t ws_bytes, void* cuda_stream);
+qb_status qb_ste_backward(const float* grad_wq, const float* w, int64_t N, int64_t K, int groups,
+                          const float* range_lo, const float* range_hi, float* grad_w, void* cuda_stream);
+
+/*
  * Diagnostic: the rate the tensor cores sustain for the GEMM's own instruction (tcgen05.mma kind::i8,
  * s8 x s8 -> s32, 128 x `tokens` x 32) with both operands resident in shared memory, no global
  * traffic, four K blocks in flight, one CTA per SM on the default stream.  (No counterpart in the

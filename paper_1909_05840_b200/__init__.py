@@ -31,6 +31,7 @@ EXPORTS = (
     "qb_workspace_init", "qb_read_status", "qb_quantize_act", "qb_quantize_pack_weights", "qb_gemm",
     "qb_layer_linears", "qb_quantize_pack_weights_noalloc", "qb_probe_i8_mma", "qb_quantize_act_batch",
     "qb_quantize_pack_weights_batch", "qb_gemm_bf16", "qb_layer_linears_bf16",
+    "qb_fake_quantize_weights", "qb_ste_backward",
 )
 NOALLOC_MAX_GROUPS = 4096
 
@@ -107,6 +108,10 @@ def lib() -> ctypes.CDLL:
     L.qb_gemm.restype = i32
     L.qb_layer_linears.argtypes = [ctypes.POINTER(LinearDescC), i32, vp, sz, vp]
     L.qb_layer_linears.restype = i32
+    L.qb_fake_quantize_weights.argtypes = [vp, i64, i64, ctypes.c_int, ctypes.c_int, vp, vp, vp, vp, vp, vp, sz, vp]
+    L.qb_fake_quantize_weights.restype = i32
+    L.qb_ste_backward.argtypes = [vp, vp, i64, i64, ctypes.c_int, vp, vp, vp, vp]
+    L.qb_ste_backward.restype = i32
     L.qb_gemm_bf16.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, ctypes.c_int, ctypes.c_int, vp, vp, sz, vp]
     L.qb_gemm_bf16.restype = i32
     L.qb_layer_linears_bf16.argtypes = [ctypes.POINTER(LinearDescC), i32, vp, sz, vp]
@@ -183,6 +188,32 @@ def quantize_pack_weights(w: torch.Tensor, bits: int, groups: int, ws: torch.Ten
                                           packed.data_ptr(), delta.data_ptr(), q0.data_ptr(), ws.data_ptr(),
                                           ws.numel(), _stream()), "qb_quantize_pack_weights")
     return packed, delta, q0
+
+
+def fake_quantize_weights(w: torch.Tensor, bits: int, groups: int, ws: torch.Tensor,
+                          range_lo: Optional[torch.Tensor] = None, range_hi: Optional[torch.Tensor] = None,
+                          wq: Optional[torch.Tensor] = None):
+    """``qb_fake_quantize_weights``: fp32 [N,K] -> (Q(W) fp32 [N,K], delta [G], q0 [G])."""
+    assert w.is_cuda and w.dtype == torch.float32 and w.dim() == 2 and w.is_contiguous()
+    N, K = w.shape
+    wq = torch.empty_like(w) if wq is None else wq
+    delta = torch.empty(groups, dtype=torch.float32, device=w.device)
+    q0 = torch.empty(groups, dtype=torch.float32, device=w.device)
+    _check(lib().qb_fake_quantize_weights(w.data_ptr(), N, K, bits, groups, _ptr(range_lo), _ptr(range_hi),
+                                          wq.data_ptr(), delta.data_ptr(), q0.data_ptr(), ws.data_ptr(), ws.numel(),
+                                          _stream()), "qb_fake_quantize_weights")
+    return wq, delta, q0
+
+
+def ste_backward(grad_wq: torch.Tensor, w: torch.Tensor, groups: int, range_lo: Optional[torch.Tensor] = None,
+                 range_hi: Optional[torch.Tensor] = None, grad_w: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """``qb_ste_backward``: straight-through gradient of the quantizer with respect to the weights."""
+    assert grad_wq.is_cuda and grad_wq.dtype == torch.float32 and grad_wq.is_contiguous() and grad_wq.shape == w.shape
+    N, K = w.shape
+    grad_w = torch.empty_like(w) if grad_w is None else grad_w
+    _check(lib().qb_ste_backward(grad_wq.data_ptr(), w.data_ptr(), N, K, groups, _ptr(range_lo), _ptr(range_hi),
+                                 grad_w.data_ptr(), _stream()), "qb_ste_backward")
+    return grad_w
 
 
 def make_act_desc_array(items):

@@ -315,6 +315,80 @@ weight_pack_kernel(const __grid_constant__ WeightBatch b) {
   }
 }
 
+// ---- fake quantization (quantization-aware fine-tuning) ------------------------------------------------
+// Forward: Q(W) = Delta * X^I + q0 in fp32 (Appendix A), same walk and same codes as weight_pack_kernel;
+// the four values of a lane are written as one float4 (`packed` of the item points to the fp32 output).
+__global__ void __launch_bounds__(kWqThreads)
+weight_fake_kernel(const __grid_constant__ WeightBatch b, int levels) {
+  const int lane = threadIdx.x & 31;
+  const int64_t gwarp = (int64_t)blockIdx.x * kWqWarps + (threadIdx.x >> 5);
+  int64_t u = gwarp * b.units_per_warp;
+  int64_t u_end = u + b.units_per_warp;
+  if (u_end > b.units_total) u_end = b.units_total;
+  if (u >= u_end) return;
+  UnitWalk pos;
+  pos.seek(b, u);
+  int cur_g = -1;
+  GroupParams gp{0.f, 0.f, 1.f};
+  float d = 1.0f;
+  while (u < u_end) {
+    const WeightItem& m = b.item[pos.it];
+    const int nload = (int)min(min((int64_t)4, u_end - u), m.units - pos.u_local);
+    float4 v[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      if (j < nload) v[j] = __ldg(m.w + (pos.u_local + j) * 32 + lane);
+    float4* const out_base = reinterpret_cast<float4*>(m.packed) + pos.u_local * 32;
+    const int group_begin = m.group_begin;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (j < nload) {
+        if (pos.g != cur_g) {  // warp-uniform
+          cur_g = pos.g;
+          const bool publish = lane == 0 && pos.row_in_group == 0 && pos.col_unit == 0;
+          gp = load_group(cur_g - group_begin, levels, b.hi_enc + group_begin, b.lo_inv + group_begin, m.range_lo,
+                          m.range_hi, m.delta, m.q0, publish, b.ws);
+          // Delta as finish_group publishes it (a constant group comes back with hi == lo: Delta = 1)
+          d = __fdiv_rn(__fsub_rn(gp.hi, gp.lo), (float)levels);
+          if (!(d > 0.0f)) d = 1.0f;
+        }
+        const float e[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
+        float q[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float xc = fminf(fmaxf(e[i], gp.lo), gp.hi);        // Clamp(X, q0, qmax)
+          const float t = __fmul_rn(__fsub_rn(xc, gp.lo), gp.inv);  // (X' - q0) * (1/Delta)
+          int c = __float2int_rn(t);                                // round half to even
+          c = min(max(c, 0), levels);
+          q[i] = __fmaf_rn(d, (float)c, gp.lo);                     // Delta * X^I + q0
+        }
+        out_base[j * 32 + lane] = make_float4(q[0], q[1], q[2], q[3]);
+        pos.advance(b);
+      }
+    }
+    u += nload;
+  }
+}
+
+// Backward (straight-through estimator): the gradient passes where Clamp passes X (lo_g <= x <= hi_g).
+__global__ void __launch_bounds__(256)
+ste_backward_kernel(const float4* __restrict__ grad_q, const float4* __restrict__ w, int64_t n4, int64_t k4,
+                    int64_t rows_per_group, const float* __restrict__ lo, const float* __restrict__ hi,
+                    float4* __restrict__ grad_w) {
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+    const int64_t g = (i / k4) / rows_per_group;
+    const float l = __ldg(lo + g), h = __ldg(hi + g);
+    const float4 x = __ldg(w + i);
+    float4 gq = __ldg(grad_q + i);
+    gq.x = (x.x >= l && x.x <= h) ? gq.x : 0.0f;
+    gq.y = (x.y >= l && x.y <= h) ? gq.y : 0.0f;
+    gq.z = (x.z >= l && x.z <= h) ? gq.z : 0.0f;
+    gq.w = (x.w >= l && x.w <= h) ? gq.w : 0.0f;
+    grad_w[i] = gq;
+  }
+}
+
 // ---- single-read path ------------------------------------------------------------------------------
 // When a whole group fits in shared memory the matrix is read from HBM once.  A persistent CTA per SM
 // takes groups round-robin.  Four producer lanes (in warps of their own) stream the CTA's groups as bulk
@@ -844,6 +918,43 @@ static qb_status launch_weight_batch(const HostWeight* m, int count, int bits, v
   return QB_OK;
 }
 
+// Fake quantization of one matrix: the range kernel of the two-pass path, then weight_fake_kernel.
+static qb_status launch_fake_quantize(const float* w, int64_t N, int64_t K, int bits, int groups,
+                                      const float* range_lo, const float* range_hi, float* wq, float* delta,
+                                      float* q0, void* ws, int sm_count, cudaStream_t stream) {
+  WeightBatch b;
+  memset(&b, 0, sizeof(b));
+  WeightItem& it = b.item[0];
+  it.w = reinterpret_cast<const float4*>(w);
+  it.packed = reinterpret_cast<uint32_t*>(wq);
+  it.delta = delta;
+  it.q0 = q0;
+  it.range_lo = range_lo;
+  it.range_hi = range_hi;
+  it.unit_begin = 0;
+  it.units = N * K / 128;
+  it.units_per_row = (int32_t)(K / 128);
+  it.rows_per_group = (int32_t)(N / groups);
+  it.group_begin = 0;
+  b.count = 1;
+  b.ws = ws;
+  b.hi_enc = reinterpret_cast<uint32_t*>(static_cast<char*>(ws) + kWsRangeOff);
+  b.lo_inv = b.hi_enc + groups;
+  b.units_total = it.units;
+  QB_CUDA_TRY(cudaMemsetAsync(b.hi_enc, 0, sizeof(uint32_t) * 2 * (size_t)groups, stream));
+  const int64_t max_warps = (int64_t)sm_count * 32;
+  int64_t upw = (it.units + max_warps - 1) / max_warps;
+  if (upw < 4) upw = 4;
+  b.units_per_warp = upw;
+  const int64_t warps = (it.units + upw - 1) / upw;
+  const unsigned blocks = (unsigned)((warps + kWqWarps - 1) / kWqWarps);
+  weight_range_kernel<<<blocks, kWqThreads, 0, stream>>>(b);
+  QB_CUDA_TRY(cudaGetLastError());
+  weight_fake_kernel<<<blocks, kWqThreads, 0, stream>>>(b, (1 << bits) - 1);
+  QB_CUDA_TRY(cudaGetLastError());
+  return QB_OK;
+}
+
 qb_status launch_quantize_pack_weights(const float* w, int64_t N, int64_t K, int bits, int groups,
                                        const float* range_lo, const float* range_hi, uint32_t* packed,
                                        float* delta, float* q0, void* ws, int sm_count, cudaStream_t stream) {
@@ -928,5 +1039,56 @@ extern "C" qb_status qb_quantize_pack_weights_batch(const qb_weight_desc* descs,
     st = qb::launch_weight_batch(m, n, bits, ws, sms, (cudaStream_t)cuda_stream);
     if (st != QB_OK) return st;
   }
+  return QB_OK;
+}
+
+extern "C" qb_status qb_fake_quantize_weights(const float* w, int64_t N, int64_t K, int bits, int groups,
+                                              const float* range_lo, const float* range_hi, float* wq, float* delta,
+                                              float* q0, void* ws, size_t ws_bytes, void* cuda_stream) {
+  qb_status st = qb::validate_weight("qb_fake_quantize_weights", w, N, K, bits, groups, range_lo, range_hi,
+                                     reinterpret_cast<const uint32_t*>(wq), delta, q0);
+  if (st != QB_OK) return st;
+  if (!ws || ws_bytes < qb::ws_bytes_needed(groups)) {
+    qb::set_last_error("qb_fake_quantize_weights: workspace null or smaller than %zu bytes",
+                       qb::ws_bytes_needed(groups));
+    return QB_ERR_WORKSPACE;
+  }
+  int sms = 0;
+  st = qb::require_sm100(&sms);
+  if (st != QB_OK) return st;
+  return qb::launch_fake_quantize(w, N, K, bits, groups, range_lo, range_hi, wq, delta, q0, ws, sms,
+                                  (cudaStream_t)cuda_stream);
+}
+
+extern "C" qb_status qb_ste_backward(const float* grad_wq, const float* w, int64_t N, int64_t K, int groups,
+                                     const float* range_lo, const float* range_hi, float* grad_w,
+                                     void* cuda_stream) {
+  if (!grad_wq || !w || !grad_w || N <= 0 || K <= 0 || N > QB_MAX_MN || K > QB_MAX_K || groups < 1 ||
+      N % groups != 0 || ((range_lo == nullptr) != (range_hi == nullptr))) {
+    qb::set_last_error("qb_ste_backward: invalid argument (N=%lld K=%lld groups=%d)", (long long)N, (long long)K,
+                       groups);
+    return QB_ERR_INVALID;
+  }
+  if (K % 128 != 0 || !qb::aligned16(grad_wq) || !qb::aligned16(w) || !qb::aligned16(grad_w)) {
+    qb::set_last_error("qb_ste_backward: K must be a multiple of 128 and grad_wq, w, grad_w 16-byte aligned");
+    return QB_ERR_ALIGN;
+  }
+  int sms = 0;
+  qb_status st = qb::require_sm100(&sms);
+  if (st != QB_OK) return st;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  if (range_lo == nullptr) {  // the group's own [min, max]: every element is inside, the gradient passes unchanged
+    if (grad_w != grad_wq)
+      QB_CUDA_TRY(cudaMemcpyAsync(grad_w, grad_wq, sizeof(float) * (size_t)N * (size_t)K, cudaMemcpyDeviceToDevice,
+                                  stream));
+    return QB_OK;
+  }
+  const int64_t n4 = N * K / 4;
+  int64_t blocks = (n4 + 256 * 4 - 1) / (256 * 4);
+  if (blocks > (int64_t)sms * 8) blocks = (int64_t)sms * 8;
+  qb::ste_backward_kernel<<<(unsigned)blocks, 256, 0, stream>>>(
+      reinterpret_cast<const float4*>(grad_wq), reinterpret_cast<const float4*>(w), n4, K / 4, N / groups, range_lo,
+      range_hi, reinterpret_cast<float4*>(grad_w));
+  QB_CUDA_TRY(cudaGetLastError());
   return QB_OK;
 }

@@ -81,6 +81,13 @@ def test_argument_errors_are_returned_before_any_launch(lib):
     assert lib.qb_gemm_bf16(A, A, A, A, A, A, None, 8, 12, 128, 4, 5, A, A, ws_bytes, None) == qb.QB_ERR_INVALID
     assert lib.qb_gemm_bf16(A, A, A, A, A, A, None, 8, 12, 192, 4, 3, A, A, ws_bytes, None) == qb.QB_ERR_ALIGN
     assert lib.qb_gemm_bf16(A, A, A, A, A, A, None, 8, 12, 128, 4, 3, None, A, ws_bytes, None) == qb.QB_ERR_INVALID
+    # fake quantization and its straight-through backward
+    assert lib.qb_fake_quantize_weights(A, 12, 128, 5, 1, None, None, A, A, A, A, ws_bytes, None) == qb.QB_ERR_INVALID
+    assert lib.qb_fake_quantize_weights(A, 12, 100, 4, 3, None, None, A, A, A, A, ws_bytes, None) == qb.QB_ERR_ALIGN
+    assert lib.qb_fake_quantize_weights(A, 12, 128, 4, 3, None, None, A, A, A, None, ws_bytes, None) == qb.QB_ERR_WORKSPACE
+    assert lib.qb_ste_backward(A, A, 12, 128, 5, None, None, A, None) == qb.QB_ERR_INVALID
+    assert lib.qb_ste_backward(A, A, 12, 128, 3, A, None, A, None) == qb.QB_ERR_INVALID
+    assert lib.qb_ste_backward(A, A + 4, 12, 128, 3, None, None, A, None) == qb.QB_ERR_ALIGN
     # stack: every descriptor is validated before the first launch
     good = qb.LinearDescC(A, A, A, A, A, A, None, 8, 12, 128, 4, 3, A)
     bad = qb.LinearDescC(A, A, A, A, A, A, None, 8, 12, 128, 7, 3, A)

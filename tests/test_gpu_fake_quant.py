@@ -1,0 +1,83 @@
+"""Fake quantization (forward Q(W) in fp32) and the straight-through backward on the GPU, against the
+oracle: both are bit-exact (the forward runs the same IEEE operations in the same order; the backward
+only selects)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_1909_05840_b200 as qb
+from paper_1909_05840_b200 import synth
+
+import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ws():
+    return qb.workspace(groups=4096)
+
+
+@pytest.mark.parametrize("bits", (2, 3, 4, 8))
+@pytest.mark.parametrize("N,K,groups", [(768, 768, 12), (264, 384, 11), (96, 3072, 96), (128, 128, 1), (3072, 768, 128)])
+def test_fake_quantize_matches_oracle(ws, bits, N, K, groups):
+    w = synth.weights(N, K, seed=3 * N + K + groups + bits)
+    wq = gu.poison(torch.empty((N, K), dtype=torch.float32, device="cuda"))
+    wq, delta, q0 = qb.fake_quantize_weights(gu.dev(w), bits, groups, ws, wq=wq)
+    assert qb.read_status(ws) == qb.QB_OK
+    st, o_q, o_delta, o_q0 = oracle.fake_quantize_weights(w, bits, groups)
+    assert st == oracle.OK
+    assert np.array_equal(delta.cpu().numpy(), o_delta) and np.array_equal(q0.cpu().numpy(), o_q0)
+    assert np.array_equal(wq.cpu().numpy().view(np.uint32), o_q.view(np.uint32))
+    # and it is the dequantized form of what the packer stores
+    packed, d2, z2 = qb.quantize_pack_weights(gu.dev(w), bits, groups, ws)
+    codes = oracle.unpack(gu.words_np(packed), K, bits)
+    assert np.array_equal(oracle.dequantize_weights(codes, groups, d2.cpu().numpy(), z2.cpu().numpy()).view(np.uint32),
+                          wq.cpu().numpy().view(np.uint32))
+
+
+def test_fake_quantize_clipped_ranges_constant_group_and_nonfinite(ws):
+    N, K, G = 64, 256, 4
+    w = synth.weights(N, K, seed=21)
+    w[16:32] = 0.25                                   # a constant group
+    lo = np.quantile(w.reshape(G, -1), 0.02, axis=1).astype(np.float32)
+    hi = np.quantile(w.reshape(G, -1), 0.98, axis=1).astype(np.float32)
+    for bits in (2, 3, 4, 8):
+        wq, delta, q0 = qb.fake_quantize_weights(gu.dev(w), bits, G, ws)
+        st, o_q, o_delta, o_q0 = oracle.fake_quantize_weights(w, bits, G)
+        assert np.array_equal(wq.cpu().numpy().view(np.uint32), o_q.view(np.uint32))
+        assert delta.cpu().numpy()[1] == 1.0 and np.all(wq.cpu().numpy()[16:32] == 0.25)
+        wq, delta, q0 = qb.fake_quantize_weights(gu.dev(w), bits, G, ws, gu.dev(lo), gu.dev(hi))
+        st, o_q, o_delta, o_q0 = oracle.fake_quantize_weights(w, bits, G, lo, hi)
+        assert np.array_equal(wq.cpu().numpy().view(np.uint32), o_q.view(np.uint32))
+        assert np.array_equal(delta.cpu().numpy(), o_delta) and np.array_equal(q0.cpu().numpy(), o_q0)
+    assert qb.read_status(ws) == qb.QB_OK
+    bad = w.copy(); bad[3, 7] = np.inf
+    ws2 = qb.workspace(groups=64)
+    qb.fake_quantize_weights(gu.dev(bad), 4, G, ws2)
+    assert qb.read_status(ws2) == qb.QB_ERR_NONFINITE
+
+
+@pytest.mark.parametrize("N,K,groups", [(768, 768, 12), (264, 384, 11), (3072, 768, 128), (8, 128, 1)])
+def test_ste_backward_matches_oracle(N, K, groups):
+    rng = np.random.default_rng(N + K)
+    w = synth.weights(N, K, seed=N + groups)
+    grad = rng.standard_normal((N, K)).astype(np.float32)
+    lo = np.quantile(w.reshape(groups, -1), 0.05, axis=1).astype(np.float32)
+    hi = np.quantile(w.reshape(groups, -1), 0.95, axis=1).astype(np.float32)
+    w[0, 0], w[0, 1] = lo[0], hi[0]                  # the ends of the range count as inside
+    out = gu.poison(torch.empty((N, K), dtype=torch.float32, device="cuda"))
+    qb.ste_backward(gu.dev(grad), gu.dev(w), groups, gu.dev(lo), gu.dev(hi), grad_w=out)
+    ref = oracle.ste_backward(grad, w, groups, lo, hi)
+    assert np.array_equal(out.cpu().numpy().view(np.uint32), ref.view(np.uint32))
+    assert 0 < (ref == 0).sum() < ref.size
+    # default range: the gradient passes unchanged, also in place
+    out2 = qb.ste_backward(gu.dev(grad), gu.dev(w), groups)
+    assert np.array_equal(out2.cpu().numpy(), grad)
+    g_dev = gu.dev(grad)
+    assert qb.ste_backward(g_dev, gu.dev(w), groups, grad_w=g_dev) is g_dev and np.array_equal(g_dev.cpu().numpy(), grad)
+    # masked in place
+    g_dev = gu.dev(grad)
+    qb.ste_backward(g_dev, gu.dev(w), groups, gu.dev(lo), gu.dev(hi), grad_w=g_dev)
+    assert np.array_equal(g_dev.cpu().numpy(), ref)
