@@ -548,6 +548,28 @@ def run_quantizer_sweep(args):
     ws = qb.workspace(groups=64, device=dev)
     ms_act = timed(lambda: qb.quantize_act(x, ws, xq, sc, rs))
     act_gbs = (9.0 * M * K + 4 * M) / (ms_act * 1e-3) / 1e9
+    # fake quantization and its straight-through backward on the largest encoder matrix shape, one
+    # matrix per call (single-matrix entry points): 3072 x 768 at 128 groups, and the 768 x 30720 table
+    fq = {}
+    for n, k in ((3072, 768), (768, 30720)):
+        w = torch.from_numpy(synth.weights(n, k, synth.seed_for(4, 1, n))).to(dev)
+        wq = torch.empty_like(w)
+        grad = torch.randn_like(w)
+        gout = torch.empty_like(w)
+        wsf = qb.workspace(groups=128, device=dev)
+        lo = torch.full((128,), -0.05, device=dev)
+        hi = torch.full((128,), 0.05, device=dev)
+        ms_f = timed(lambda: qb.fake_quantize_weights(w, 4, 128, wsf, wq=wq))
+        ms_b = timed(lambda: qb.ste_backward(grad, w, 128, lo, hi, grad_w=gout))
+        fq[f"{n}x{k}"] = {
+            "fake_quantize_k4_g128": {"ms": ms_f, "GBps": 8.0 * n * k / (ms_f * 1e-3) / 1e9,
+                                      "frac_hbm": 8.0 * n * k / (ms_f * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                      "bytes": "8 B per weight (one DRAM read, one write; the second read hits L2)"},
+            "ste_backward": {"ms": ms_b, "GBps": 12.0 * n * k / (ms_b * 1e-3) / 1e9,
+                             "frac_hbm": 12.0 * n * k / (ms_b * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                             "bytes": "12 B per weight (gradient and weight read, gradient written)"}}
+        launches += 3 * (3 + steps)
+        del w, wq, grad, gout
     best = max(table.values(), key=lambda r: r["frac_hbm"])
     line = {
         "metric": METRIC, "value": act_gbs, "unit": "GB/s", "n_gpus": 1, "steps": steps, "warmup": 3,
@@ -566,6 +588,7 @@ def run_quantizer_sweep(args):
                          "useful_5B_per_element_GBps": 5.0 * M * K / (ms_act * 1e-3) / 1e9},
         "quantize_pack_weights": table,
         "quantize_pack_weights_best_frac_hbm": best["frac_hbm"],
+        "fine_tuning": fq,
     }
     print(json.dumps(line))
 
