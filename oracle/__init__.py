@@ -57,6 +57,10 @@ def _lib(omp: bool = False) -> ctypes.CDLL:
         lib.qo_pack.restype = i32
         lib.qo_unpack.argtypes = [vp, i64, i64, i32, vp]
         lib.qo_unpack.restype = i32
+        lib.qo_quantize_embedding.argtypes = [vp, i64, i64, i32, i32, vp, vp, vp]
+        lib.qo_quantize_embedding.restype = i32
+        lib.qo_embedding_lookup.argtypes = [vp, i64, vp, i64, i64, i32, vp, vp, i32, vp]
+        lib.qo_embedding_lookup.restype = i32
         lib.qo_ste_backward.argtypes = [vp, vp, i64, i64, i32, vp, vp, vp]
         lib.qo_ste_backward.restype = None
         lib.qo_round_bf16.argtypes = [vp, i64, vp]
@@ -227,4 +231,28 @@ def ste_backward(grad_q, w, groups: int, lo, hi) -> np.ndarray:
     N, K = w.shape
     out = np.empty((N, K), dtype=np.float32)
     _lib().qo_ste_backward(_p(grad_q), _p(w), N, K, groups, _p(lo), _p(hi), _p(out))
+    return out
+
+
+def quantize_embedding(e, bits: int, groups: int):
+    """Column-group quantizer of an embedding table E [V,D]: (status, codes uint8 [V,D], delta [G], q0 [G])."""
+    e = _c(e, np.float32)
+    V, D = e.shape
+    codes = np.empty((V, D), dtype=np.uint8)
+    delta = np.empty(groups, dtype=np.float32)
+    q0 = np.empty(groups, dtype=np.float32)
+    st = _lib().qo_quantize_embedding(_p(e), V, D, bits, groups, _p(codes), _p(delta), _p(q0))
+    return st, codes, delta, q0
+
+
+def embedding_lookup(ids, codes, groups: int, delta, q0, out=None) -> np.ndarray:
+    """Dequantizing lookup; with ``out`` given the looked-up rows are added to it."""
+    ids = _c(ids, np.int32)
+    codes = _c(codes, np.uint8)
+    V, D = codes.shape
+    acc = out is not None
+    out = np.empty((ids.size, D), dtype=np.float32) if out is None else _c(out, np.float32).copy()
+    st = _lib().qo_embedding_lookup(_p(ids), ids.size, _p(codes), V, D, groups, _p(_c(delta, np.float32)),
+                                    _p(_c(q0, np.float32)), int(acc), _p(out))
+    assert st == OK, "id out of range"
     return out

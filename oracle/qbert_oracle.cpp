@@ -329,4 +329,78 @@ void qo_ste_backward(const float* grad_q, const float* w, int64_t N, int64_t K, 
   }
 }
 
+// ---------------------------------------------------------------------------
+// Embedding tables (Section 5.1 and the appendix on mixed-precision embedding: the 768 output
+// neurons of the word and position embedding layers are bucketed into 128 groups; 4-bit word and
+// 8-bit position embedding).  The table is stored as it is looked up, E[v][d] (one row per
+// vocabulary entry or position, D embedding dimensions), so a group is a block of D / G consecutive
+// COLUMNS over all V rows.  Per group the quantizer is Appendix A's Q with the group's exact
+// [min, max], as in qo_quantize_weights; codes[v][d] in {0 .. 2^k - 1}.
+// ---------------------------------------------------------------------------
+int qo_quantize_embedding(const float* e, int64_t V, int64_t D, int bits, int groups, uint8_t* codes,
+                          float* delta, float* q0) {
+  if (!e || !codes || !delta || !q0 || V <= 0 || D <= 0 || groups < 1 || !qo_valid_bits(bits) || D % groups != 0)
+    return QO_ERR_INVALID;
+  const int64_t C = D / groups;  // columns per group
+  const int L = (1 << bits) - 1;
+  int status = QO_OK;
+  for (int64_t g = 0; g < groups; ++g) {
+    float lo = std::numeric_limits<float>::infinity();
+    float hi = -std::numeric_limits<float>::infinity();
+    bool finite = true;
+    for (int64_t v = 0; v < V; ++v)
+      for (int64_t d = g * C; d < (g + 1) * C; ++d) {
+        const float x = e[v * D + d];
+        if (!std::isfinite(x)) finite = false;
+        if (x < lo) lo = x;
+        if (x > hi) hi = x;
+      }
+    if (!finite) {
+      status = QO_ERR_NONFINITE;
+      delta[g] = 1.0f;
+      q0[g] = 0.0f;
+      for (int64_t v = 0; v < V; ++v)
+        for (int64_t d = g * C; d < (g + 1) * C; ++d) codes[v * D + d] = 0;
+      continue;
+    }
+    float dl = (hi - lo) / (float)L;
+    float inv = 1.0f / dl;
+    if (!(dl > 0.0f) || !std::isfinite(inv)) {  // constant group
+      dl = 1.0f;
+      inv = 1.0f;
+      hi = lo;
+    }
+    delta[g] = dl;
+    q0[g] = lo;
+    for (int64_t v = 0; v < V; ++v)
+      for (int64_t d = g * C; d < (g + 1) * C; ++d) {
+        float x = e[v * D + d];
+        x = x < lo ? lo : x;
+        x = x > hi ? hi : x;
+        const float t = (x - lo) * inv;
+        int u = (int)std::nearbyintf(t);
+        u = u < 0 ? 0 : (u > L ? L : u);
+        codes[v * D + d] = (uint8_t)u;
+      }
+  }
+  return status;
+}
+
+// Dequantizing lookup: out[t][d] (+)= Q(E)[ids[t]][d] = Delta_g * code + q0_g, g = d / (D / G).
+// With `accumulate` the value is added to what out already holds (one fp32 addition), which is how
+// the word and the position embedding of a token are summed.  ids must lie in [0, V).
+int qo_embedding_lookup(const int32_t* ids, int64_t T, const uint8_t* codes, int64_t V, int64_t D, int groups,
+                        const float* delta, const float* q0, int accumulate, float* out) {
+  const int64_t C = D / groups;
+  for (int64_t t = 0; t < T; ++t) {
+    if (ids[t] < 0 || ids[t] >= V) return QO_ERR_INVALID;
+    for (int64_t d = 0; d < D; ++d) {
+      const int64_t g = d / C;
+      const float q = std::fmaf(delta[g], (float)codes[(int64_t)ids[t] * D + d], q0[g]);
+      out[t * D + d] = accumulate ? out[t * D + d] + q : q;
+    }
+  }
+  return QO_OK;
+}
+
 }  // extern "C"
