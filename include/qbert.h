@@ -273,6 +273,35 @@ qb_status qb_ste_backward(const float* grad_wq, const float* w, int64_t N, int64
                           const float* range_lo, const float* range_hi, float* grad_w, void* cuda_stream);
 
 /*
+ * Group-wise quantized embedding tables (Section 5.1: embedding quantized separately from the
+ * encoder, word and position embedding at their own precisions; appendix on mixed-precision
+ * embedding: the embedding dimensions are bucketed into 128 groups, 4-bit word and 8-bit position
+ * embedding).  The table is kept in lookup order, E[v][d] with one row per vocabulary entry or
+ * position, so a group is a block of D / G consecutive COLUMNS over all V rows; per group the
+ * quantizer is the one of qb_quantize_pack_weights (exact [min, max] of the group, Appendix A).
+ * Row v of `packed` is the dense little-endian bit stream of its D codes, D*k/32 words.
+ *   table    dev fp32 [V][D], 16-byte aligned                     (read)
+ *   packed   dev uint32 [V][D*bits/32], 16-byte aligned           (written)
+ *   delta,q0 dev fp32 [G]                                         (written)
+ * D must be a multiple of 128, at most 4096, and divisible by G.  The workspace must hold
+ * qb_workspace_bytes(0, 0, 0, 0, D) bytes (8 per column).  Two kernels: per-column min/max into the
+ * workspace, then round/clamp/pack.
+ *
+ * qb_embedding_lookup gathers and dequantizes: out[t][d] = Delta_g * code[ids[t]][d] + q0_g (one fused
+ * multiply-add), g = d / (D / G); with accumulate != 0 that value is added to what `out` holds (one
+ * fp32 addition), which sums the word and the position embedding of a token in two calls.
+ *   ids      dev int32 [T], each in [0, V)                        (read)
+ *   out      dev fp32 [T][D], 16-byte aligned                     (written, or read and written)
+ * An id outside [0, V) writes zeros for that token and records QB_ERR_INVALID in the status word of `ws`.
+ */
+qb_status qb_quantize_embedding(const float* table, int64_t V, int64_t D, int bits, int groups,
+                                uint32_t* packed, float* delta, float* q0, void* ws, size_t ws_bytes,
+                                void* cuda_stream);
+qb_status qb_embedding_lookup(const int32_t* ids, int64_t T, const uint32_t* packed, const float* delta,
+                              const float* q0, int64_t V, int64_t D, int bits, int groups, int accumulate,
+                              float* out, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
  * Diagnostic: the rate the tensor cores sustain for the GEMM's own instruction (tcgen05.mma kind::i8,
  * s8 x s8 -> s32, 128 x `tokens` x 32) with both operands resident in shared memory, no global
  * traffic, four K blocks in flight, one CTA per SM on the default stream.  (No counterpart in the

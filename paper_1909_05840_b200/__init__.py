@@ -31,7 +31,7 @@ EXPORTS = (
     "qb_workspace_init", "qb_read_status", "qb_quantize_act", "qb_quantize_pack_weights", "qb_gemm",
     "qb_layer_linears", "qb_quantize_pack_weights_noalloc", "qb_probe_i8_mma", "qb_quantize_act_batch",
     "qb_quantize_pack_weights_batch", "qb_gemm_bf16", "qb_layer_linears_bf16",
-    "qb_fake_quantize_weights", "qb_ste_backward",
+    "qb_fake_quantize_weights", "qb_ste_backward", "qb_quantize_embedding", "qb_embedding_lookup",
 )
 NOALLOC_MAX_GROUPS = 4096
 
@@ -112,6 +112,11 @@ def lib() -> ctypes.CDLL:
     L.qb_fake_quantize_weights.restype = i32
     L.qb_ste_backward.argtypes = [vp, vp, i64, i64, ctypes.c_int, vp, vp, vp, vp]
     L.qb_ste_backward.restype = i32
+    L.qb_quantize_embedding.argtypes = [vp, i64, i64, ctypes.c_int, ctypes.c_int, vp, vp, vp, vp, sz, vp]
+    L.qb_quantize_embedding.restype = i32
+    L.qb_embedding_lookup.argtypes = [vp, i64, vp, vp, vp, i64, i64, ctypes.c_int, ctypes.c_int, ctypes.c_int, vp, vp,
+                                      sz, vp]
+    L.qb_embedding_lookup.restype = i32
     L.qb_gemm_bf16.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, ctypes.c_int, ctypes.c_int, vp, vp, sz, vp]
     L.qb_gemm_bf16.restype = i32
     L.qb_layer_linears_bf16.argtypes = [ctypes.POINTER(LinearDescC), i32, vp, sz, vp]
@@ -214,6 +219,36 @@ def ste_backward(grad_wq: torch.Tensor, w: torch.Tensor, groups: int, range_lo: 
     _check(lib().qb_ste_backward(grad_wq.data_ptr(), w.data_ptr(), N, K, groups, _ptr(range_lo), _ptr(range_hi),
                                  grad_w.data_ptr(), _stream()), "qb_ste_backward")
     return grad_w
+
+
+def quantize_embedding(table: torch.Tensor, bits: int, groups: int, ws: torch.Tensor,
+                       packed: Optional[torch.Tensor] = None):
+    """``qb_quantize_embedding``: fp32 [V,D] -> (int32-viewed packed rows [V, D*bits/32], delta [G], q0 [G])."""
+    assert table.is_cuda and table.dtype == torch.float32 and table.dim() == 2 and table.is_contiguous()
+    V, D = table.shape
+    if packed is None:
+        packed = torch.empty((V, D * bits // 32), dtype=torch.int32, device=table.device)
+    delta = torch.empty(groups, dtype=torch.float32, device=table.device)
+    q0 = torch.empty(groups, dtype=torch.float32, device=table.device)
+    _check(lib().qb_quantize_embedding(table.data_ptr(), V, D, bits, groups, packed.data_ptr(), delta.data_ptr(),
+                                       q0.data_ptr(), ws.data_ptr(), ws.numel(), _stream()), "qb_quantize_embedding")
+    return packed, delta, q0
+
+
+def embedding_lookup(ids: torch.Tensor, packed: torch.Tensor, delta: torch.Tensor, q0: torch.Tensor, D: int,
+                     bits: int, groups: int, ws: torch.Tensor, out: Optional[torch.Tensor] = None,
+                     accumulate: bool = False) -> torch.Tensor:
+    """``qb_embedding_lookup``: int32 ids [T] -> fp32 [T,D]; with ``accumulate`` the rows are added to ``out``."""
+    assert ids.is_cuda and ids.dtype == torch.int32 and ids.is_contiguous()
+    T = ids.numel()
+    V = packed.shape[0]
+    if out is None:
+        assert not accumulate
+        out = torch.empty((T, D), dtype=torch.float32, device=ids.device)
+    _check(lib().qb_embedding_lookup(ids.data_ptr(), T, packed.data_ptr(), delta.data_ptr(), q0.data_ptr(), V, D, bits,
+                                     groups, 1 if accumulate else 0, out.data_ptr(), ws.data_ptr(), ws.numel(),
+                                     _stream()), "qb_embedding_lookup")
+    return out
 
 
 def make_act_desc_array(items):

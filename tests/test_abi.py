@@ -88,6 +88,13 @@ def test_argument_errors_are_returned_before_any_launch(lib):
     assert lib.qb_ste_backward(A, A, 12, 128, 5, None, None, A, None) == qb.QB_ERR_INVALID
     assert lib.qb_ste_backward(A, A, 12, 128, 3, A, None, A, None) == qb.QB_ERR_INVALID
     assert lib.qb_ste_backward(A, A + 4, 12, 128, 3, None, None, A, None) == qb.QB_ERR_ALIGN
+    # embedding tables
+    assert lib.qb_quantize_embedding(A, 100, 768, 4, 100, A, A, A, A, qb.workspace_bytes(groups=768), None) == qb.QB_ERR_INVALID
+    assert lib.qb_quantize_embedding(A, 100, 800, 4, 100, A, A, A, A, qb.workspace_bytes(groups=800), None) == qb.QB_ERR_ALIGN
+    assert lib.qb_quantize_embedding(A, 100, 768, 4, 128, A, A, A, A, 256, None) == qb.QB_ERR_WORKSPACE
+    assert lib.qb_quantize_embedding(A, 100, 8192, 4, 128, A, A, A, A, ws_bytes, None) == qb.QB_ERR_INVALID
+    assert lib.qb_embedding_lookup(None, 4, A, A, A, 100, 768, 4, 128, 0, A, A, ws_bytes, None) == qb.QB_ERR_INVALID
+    assert lib.qb_embedding_lookup(A, 4, A, A, A, 100, 768, 4, 128, 0, A + 4, A, ws_bytes, None) == qb.QB_ERR_ALIGN
     # stack: every descriptor is validated before the first launch
     good = qb.LinearDescC(A, A, A, A, A, A, None, 8, 12, 128, 4, 3, A)
     bad = qb.LinearDescC(A, A, A, A, A, A, None, 8, 12, 128, 7, 3, A)
