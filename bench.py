@@ -570,6 +570,37 @@ def run_quantizer_sweep(args):
                              "bytes": "12 B per weight (gradient and weight read, gradient written)"}}
         launches += 3 * (3 + steps)
         del w, wq, grad, gout
+    # embedding tables: the BERT-base word table (30522 x 768) at 4 bits and the position table (512 x 768) at
+    # 8 bits, 128 column groups each; lookup of 64 x 384 tokens (word, then position accumulated)
+    emb = {}
+    V, D, G = 30522, 768, 128
+    rng = np.random.default_rng(synth.seed_for(4, 2))
+    tab = torch.from_numpy((rng.standard_normal((V, D)) * 0.02).astype(np.float32)).to(dev)
+    ptab = torch.from_numpy((rng.standard_normal((512, D)) * 0.02).astype(np.float32)).to(dev)
+    wse = qb.workspace(groups=4096, device=dev)
+    pk = torch.empty((V, D * 4 // 32), dtype=torch.int32, device=dev)
+    ms_q = timed(lambda: qb.quantize_embedding(tab, 4, G, wse, packed=pk))
+    pk, dl, z0 = qb.quantize_embedding(tab, 4, G, wse, packed=pk)
+    ppk, pdl, pz0 = qb.quantize_embedding(ptab, 8, G, wse)
+    T = 64 * 384
+    ids = torch.from_numpy(rng.integers(0, V, T).astype(np.int32)).to(dev)
+    pos = torch.arange(384, dtype=torch.int32, device=dev).repeat(64)
+    outb = torch.empty((T, D), dtype=torch.float32, device=dev)
+
+    def look():
+        qb.embedding_lookup(ids, pk, dl, z0, D, 4, G, wse, out=outb)
+        qb.embedding_lookup(pos, ppk, pdl, pz0, D, 8, G, wse, out=outb, accumulate=True)
+
+    ms_l = timed(look)
+    q_bytes = V * D * (8.0 + 0.5)       # two reads of the table (range pass, pack pass) + 4-bit codes written
+    l_bytes = T * D * (0.5 + 4.0) + T * D * (1.0 + 8.0)  # word: codes read, fp32 written; position: codes read, fp32 read and written
+    emb["quantize_embedding_word_k4_g128"] = {"ms": ms_q, "GBps": q_bytes / (ms_q * 1e-3) / 1e9,
+                                              "frac_hbm": q_bytes / (ms_q * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                              "bytes": "8.5 B per element (the 94 MB table is read by both passes)"}
+    emb["lookup_word_k4_plus_position_k8"] = {"ms": ms_l, "tokens": T, "GBps": l_bytes / (ms_l * 1e-3) / 1e9,
+                                              "frac_hbm": l_bytes / (ms_l * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                              "bytes": "13.5 B per output element over the two calls"}
+    launches += 4 * (3 + steps)
     best = max(table.values(), key=lambda r: r["frac_hbm"])
     line = {
         "metric": METRIC, "value": act_gbs, "unit": "GB/s", "n_gpus": 1, "steps": steps, "warmup": 3,
@@ -589,6 +620,7 @@ def run_quantizer_sweep(args):
         "quantize_pack_weights": table,
         "quantize_pack_weights_best_frac_hbm": best["frac_hbm"],
         "fine_tuning": fq,
+        "embedding": emb,
     }
     print(json.dumps(line))
 

@@ -22,17 +22,22 @@ constexpr int kEmbMaxD = 4096;  // blockDim = D/4 <= 1024
 
 __device__ __forceinline__ bool finite_f(float x) { return fabsf(x) <= 3.402823466e38f; }
 
-__global__ void emb_range_kernel(const float4* __restrict__ e, int64_t V, int d4, uint32_t* __restrict__ col_hi,
-                                 uint32_t* __restrict__ col_lo_inv, void* ws) {
-  const int q = threadIdx.x;
+// blockDim = (D/4) * slots: thread (slot, q) owns columns 4q..4q+3 of the rows slot, slot + slots, ... of the
+// block's share; the slots of a block are merged in shared memory, so that few blocks (two per SM) with
+// many loads in flight each take the place of many blocks that would queue on the same 2 D atomics.
+__global__ void emb_range_kernel(const float4* __restrict__ e, int64_t V, int d4, int slots,
+                                 uint32_t* __restrict__ col_hi, uint32_t* __restrict__ col_lo_inv, void* ws) {
+  extern __shared__ uint32_t emb_smem[];  // [slots][2][4 * d4] encoded maxima / inverted minima
+  const int q = threadIdx.x % d4, slot = threadIdx.x / d4;
   const float kInf = __int_as_float(0x7f800000);
   float lo[4] = {kInf, kInf, kInf, kInf}, hi[4] = {-kInf, -kInf, -kInf, -kInf};
   bool bad = false;
-  int64_t r = blockIdx.x;
-  for (; r + 3 * (int64_t)gridDim.x < V; r += 4 * (int64_t)gridDim.x) {  // four rows in flight
+  const int64_t step = (int64_t)gridDim.x * slots;
+  int64_t r = (int64_t)blockIdx.x * slots + slot;
+  for (; r + 3 * step < V; r += 4 * step) {  // four rows in flight per thread
     float4 v[4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) v[j] = __ldg(e + (r + j * (int64_t)gridDim.x) * d4 + q);
+    for (int j = 0; j < 4; ++j) v[j] = __ldg(e + (r + j * step) * d4 + q);
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const float x[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
@@ -44,7 +49,7 @@ __global__ void emb_range_kernel(const float4* __restrict__ e, int64_t V, int d4
       }
     }
   }
-  for (; r < V; r += gridDim.x) {
+  for (; r < V; r += step) {
     const float4 v = __ldg(e + r * d4 + q);
     const float x[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
@@ -55,11 +60,25 @@ __global__ void emb_range_kernel(const float4* __restrict__ e, int64_t V, int d4
     }
   }
   if (bad) report_status(ws, QB_ERR_NONFINITE);
-  if ((int64_t)blockIdx.x < V) {
+  const int D = 4 * d4;
+  uint32_t* mine = emb_smem + (size_t)slot * 2 * D;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {  // a thread that saw no row contributes the neutral encodings of -inf / +inf
+    mine[4 * q + i] = float_to_ordered(hi[i]);
+    mine[D + 4 * q + i] = ~float_to_ordered(lo[i]);
+  }
+  __syncthreads();
+  if (slot == 0) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      atomicMax(col_hi + 4 * q + i, float_to_ordered(hi[i]));
-      atomicMax(col_lo_inv + 4 * q + i, ~float_to_ordered(lo[i]));
+      uint32_t eh = 0, el = 0;
+      for (int s2 = 0; s2 < slots; ++s2) {
+        eh = max(eh, emb_smem[(size_t)s2 * 2 * D + 4 * q + i]);
+        el = max(el, emb_smem[(size_t)s2 * 2 * D + D + 4 * q + i]);
+      }
+      // the slots in the workspace only ever grow: skip the atomic when it cannot change anything
+      if (eh > __ldcg(col_hi + 4 * q + i)) atomicMax(col_hi + 4 * q + i, eh);
+      if (el > __ldcg(col_lo_inv + 4 * q + i)) atomicMax(col_lo_inv + 4 * q + i, el);
     }
   }
 }
@@ -117,8 +136,7 @@ __global__ void emb_pack_kernel(const float4* __restrict__ e, int64_t V, int d4,
   }
   const int first_src = (32 * lane) / F;  // lanes whose fields overlap output word `lane` of the unit
   const int64_t words_per_row = (int64_t)d4 * 4 * BITS / 32;
-  for (int64_t r = blockIdx.x; r < V; r += gridDim.x) {
-    const float4 v = __ldg(e + r * d4 + q);
+  auto pack_row = [&](int64_t r, const float4 v) {
     const float x[4] = {v.x, v.y, v.z, v.w};
     uint32_t field = 0;
 #pragma unroll
@@ -142,7 +160,17 @@ __global__ void emb_pack_kernel(const float4* __restrict__ e, int64_t V, int d4,
       }
     }
     if (lane < WORDS) packed[r * words_per_row + unit * WORDS + lane] = word;
+  };
+  int64_t r = blockIdx.x;
+  const int64_t step = gridDim.x;
+  for (; r + 3 * step < V; r += 4 * step) {  // four rows in flight
+    float4 v[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) v[j] = __ldg(e + (r + j * step) * d4 + q);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) pack_row(r + j * step, v[j]);
   }
+  for (; r < V; r += step) pack_row(r, __ldg(e + r * d4 + q));
 }
 
 template <int BITS>
@@ -239,8 +267,16 @@ extern "C" qb_status qb_quantize_embedding(const float* table, int64_t V, int64_
   int64_t blocks = (int64_t)sms * per_sm;
   if (blocks > V) blocks = V;
   const float4* e4 = reinterpret_cast<const float4*>(table);
-  qb::emb_range_kernel<<<(unsigned)blocks, threads, 0, stream>>>(e4, V, threads, col_hi, col_lo, ws);
-  QB_CUDA_TRY(cudaGetLastError());
+  {
+    int slots = 1024 / threads;  // rows a block reads side by side
+    if (slots > 4) slots = 4;
+    int64_t rblocks = (int64_t)sms * 2;
+    if (rblocks * slots > V) rblocks = (V + slots - 1) / slots;
+    const size_t smem = (size_t)slots * 2 * (size_t)D * sizeof(uint32_t);  // <= 32 KB... 4 x 2 x 4096 x 4 = 128 KB at most
+    QB_CUDA_TRY(cudaFuncSetAttribute(qb::emb_range_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 131072));
+    qb::emb_range_kernel<<<(unsigned)rblocks, threads * slots, smem, stream>>>(e4, V, threads, slots, col_hi, col_lo, ws);
+    QB_CUDA_TRY(cudaGetLastError());
+  }
   const int cpg = (int)(D / groups);
   switch (bits) {
     case 2: qb::emb_pack_kernel<2><<<(unsigned)blocks, threads, 0, stream>>>(e4, V, threads, cpg, col_hi, col_lo, packed, delta, q0); break;
