@@ -61,6 +61,10 @@ def _lib(omp: bool = False) -> ctypes.CDLL:
         lib.qo_quantize_embedding.restype = i32
         lib.qo_embedding_lookup.argtypes = [vp, i64, vp, i64, i64, i32, vp, vp, i32, vp]
         lib.qo_embedding_lookup.restype = i32
+        lib.qo_requantize_i8.argtypes = [vp, i64, f32, vp]
+        lib.qo_requantize_i8.restype = i32
+        lib.qo_rowsum_i8.argtypes = [vp, i64, i64, vp]
+        lib.qo_rowsum_i8.restype = None
         lib.qo_ste_backward.argtypes = [vp, vp, i64, i64, i32, vp, vp, vp]
         lib.qo_ste_backward.restype = None
         lib.qo_round_bf16.argtypes = [vp, i64, vp]
@@ -255,4 +259,21 @@ def embedding_lookup(ids, codes, groups: int, delta, q0, out=None) -> np.ndarray
     st = _lib().qo_embedding_lookup(_p(ids), ids.size, _p(codes), V, D, groups, _p(_c(delta, np.float32)),
                                     _p(_c(q0, np.float32)), int(acc), _p(out))
     assert st == OK, "id out of range"
+    return out
+
+
+def requantize_i8(y, s_out: float) -> np.ndarray:
+    """fp32 -> int8 codes on the grid of step ``s_out``: clamp(round_half_even(y / s_out), -127, 127)."""
+    y = _c(np.asarray(y), np.float32)
+    out = np.empty(y.shape, dtype=np.int8)
+    st = _lib().qo_requantize_i8(_p(y), y.size, ctypes.c_float(s_out), _p(out))
+    assert st == OK, "s_out must be finite and positive"
+    return out
+
+
+def rowsum_i8(xq) -> np.ndarray:
+    xq = _c(xq, np.int8)
+    M, K = xq.shape
+    out = np.empty(M, dtype=np.int32)
+    _lib().qo_rowsum_i8(_p(xq), M, K, _p(out))
     return out

@@ -403,4 +403,30 @@ int qo_embedding_lookup(const int32_t* ids, int64_t T, const uint8_t* codes, int
   return QO_OK;
 }
 
+// Re-quantized output: the fp32 result of a linear narrowed back to the 8-bit activation format that
+// the next linear consumes (Table 1 caption: 8-bit activations throughout), with a scale s_out that the
+// caller supplies (a static, calibrated activation scale).  It is qo_quantize_act's grid with a given
+// step instead of the tensor's own maximum: code = clamp(round_half_even(y * (1 / s_out)), -127, 127);
+// values beyond 127 * s_out saturate.  s_out must be finite and positive.
+int qo_requantize_i8(const float* y, int64_t n, float s_out, int8_t* out) {
+  if (!(s_out > 0.0f) || !std::isfinite(s_out)) return QO_ERR_INVALID;
+  const float inv = 1.0f / s_out;  // one IEEE division
+  for (int64_t i = 0; i < n; ++i) {
+    const float t = y[i] * inv;
+    int c = (int)std::nearbyintf(t < -128.0f ? -128.0f : (t > 128.0f ? 128.0f : t));
+    c = c < -127 ? -127 : (c > 127 ? 127 : c);
+    out[i] = (int8_t)c;
+  }
+  return QO_OK;
+}
+
+// Row sums of int8 codes (the rank-1 offset term of the next linear's epilogue needs them).
+void qo_rowsum_i8(const int8_t* xq, int64_t M, int64_t K, int32_t* rowsum) {
+  for (int64_t m = 0; m < M; ++m) {
+    int32_t s = 0;
+    for (int64_t k = 0; k < K; ++k) s += xq[m * K + k];
+    rowsum[m] = s;
+  }
+}
+
 }  // extern "C"
