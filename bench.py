@@ -601,6 +601,32 @@ def run_quantizer_sweep(args):
                                               "frac_hbm": l_bytes / (ms_l * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                               "bytes": "13.5 B per output element over the two calls"}
     launches += 4 * (3 + steps)
+    # output forms of one GEMM (the QKV projection of config 1: M=4096, N=2304, K=768, 3 bits): fp32, bfloat16,
+    # int8 re-quantized (+ the row sums the next linear needs)
+    outs = {}
+    Mg, Ng, Kg, kb, Gg = 4096, 2304, 768, 3, 384
+    xg = torch.from_numpy(synth.activations(Mg, Kg, synth.seed_for(1, 0, 0))).to(dev)
+    wg = torch.from_numpy(synth.weights(Ng, Kg, synth.seed_for(1, 0, 0))).to(dev)
+    bg = torch.from_numpy(synth.bias(Ng, synth.seed_for(1, 0, 0))).to(dev)
+    wsg = qb.workspace(groups=4096, device=dev)
+    xqg, scg, rsg = qb.quantize_act(xg, wsg)
+    pkg, dlg, zg = qb.quantize_pack_weights(wg, kb, Gg, wsg)
+    y32 = torch.empty((Mg, Ng), dtype=torch.float32, device=dev)
+    y16 = torch.empty((Mg, Ng), dtype=torch.bfloat16, device=dev)
+    y8 = torch.empty((Mg, Ng), dtype=torch.int8, device=dev)
+    rs8 = torch.empty(Mg, dtype=torch.int32, device=dev)
+    s_out = (y32.new_tensor([1.0]))
+    qb.gemm(xqg, scg, rsg, pkg, dlg, zg, bg, Ng, kb, Gg, wsg, y=y32)
+    s_out = (y32.abs().max() / 127.0).reshape(1).contiguous()
+    outs["fp32"] = {"ms": timed(lambda: qb.gemm(xqg, scg, rsg, pkg, dlg, zg, bg, Ng, kb, Gg, wsg, y=y32))}
+    outs["bf16"] = {"ms": timed(lambda: qb.gemm_bf16(xqg, scg, rsg, pkg, dlg, zg, bg, Ng, kb, Gg, wsg, y=y16))}
+    outs["int8"] = {"ms": timed(lambda: qb.gemm_i8(xqg, scg, rsg, pkg, dlg, zg, bg, Ng, kb, Gg, s_out, wsg, yq=y8))}
+    outs["rowsum_i8"] = {"ms": timed(lambda: qb.rowsum_i8(y8, rs8))}
+    for name, ob in (("fp32", 4.0), ("bf16", 2.0), ("int8", 1.0)):
+        byts = Mg * Kg + Ng * Kg * kb / 8 + ob * Mg * Ng
+        outs[name].update({"TOPS": 2.0 * Mg * Ng * Kg / (outs[name]["ms"] * 1e-3) / 1e12,
+                           "GBps": byts / (outs[name]["ms"] * 1e-3) / 1e9})
+    launches += 4 * (3 + steps)
     best = max(table.values(), key=lambda r: r["frac_hbm"])
     line = {
         "metric": METRIC, "value": act_gbs, "unit": "GB/s", "n_gpus": 1, "steps": steps, "warmup": 3,
@@ -621,6 +647,7 @@ def run_quantizer_sweep(args):
         "quantize_pack_weights_best_frac_hbm": best["frac_hbm"],
         "fine_tuning": fq,
         "embedding": emb,
+        "gemm_output_forms_qkv_config1": outs,
     }
     print(json.dumps(line))
 

@@ -245,6 +245,25 @@ qb_status qb_layer_linears_bf16(const qb_linear_desc* descs /*host*/, int32_t co
                                 size_t ws_bytes, void* cuda_stream);
 
 /*
+ * Re-quantized output: the result of a linear written directly in the 8-bit activation format that the
+ * next linear reads (Table 1 caption: 8-bit activations throughout), so that no fp32 tensor and no
+ * separate activation-quantizer pass lie between two linears.  The output grid has a step the caller
+ * supplies (a static, calibrated scale; the dynamic per-tensor maximum of qb_quantize_act cannot be
+ * known before the product is finished):
+ *     yq[m][n] = clamp(round_half_even(y[m][n] * (1 / *out_scale)), -127, 127),
+ * y the fp32 value qb_gemm writes for the same arguments.  Values beyond 127 * out_scale saturate.
+ *   out_scale dev fp32 [1], finite and > 0; it is the act_scale of the consuming linear   (read)
+ *   yq        dev int8 [M][N]                                                              (written)
+ * qb_rowsum_i8 gives the row sums the consuming linear also needs: rowsum[m] = sum_k xq[m][k]
+ * (xq dev int8 [M][K], 16-byte aligned, K a multiple of 128; rowsum dev int32 [M]).
+ */
+qb_status qb_gemm_i8(const int8_t* xq, const float* act_scale, const int32_t* rowsum,
+                     const uint32_t* packed, const float* delta, const float* q0, const float* bias,
+                     int64_t M, int64_t N, int64_t K, int bits, int groups, const float* out_scale,
+                     int8_t* yq, void* ws, size_t ws_bytes, void* cuda_stream);
+qb_status qb_rowsum_i8(const int8_t* xq, int64_t M, int64_t K, int32_t* rowsum, void* cuda_stream);
+
+/*
  * Quantization-aware fine-tuning (Section 3.1: gradients pass through Q by the straight-through
  * estimator; Appendix A: forward and backward of the quantization process).
  *

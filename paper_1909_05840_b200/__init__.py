@@ -32,6 +32,7 @@ EXPORTS = (
     "qb_layer_linears", "qb_quantize_pack_weights_noalloc", "qb_probe_i8_mma", "qb_quantize_act_batch",
     "qb_quantize_pack_weights_batch", "qb_gemm_bf16", "qb_layer_linears_bf16",
     "qb_fake_quantize_weights", "qb_ste_backward", "qb_quantize_embedding", "qb_embedding_lookup",
+    "qb_gemm_i8", "qb_rowsum_i8",
 )
 NOALLOC_MAX_GROUPS = 4096
 
@@ -117,6 +118,10 @@ def lib() -> ctypes.CDLL:
     L.qb_embedding_lookup.argtypes = [vp, i64, vp, vp, vp, i64, i64, ctypes.c_int, ctypes.c_int, ctypes.c_int, vp, vp,
                                       sz, vp]
     L.qb_embedding_lookup.restype = i32
+    L.qb_gemm_i8.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, ctypes.c_int, ctypes.c_int, vp, vp, vp, sz, vp]
+    L.qb_gemm_i8.restype = i32
+    L.qb_rowsum_i8.argtypes = [vp, i64, i64, vp, vp]
+    L.qb_rowsum_i8.restype = i32
     L.qb_gemm_bf16.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, ctypes.c_int, ctypes.c_int, vp, vp, sz, vp]
     L.qb_gemm_bf16.restype = i32
     L.qb_layer_linears_bf16.argtypes = [ctypes.POINTER(LinearDescC), i32, vp, sz, vp]
@@ -333,6 +338,29 @@ def gemm_bf16(xq: torch.Tensor, act_scale: torch.Tensor, rowsum: torch.Tensor, p
                               delta.data_ptr(), q0.data_ptr(), _ptr(bias), M, N, K, bits, groups, y.data_ptr(),
                               ws.data_ptr(), ws.numel(), _stream()), "qb_gemm_bf16")
     return y
+
+
+def gemm_i8(xq: torch.Tensor, act_scale: torch.Tensor, rowsum: torch.Tensor, packed: torch.Tensor,
+            delta: torch.Tensor, q0: torch.Tensor, bias: Optional[torch.Tensor], N: int, bits: int, groups: int,
+            out_scale: torch.Tensor, ws: torch.Tensor, yq: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """``qb_gemm_i8``: returns int8 codes [M,N] on the grid of step ``out_scale`` (device fp32 [1])."""
+    assert xq.is_cuda and xq.dtype == torch.int8 and xq.is_contiguous()
+    assert out_scale.is_cuda and out_scale.dtype == torch.float32
+    M, K = xq.shape
+    yq = torch.empty((M, N), dtype=torch.int8, device=xq.device) if yq is None else yq
+    _check(lib().qb_gemm_i8(xq.data_ptr(), act_scale.data_ptr(), rowsum.data_ptr(), packed.data_ptr(),
+                            delta.data_ptr(), q0.data_ptr(), _ptr(bias), M, N, K, bits, groups, out_scale.data_ptr(),
+                            yq.data_ptr(), ws.data_ptr(), ws.numel(), _stream()), "qb_gemm_i8")
+    return yq
+
+
+def rowsum_i8(xq: torch.Tensor, rowsum: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """``qb_rowsum_i8``: int32 row sums of int8 codes [M,K]."""
+    assert xq.is_cuda and xq.dtype == torch.int8 and xq.dim() == 2 and xq.is_contiguous()
+    M, K = xq.shape
+    rowsum = torch.empty(M, dtype=torch.int32, device=xq.device) if rowsum is None else rowsum
+    _check(lib().qb_rowsum_i8(xq.data_ptr(), M, K, rowsum.data_ptr(), _stream()), "qb_rowsum_i8")
+    return rowsum
 
 
 @dataclass

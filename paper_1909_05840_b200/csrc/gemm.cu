@@ -63,7 +63,8 @@ struct Problem {
   const float* delta;
   const float* q0;
   const float* bias;
-  void* y;           // fp32 [M][N], or bfloat16 [M][N] in the narrow-output kernels
+  void* y;           // fp32 [M][N], or bfloat16 / int8 [M][N] in the narrow-output kernels
+  const float* out_scale;  // int8 output only: dev [1], step of the output grid
   int32_t* acc_out;
   int32_t M, N, K;
   int32_t rows_per_group;
@@ -258,8 +259,11 @@ struct TileCursor {
   }
 };
 
-// BF16: the epilogue rounds its fp32 result to bfloat16 (round to nearest even) and Y is bfloat16 [M][N].
-template <int BT, int BITS, bool BF16>
+// OUT selects what the epilogue writes: the fp32 result; that result rounded to bfloat16 (round to nearest
+// even), Y bfloat16 [M][N]; or that result re-quantized to the 8-bit activation grid of step *out_scale,
+// clamp(round_half_even(y * (1 / out_scale)), -127, 127), Y int8 [M][N].
+enum { kOutF32 = 0, kOutBf16 = 1, kOutI8 = 2 };
+template <int BT, int BITS, int OUT>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
   using Cfg = GemmCfg<BT>;
@@ -566,6 +570,9 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
       const bool tma_store = pr.tma_store != 0;
       float* const y_ptr = reinterpret_cast<float*>(pr.y);
       uint16_t* const y16_ptr = reinterpret_cast<uint16_t*>(pr.y);
+      int8_t* const y8_ptr = reinterpret_cast<int8_t*>(pr.y);
+      float out_inv = 0.0f;
+      if constexpr (OUT == kOutI8) out_inv = __fdiv_rn(1.0f, __ldg(pr.out_scale));
       int32_t* const acc_ptr = pr.acc_out;
       float alpha = 0.f, beta = 0.f, b = 0.f;
       if (nvalid) {
@@ -631,11 +638,18 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
               if (lane == 0) ptx::tma_store_wait_read1();  // the store before last (same buffer) has read it
               __syncwarp();
             }
-            if constexpr (BF16) {  // rows of 32 bfloat16 (64 bytes): the first half of the fp32 buffer
+            if constexpr (OUT == kOutBf16) {  // rows of 32 bfloat16 (64 bytes): the first half of the fp32 buffer
               uint16_t* buf16 = reinterpret_cast<uint16_t*>(buf);
 #pragma unroll
               for (int j = 0; j < 16; ++j)
                 buf16[(16 * h + j) * 32 + lane] = __bfloat16_as_ushort(__float2bfloat16_rn(yv[j]));
+            } else if constexpr (OUT == kOutI8) {  // rows of 32 codes (32 bytes): the first quarter of the buffer
+              int8_t* buf8 = reinterpret_cast<int8_t*>(buf);
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                const int c = __float2int_rn(__fmul_rn(yv[j], out_inv));
+                buf8[(16 * h + j) * 32 + lane] = (int8_t)min(max(c, -127), 127);
+              }
             } else {
 #pragma unroll
               for (int j = 0; j < 16; ++j) buf[(16 * h + j) * 32 + lane] = yv[j];
@@ -651,6 +665,7 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
         if (!tma_store || acc_ptr != nullptr) {
           float* yrow = y_ptr + (size_t)mc * pN + n;
           uint16_t* yrow16 = y16_ptr + (size_t)mc * pN + n;
+          int8_t* yrow8 = y8_ptr + (size_t)mc * pN + n;
           int32_t* arow = acc_ptr ? acc_ptr + (size_t)mc * pN + n : nullptr;
           const int rows = min(32, pM - mc);  // warp-uniform
 #pragma unroll
@@ -664,8 +679,10 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
               if (nvalid && j < rows) {
                 if (!tma_store) {
                   const float yv = __fmaf_rn(alpha, (float)ac, __fmaf_rn(beta, rs[i], b));
-                  if constexpr (BF16)
+                  if constexpr (OUT == kOutBf16)
                     yrow16[(size_t)j * pN] = __bfloat16_as_ushort(__float2bfloat16_rn(yv));
+                  else if constexpr (OUT == kOutI8)
+                    yrow8[(size_t)j * pN] = (int8_t)min(max(__float2int_rn(__fmul_rn(yv, out_inv)), -127), 127);
                   else
                     yrow[(size_t)j * pN] = yv;
                 }
@@ -739,15 +756,19 @@ static qb_status make_x_tensormap(CUtensorMap* tm, const int8_t* xq, int64_t M, 
 
 // Outputs [M][N] (fp32 or bfloat16), N contiguous; box = 32 neurons x 32 tokens, no swizzle (plain row-major
 // in smem).
-static qb_status make_y_tensormap(CUtensorMap* tm, void* y, int64_t M, int64_t N, bool bf16) {
+static qb_status make_y_tensormap(CUtensorMap* tm, void* y, int64_t M, int64_t N, int out) {
+  const int esize = out == kOutF32 ? 4 : (out == kOutBf16 ? 2 : 1);
+  const CUtensorMapDataType dtype = out == kOutF32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                                   : (out == kOutBf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16
+                                                                      : CU_TENSOR_MAP_DATA_TYPE_UINT8);
   EncodeTiledFn encode = nullptr;
   qb_status st = get_encode_fn(&encode);
   if (st != QB_OK) return st;
   const cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
-  const cuuint64_t strides[1] = {(cuuint64_t)N * (bf16 ? 2 : 4)};
+  const cuuint64_t strides[1] = {(cuuint64_t)N * esize};
   const cuuint32_t box[2] = {32, 32};
   const cuuint32_t elem[2] = {1, 1};
-  CUresult r = encode(tm, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, y, dims, strides,
+  CUresult r = encode(tm, dtype, 2, y, dims, strides,
                       box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE,
                       CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
@@ -758,10 +779,10 @@ static qb_status make_y_tensormap(CUtensorMap* tm, void* y, int64_t M, int64_t N
   return QB_OK;
 }
 
-template <int BT, int BITS, bool BF16>
+template <int BT, int BITS, int OUT>
 static qb_status launch_group_inst(const GroupedParams& gp, int grid, cudaStream_t stream) {
   using Cfg = GemmCfg<BT>;
-  auto kernel = qb_gemm_kernel<BT, BITS, BF16>;
+  auto kernel = qb_gemm_kernel<BT, BITS, OUT>;
   static bool attr_set[64] = {};
   int dev = 0;
   QB_CUDA_TRY(cudaGetDevice(&dev));
@@ -774,13 +795,13 @@ static qb_status launch_group_inst(const GroupedParams& gp, int grid, cudaStream
   return QB_OK;
 }
 
-template <int BT, bool BF16>
+template <int BT, int OUT>
 static qb_status launch_group_bits(int bits, const GroupedParams& gp, int grid, cudaStream_t stream) {
   switch (bits) {
-    case 2: return launch_group_inst<BT, 2, BF16>(gp, grid, stream);
-    case 3: return launch_group_inst<BT, 3, BF16>(gp, grid, stream);
-    case 4: return launch_group_inst<BT, 4, BF16>(gp, grid, stream);
-    case 8: return launch_group_inst<BT, 8, BF16>(gp, grid, stream);
+    case 2: return launch_group_inst<BT, 2, OUT>(gp, grid, stream);
+    case 3: return launch_group_inst<BT, 3, OUT>(gp, grid, stream);
+    case 4: return launch_group_inst<BT, 4, OUT>(gp, grid, stream);
+    case 8: return launch_group_inst<BT, 8, OUT>(gp, grid, stream);
     default: return QB_ERR_INVALID;
   }
 }
@@ -818,7 +839,7 @@ static qb_status validate_gemm(const int8_t* xq, const float* act_scale, const i
 // One launch over descriptors d[idx[0..count)] (count <= kMaxProblems), all with the same bit width, on at
 // most `max_ctas` CTAs.
 static qb_status launch_group(const qb_linear_desc* d, const int* idx, int count, int32_t* acc_out, void* ws,
-                              int max_ctas, cudaStream_t stream, bool bf16) {
+                              int max_ctas, cudaStream_t stream, int out, const float* out_scale = nullptr) {
   const int sm_count = max_ctas;
   const int bits = d[idx[0]].bits;
   const int bt = choose_token_tile(d, idx, count, sm_count);
@@ -832,9 +853,9 @@ static qb_status launch_group(const qb_linear_desc* d, const int* idx, int count
     qb_status st = make_x_tensormap(&gp.tmx[i], q.xq, q.M, q.K, bt);
     if (st != QB_OK) return st;
     // Y rows 16-byte aligned: the epilogue stages tiles in shared memory and stores them with TMA
-    const bool tma_store = (q.N % (bf16 ? 8 : 4) == 0) && aligned16(q.y);
+    const bool tma_store = (q.N % (out == kOutF32 ? 4 : (out == kOutBf16 ? 8 : 16)) == 0) && aligned16(q.y);
     if (tma_store) {
-      st = make_y_tensormap(&gp.tmy[i], q.y, q.M, q.N, bf16);
+      st = make_y_tensormap(&gp.tmy[i], q.y, q.M, q.N, out);
       if (st != QB_OK) return st;
     } else {
       gp.tmy[i] = gp.tmx[i];  // unused by the kernel
@@ -847,6 +868,7 @@ static qb_status launch_group(const qb_linear_desc* d, const int* idx, int count
     p.q0 = q.q0;
     p.bias = q.bias;
     p.y = q.y;
+    p.out_scale = out_scale;
     p.acc_out = acc_out;
     p.M = (int32_t)q.M;
     p.N = (int32_t)q.N;
@@ -896,11 +918,14 @@ static qb_status launch_group(const qb_linear_desc* d, const int* idx, int count
       }
     }
   }
-  if (bf16)
-    return bt == 256 ? launch_group_bits<256, true>(bits, gp, grid, stream)
-                     : launch_group_bits<128, true>(bits, gp, grid, stream);
-  return bt == 256 ? launch_group_bits<256, false>(bits, gp, grid, stream)
-                   : launch_group_bits<128, false>(bits, gp, grid, stream);
+  if (out == kOutBf16)
+    return bt == 256 ? launch_group_bits<256, kOutBf16>(bits, gp, grid, stream)
+                     : launch_group_bits<128, kOutBf16>(bits, gp, grid, stream);
+  if (out == kOutI8)
+    return bt == 256 ? launch_group_bits<256, kOutI8>(bits, gp, grid, stream)
+                     : launch_group_bits<128, kOutI8>(bits, gp, grid, stream);
+  return bt == 256 ? launch_group_bits<256, kOutF32>(bits, gp, grid, stream)
+                   : launch_group_bits<128, kOutF32>(bits, gp, grid, stream);
 }
 
 // Side streams and events for launches of one stack that run side by side (host objects, created once per
@@ -941,6 +966,7 @@ static qb_status side_streams(SideStreams** out) {
 // caller's stream before the call returns.  Large stacks keep one launch after the other on all SMs.
 static qb_status launch_stack(const qb_linear_desc* d, int count, void* ws, int sm_count, cudaStream_t stream,
                               bool bf16) {
+  const int out = bf16 ? kOutBf16 : kOutF32;
   std::vector<int> order(count);
   for (int i = 0; i < count; ++i) order[i] = i;
   std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
@@ -978,7 +1004,7 @@ static qb_status launch_stack(const qb_linear_desc* d, int count, void* ws, int 
                             all_tiles < (int64_t)16 * sm_count;
   if (!side_by_side) {
     for (const Group& g : groups) {
-      qb_status st = launch_group(d, order.data() + g.begin, g.count, nullptr, ws, sm_count, stream, bf16);
+      qb_status st = launch_group(d, order.data() + g.begin, g.count, nullptr, ws, sm_count, stream, out);
       if (st != QB_OK) return st;
     }
     return QB_OK;
@@ -1019,7 +1045,7 @@ static qb_status launch_stack(const qb_linear_desc* d, int count, void* ws, int 
   qb_status first_error = QB_OK;
   for (int g = 0; g < n_groups; ++g) {
     cudaStream_t sg = g == 0 ? stream : side->stream[g - 1];
-    st = launch_group(d, order.data() + groups[g].begin, groups[g].count, nullptr, ws, share[g], sg, bf16);
+    st = launch_group(d, order.data() + groups[g].begin, groups[g].count, nullptr, ws, share[g], sg, out);
     if (st != QB_OK && first_error == QB_OK) first_error = st;
   }
   // always join, also after an error: the caller's stream must not run ahead of the side streams
@@ -1036,7 +1062,7 @@ static qb_status launch_stack(const qb_linear_desc* d, int count, void* ws, int 
 static qb_status gemm_entry(const int8_t* xq, const float* act_scale, const int32_t* rowsum, const uint32_t* packed,
                             const float* delta, const float* q0, const float* bias, int64_t M, int64_t N, int64_t K,
                             int bits, int groups, void* y, int32_t* acc_out, void* ws, size_t ws_bytes,
-                            void* cuda_stream, bool bf16) {
+                            void* cuda_stream, int out, const float* out_scale = nullptr) {
   qb_status st = qb::validate_gemm(xq, act_scale, rowsum, packed, delta, q0, M, N, K, bits, groups, y, ws, ws_bytes);
   if (st != QB_OK) return st;
   int sms = 0;
@@ -1057,7 +1083,7 @@ static qb_status gemm_entry(const int8_t* xq, const float* act_scale, const int3
   d.groups = groups;
   d.y = static_cast<float*>(y);
   const int idx = 0;
-  return qb::launch_group(&d, &idx, 1, acc_out, ws, sms, (cudaStream_t)cuda_stream, bf16);
+  return qb::launch_group(&d, &idx, 1, acc_out, ws, sms, (cudaStream_t)cuda_stream, out, out_scale);
 }
 
 static qb_status stack_entry(const char* who, const qb_linear_desc* descs, int32_t count, void* ws, size_t ws_bytes,
@@ -1083,7 +1109,7 @@ extern "C" qb_status qb_gemm(const int8_t* xq, const float* act_scale, const int
                              int64_t M, int64_t N, int64_t K, int bits, int groups, float* y, int32_t* acc_out,
                              void* ws, size_t ws_bytes, void* cuda_stream) {
   return gemm_entry(xq, act_scale, rowsum, packed, delta, q0, bias, M, N, K, bits, groups, y, acc_out, ws, ws_bytes,
-                    cuda_stream, false);
+                    cuda_stream, qb::kOutF32);
 }
 
 extern "C" qb_status qb_gemm_bf16(const int8_t* xq, const float* act_scale, const int32_t* rowsum,
@@ -1091,7 +1117,60 @@ extern "C" qb_status qb_gemm_bf16(const int8_t* xq, const float* act_scale, cons
                                   int64_t M, int64_t N, int64_t K, int bits, int groups, uint16_t* y, void* ws,
                                   size_t ws_bytes, void* cuda_stream) {
   return gemm_entry(xq, act_scale, rowsum, packed, delta, q0, bias, M, N, K, bits, groups, y, nullptr, ws, ws_bytes,
-                    cuda_stream, true);
+                    cuda_stream, qb::kOutBf16);
+}
+
+extern "C" qb_status qb_gemm_i8(const int8_t* xq, const float* act_scale, const int32_t* rowsum,
+                                const uint32_t* packed, const float* delta, const float* q0, const float* bias,
+                                int64_t M, int64_t N, int64_t K, int bits, int groups, const float* out_scale,
+                                int8_t* yq, void* ws, size_t ws_bytes, void* cuda_stream) {
+  if (!out_scale) {
+    qb::set_last_error("qb_gemm_i8: out_scale is null");
+    return QB_ERR_INVALID;
+  }
+  return gemm_entry(xq, act_scale, rowsum, packed, delta, q0, bias, M, N, K, bits, groups, yq, nullptr, ws, ws_bytes,
+                    cuda_stream, qb::kOutI8, out_scale);
+}
+
+namespace qb {
+// one warp per row, 16 codes per lane and load
+__global__ void __launch_bounds__(256) rowsum_i8_kernel(const int4* __restrict__ xq, int64_t M, int64_t k16,
+                                                        int32_t* __restrict__ rowsum) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warps = (int64_t)gridDim.x * 8;
+  for (int64_t m = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5); m < M; m += warps) {
+    int s = 0;
+    for (int64_t c = lane; c < k16; c += 32) {
+      const int4 v = __ldg(xq + m * k16 + c);
+      s = __dp4a(v.x, 0x01010101, s);
+      s = __dp4a(v.y, 0x01010101, s);
+      s = __dp4a(v.z, 0x01010101, s);
+      s = __dp4a(v.w, 0x01010101, s);
+    }
+    s = __reduce_add_sync(0xffffffffu, s);
+    if (lane == 0) rowsum[m] = s;
+  }
+}
+}  // namespace qb
+
+extern "C" qb_status qb_rowsum_i8(const int8_t* xq, int64_t M, int64_t K, int32_t* rowsum, void* cuda_stream) {
+  if (!xq || !rowsum || M <= 0 || K <= 0 || M > QB_MAX_MN || K > QB_MAX_K) {
+    qb::set_last_error("qb_rowsum_i8: null pointer or size out of range (M=%lld K=%lld)", (long long)M, (long long)K);
+    return QB_ERR_INVALID;
+  }
+  if (K % 128 != 0 || !qb::aligned16(xq)) {
+    qb::set_last_error("qb_rowsum_i8: K must be a multiple of 128 and xq 16-byte aligned");
+    return QB_ERR_ALIGN;
+  }
+  int sms = 0;
+  qb_status st = qb::require_sm100(&sms);
+  if (st != QB_OK) return st;
+  int64_t blocks = (M + 7) / 8;
+  if (blocks > (int64_t)sms * 8) blocks = (int64_t)sms * 8;
+  qb::rowsum_i8_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)cuda_stream>>>(reinterpret_cast<const int4*>(xq), M,
+                                                                                K / 16, rowsum);
+  QB_CUDA_TRY(cudaGetLastError());
+  return QB_OK;
 }
 
 extern "C" qb_status qb_layer_linears(const qb_linear_desc* descs, int32_t count, void* ws, size_t ws_bytes,

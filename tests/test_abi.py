@@ -81,6 +81,11 @@ def test_argument_errors_are_returned_before_any_launch(lib):
     assert lib.qb_gemm_bf16(A, A, A, A, A, A, None, 8, 12, 128, 4, 5, A, A, ws_bytes, None) == qb.QB_ERR_INVALID
     assert lib.qb_gemm_bf16(A, A, A, A, A, A, None, 8, 12, 192, 4, 3, A, A, ws_bytes, None) == qb.QB_ERR_ALIGN
     assert lib.qb_gemm_bf16(A, A, A, A, A, A, None, 8, 12, 128, 4, 3, None, A, ws_bytes, None) == qb.QB_ERR_INVALID
+    # re-quantized output and int8 row sums
+    assert lib.qb_gemm_i8(A, A, A, A, A, A, None, 8, 12, 128, 4, 3, None, A, A, ws_bytes, None) == qb.QB_ERR_INVALID
+    assert lib.qb_gemm_i8(A, A, A, A, A, A, None, 8, 12, 192, 4, 3, A, A, A, ws_bytes, None) == qb.QB_ERR_ALIGN
+    assert lib.qb_rowsum_i8(A, 8, 100, A, None) == qb.QB_ERR_ALIGN
+    assert lib.qb_rowsum_i8(None, 8, 128, A, None) == qb.QB_ERR_INVALID
     # fake quantization and its straight-through backward
     assert lib.qb_fake_quantize_weights(A, 12, 128, 5, 1, None, None, A, A, A, A, ws_bytes, None) == qb.QB_ERR_INVALID
     assert lib.qb_fake_quantize_weights(A, 12, 100, 4, 3, None, None, A, A, A, A, ws_bytes, None) == qb.QB_ERR_ALIGN
