@@ -41,7 +41,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 NCU_GEMM_TRAFFIC = {
     # "<sha256 of csrc/gemm.cu + csrc/ptx.cuh>": {<config>: bytes per launch}
     # profiles/qb_gemm_kernel_config1.md, _config2.md, _config3.md (launch averages of the fp32 kernels)
-    "50eb2ced7e8c1609": {"1": 78.1e6, "2": 8.18e6, "3": 4300.2e6},
+    "b8def758e37a61aa": {"1": 78.1e6, "2": 8.18e6, "3": 4299.1e6},
 }
 
 
