@@ -272,8 +272,8 @@ extern "C" qb_status qb_quantize_embedding(const float* table, int64_t V, int64_
     if (slots > 4) slots = 4;
     int64_t rblocks = (int64_t)sms * 2;
     if (rblocks * slots > V) rblocks = (V + slots - 1) / slots;
-    const size_t smem = (size_t)slots * 2 * (size_t)D * sizeof(uint32_t);  // <= 32 KB... 4 x 2 x 4096 x 4 = 128 KB at most
-    QB_CUDA_TRY(cudaFuncSetAttribute(qb::emb_range_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 131072));
+    // slots * D <= 4096 columns (blockDim <= 1024 threads of four columns each): at most 32 KB
+    const size_t smem = (size_t)slots * 2 * (size_t)D * sizeof(uint32_t);
     qb::emb_range_kernel<<<(unsigned)rblocks, threads * slots, smem, stream>>>(e4, V, threads, slots, col_hi, col_lo, ws);
     QB_CUDA_TRY(cudaGetLastError());
   }

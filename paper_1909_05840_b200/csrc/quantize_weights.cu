@@ -754,6 +754,92 @@ weight_fused_kernel(const __grid_constant__ FusedBatch b) {
   }
 }
 
+// ---- register-resident path ---------------------------------------------------------------------------
+// Small groups (up to 72 units = 9,216 weights: one range per output row, or six 768-wide rows) are read
+// from HBM once and never leave the registers: a team of W warps (W = 1, 2 or 4, the same for a launch)
+// loads its group as up to 18 float4 per thread, all in flight at once, reduces the range (warp redux,
+// then the team's named barrier), and packs from the same registers with the unit packer of the two-pass
+// path.  A block holds 4 to 16 teams, so loads of some overlap the packing of others.  With larger
+// teams (the kernel takes up to 16 warps per group) a block has only one or two groups in flight and
+// the load and pack phases no longer overlap: measured slower than the shared-memory ring, which keeps
+// those groups (config 4, 128 groups per matrix: 0.41-0.51 of the copy bandwidth against 0.48-0.54).
+constexpr int kRegUnitsPerThread = 18;
+constexpr int kRegWarps = 16;
+constexpr int kRegThreads = 32 * kRegWarps;
+constexpr int kRegMaxGroupUnits = kRegUnitsPerThread * kRegWarps;  // 288: what the kernel can hold
+constexpr int kRegPathMaxUnits = kRegUnitsPerThread * 4;           // 72: what is sent to it
+
+template <int BITS>
+__global__ void __launch_bounds__(kRegThreads, 1)
+weight_reg_kernel(const __grid_constant__ FusedBatch b) {
+  constexpr int L = (1 << BITS) - 1;
+  constexpr int WORDS = 4 * BITS;
+  __shared__ uint32_t s_hi[2][kRegWarps], s_lo[2][kRegWarps];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int W = b.team_warps;
+  const int team = warp / W, tw = warp - team * W;
+  const int teams_per_block = kRegWarps / W;
+  const int64_t total_teams = (int64_t)gridDim.x * teams_per_block;
+  const int first_src = (32 * lane) / (4 * BITS);
+  const float kInf = __int_as_float(0x7f800000);
+  int it = 0, flip = 0;
+  for (int64_t g = (int64_t)blockIdx.x * teams_per_block + team; g < b.total_groups; g += total_teams) {
+    while (it + 1 < b.count && g >= b.item[it + 1].group_begin) ++it;
+    const WeightItem& m = b.item[it];
+    const int gl = (int)(g - m.group_begin);
+    const int ug = m.rows_per_group * m.units_per_row;
+    const float4* const src = m.w + (int64_t)gl * ug * 32;
+    float4 v[kRegUnitsPerThread];
+#pragma unroll
+    for (int j = 0; j < kRegUnitsPerThread; ++j) {
+      const int u = j * W + tw;  // warp-uniform
+      if (u < ug) v[j] = __ldg(src + (int64_t)u * 32 + lane);
+    }
+    float lo = kInf, hi = -kInf;
+#pragma unroll
+    for (int j = 0; j < kRegUnitsPerThread; ++j) {
+      if (j * W + tw < ug) {
+        lo = min_nan(min_nan(lo, v[j].x), min_nan(v[j].y, min_nan(v[j].z, v[j].w)));
+        hi = max_nan(max_nan(hi, v[j].x), max_nan(v[j].y, max_nan(v[j].z, v[j].w)));
+      }
+    }
+    // NaN anywhere makes hi NaN (encoded above every number); Inf shows as hi = +Inf or lo = -Inf
+    uint32_t e_hi = __reduce_max_sync(0xffffffffu, float_to_ordered(hi));
+    uint32_t e_lo = __reduce_max_sync(0xffffffffu, ~float_to_ordered(lo));
+    if (W > 1) {
+      if (lane == 0) {
+        s_hi[flip][warp] = e_hi;
+        s_lo[flip][warp] = e_lo;
+      }
+      asm volatile("bar.sync %0, %1;" ::"r"(1 + team), "r"(32 * W) : "memory");
+      const uint32_t vh = lane < W ? s_hi[flip][team * W + lane] : 0u;
+      const uint32_t vl = lane < W ? s_lo[flip][team * W + lane] : 0u;
+      e_hi = __reduce_max_sync(0xffffffffu, vh);
+      e_lo = __reduce_max_sync(0xffffffffu, vl);
+      flip ^= 1;  // the other half is free again once every warp of the team has passed the next barrier
+    }
+    const float g_hi = ordered_to_float(e_hi);
+    const float g_lo = ordered_to_float(~e_lo);
+    const bool publish = tw == 0 && lane == 0;
+    if (publish && !(fabsf(g_hi) <= 3.402823466e38f && fabsf(g_lo) <= 3.402823466e38f))
+      report_status(b.ws, QB_ERR_NONFINITE);
+    GroupParams gp;
+    if (m.range_lo != nullptr)
+      gp = finish_group(__ldg(m.range_lo + gl), __ldg(m.range_hi + gl), true, L, gl, m.delta, m.q0, publish, b.ws);
+    else
+      gp = finish_group(g_lo, g_hi, false, L, gl, m.delta, m.q0, publish, b.ws);
+    uint32_t* const out = m.packed + (int64_t)gl * ug * WORDS;
+#pragma unroll
+    for (int j = 0; j < kRegUnitsPerThread; ++j) {
+      const int u = j * W + tw;
+      if (u < ug) {
+        const uint32_t word = pack_unit<BITS>(v[j], gp, lane, first_src);
+        if (lane < WORDS) out[(int64_t)u * WORDS + lane] = word;
+      }
+    }
+  }
+}
+
 struct HostWeight {
   const float* w;
   int64_t N, K;
@@ -845,6 +931,23 @@ static qb_status launch_fused(const HostWeight* m, int count, int bits, void* ws
   // small groups: 4 KB slots and small teams (many groups in flight); large groups: 16 KB slots
   int64_t ug_max = 1;
   for (int i = 0; i < count; ++i) ug_max = std::max(ug_max, group_units(m[i]));
+  if (ug_max <= kRegPathMaxUnits) {  // small groups: teams of at most four warps keep them in registers
+    int W = 1;
+    while ((int64_t)W * kRegUnitsPerThread < ug_max) W *= 2;
+    b.team_warps = W;
+    const int teams_per_block = kRegWarps / W;
+    int64_t blocks = (total_groups + teams_per_block - 1) / teams_per_block;
+    if (blocks > sm_count) blocks = sm_count;
+    switch (bits) {
+      case 2: weight_reg_kernel<2><<<(unsigned)blocks, kRegThreads, 0, stream>>>(b); break;
+      case 3: weight_reg_kernel<3><<<(unsigned)blocks, kRegThreads, 0, stream>>>(b); break;
+      case 4: weight_reg_kernel<4><<<(unsigned)blocks, kRegThreads, 0, stream>>>(b); break;
+      case 8: weight_reg_kernel<8><<<(unsigned)blocks, kRegThreads, 0, stream>>>(b); break;
+      default: return QB_ERR_INVALID;
+    }
+    QB_CUDA_TRY(cudaGetLastError());
+    return QB_OK;
+  }
   b.chunk_units = ug_max <= 64 ? 8 : 32;
   b.n_slots = kRingBytes / (b.chunk_units * 512);
   b.team_warps = ug_max <= 16 ? 1 : (ug_max <= 64 ? 2 : (ug_max <= 160 ? 4 : 8));
