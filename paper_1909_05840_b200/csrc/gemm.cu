@@ -806,13 +806,20 @@ static qb_status launch_group_bits(int bits, const GroupedParams& gp, int grid, 
   }
 }
 
-// Token-tile width for a launch: 256 tokens unless every problem has at most 128.  The 128-wide
-// instruction takes as long as the 256-wide one (measured with qb_probe_i8_mma: 498 vs 512 cycles per
-// K block), so narrow tiles halve the tensor rate and double the weight expansion per token.
+// Token-tile width for a launch: 256 tokens unless every problem has at most 128 or the launch is too
+// small to give every SM a 256-token tile.  The 128-wide instruction takes as long as the 256-wide one
+// (measured with qb_probe_i8_mma: 498 vs 512 cycles per K block), so narrow tiles halve the tensor rate
+// and double the weight expansion per token; they pay only when SMs would otherwise idle.
 static int choose_token_tile(const qb_linear_desc* d, const int* idx, int count, int sm_count) {
-  (void)sm_count;
-  for (int i = 0; i < count; ++i)
-    if (d[idx[i]].M > 128) return 256;
+  bool wide = false;
+  int64_t tiles256 = 0;
+  for (int i = 0; i < count; ++i) {
+    if (d[idx[i]].M > 128) wide = true;
+    tiles256 += ((d[idx[i]].N + kTileN - 1) / kTileN) * ((d[idx[i]].M + 255) / 256);
+  }
+  // a launch that cannot give every SM a 256-token tile uses 128-token tiles: twice the CTAs at work,
+  // half the epilogue per tile
+  if (wide && tiles256 >= sm_count) return 256;
   return 128;
 }
 
