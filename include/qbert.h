@@ -137,7 +137,10 @@ typedef struct {
  * tensor: BERT's matrices are a few MB each, so single launches are bound by launch latency, not by
  * memory bandwidth.  `descs` is a HOST array; every element is validated before anything is launched;
  * each result equals the single call on the same arguments bit for bit.  Each activation tensor keeps
- * its own scale (per-tensor quantization).  Weight matrices of different bit widths may be mixed.
+ * its own scale (per-tensor quantization).  Weight matrices of different bit widths may be mixed;
+ * each bit width gets its own launches, and when these are several small single-read launches (a
+ * mixed-precision stack) they run side by side on streams the library creates once per device
+ * (host objects only), forking from and joining `cuda_stream` inside the call as in qb_layer_linears.
  * Workspace: qb_workspace_bytes(0, 0, 0, 0, G) bytes with G = max(32, sum of `groups` over the batch).
  */
 qb_status qb_quantize_act_batch(const qb_act_desc* descs /*host*/, int32_t count, void* ws, size_t ws_bytes,

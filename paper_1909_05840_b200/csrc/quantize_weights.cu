@@ -977,8 +977,35 @@ static inline int fused_class(int64_t ug) { return ug <= 16 ? 0 : (ug <= 64 ? 1 
 // single-read path when together they have enough groups to occupy the GPU, one launch per size class
 // of groups (a class too small to be worth a launch joins the next larger one); the others take the
 // two-pass path.
-static qb_status launch_weight_batch(const HostWeight* m, int count, int bits, void* ws, int sm_count,
-                                     cudaStream_t stream) {
+// One launch (single-read paths) or pair of launches (two-pass path) of a batch call.
+struct WeightJob {
+  HostWeight m[kMaxWeightBatch];
+  int n;
+  int bits;
+  bool single_read;
+  int64_t bytes;  // fp32 bytes read
+};
+
+static void push_job(std::vector<WeightJob>& jobs, const HostWeight* m, int n, int bits, bool single_read) {
+  WeightJob j;
+  j.n = n;
+  j.bits = bits;
+  j.single_read = single_read;
+  j.bytes = 0;
+  for (int i = 0; i < n; ++i) {
+    j.m[i] = m[i];
+    j.bytes += m[i].N * m[i].K * 4;
+  }
+  jobs.push_back(j);
+}
+
+// `max_ctas` caps the grid of a single-read job (a share of the SMs when jobs run side by side).
+static qb_status run_weight_job(const WeightJob& j, void* ws, int sm_count, int max_ctas, cudaStream_t stream) {
+  if (j.single_read) return launch_fused(j.m, j.n, j.bits, ws, max_ctas, stream);
+  return launch_two_pass(j.m, j.n, j.bits, ws, sm_count, stream);
+}
+
+static void plan_weight_batch(const HostWeight* m, int count, int bits, int sm_count, std::vector<WeightJob>& jobs) {
   constexpr int64_t kClassWorthALaunch = 32ll << 20;  // bytes of fp32 weights
   HostWeight fused[kMaxWeightBatch], rest[kMaxWeightBatch];
   int cls[kMaxWeightBatch];
@@ -1010,15 +1037,107 @@ static qb_status launch_weight_batch(const HostWeight* m, int count, int bits, v
       bool later = false;  // does a larger class still have matrices?
       for (int i = 0; i < nf; ++i) later = later || cls[i] > c;
       if (nb > 0 && (bytes >= kClassWorthALaunch || !later)) {
-        qb_status st = launch_fused(batch, nb, bits, ws, sm_count, stream);
-        if (st != QB_OK) return st;
+        push_job(jobs, batch, nb, bits, true);
         nb = 0;
         bytes = 0;
       }
     }
   }
-  if (nr > 0) return launch_two_pass(rest, nr, bits, ws, sm_count, stream);
+  if (nr > 0) push_job(jobs, rest, nr, bits, false);
+}
+
+static qb_status launch_weight_batch(const HostWeight* m, int count, int bits, void* ws, int sm_count,
+                                     cudaStream_t stream) {
+  std::vector<WeightJob> jobs;
+  plan_weight_batch(m, count, bits, sm_count, jobs);
+  for (const WeightJob& j : jobs) {
+    qb_status st = run_weight_job(j, ws, sm_count, sm_count, stream);
+    if (st != QB_OK) return st;
+  }
   return QB_OK;
+}
+
+// Streams and events for the single-read launches of one batch call that run side by side (host objects,
+// created once per device on first use; no device memory).
+constexpr int kMaxSideJobs = 8;
+struct WeightSideStreams {
+  cudaStream_t stream[kMaxSideJobs - 1];
+  cudaEvent_t done[kMaxSideJobs - 1];
+  cudaEvent_t fork;
+  bool ready;
+};
+static qb_status weight_side_streams(WeightSideStreams** out) {
+  static WeightSideStreams per_dev[64];
+  int dev = 0;
+  QB_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) {
+    set_last_error("device ordinal %d out of range", dev);
+    return QB_ERR_CUDA;
+  }
+  WeightSideStreams& s = per_dev[dev];
+  if (!s.ready) {
+    for (int i = 0; i < kMaxSideJobs - 1; ++i) {
+      QB_CUDA_TRY(cudaStreamCreateWithFlags(&s.stream[i], cudaStreamNonBlocking));
+      QB_CUDA_TRY(cudaEventCreateWithFlags(&s.done[i], cudaEventDisableTiming));
+    }
+    QB_CUDA_TRY(cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming));
+    s.ready = true;
+  }
+  *out = &s;
+  return QB_OK;
+}
+
+// The jobs of a batch call.  Several small single-read jobs (a mixed-precision stack: one or two per bit
+// width, tens of MB each) run side by side on SM shares in proportion to their bytes, so that their
+// start-up and drain overlap; they touch nothing in the workspace but the status word.  Anything else
+// runs one job after the other (the two-pass jobs share the range tables at the head of the workspace).
+static qb_status run_weight_jobs(const std::vector<WeightJob>& jobs, void* ws, int sm_count, cudaStream_t stream) {
+  constexpr int64_t kSmallJob = 160ll << 20;
+  const int n = (int)jobs.size();
+  bool side = n >= 2 && n <= kMaxSideJobs && n * 8 <= sm_count;
+  int64_t total = 0;
+  for (const WeightJob& j : jobs) {
+    side = side && j.single_read && j.bytes <= kSmallJob;
+    total += j.bytes;
+  }
+  if (!side) {
+    for (const WeightJob& j : jobs) {
+      qb_status st = run_weight_job(j, ws, sm_count, sm_count, stream);
+      if (st != QB_OK) return st;
+    }
+    return QB_OK;
+  }
+  std::vector<int> share(n);
+  int used = 0;
+  for (int i = 0; i < n; ++i) {
+    int64_t sh = (int64_t)sm_count * jobs[i].bytes / total;
+    if (sh < 8) sh = 8;
+    share[i] = (int)sh;
+    used += share[i];
+  }
+  while (used > sm_count) {  // the minimum share can overshoot: take from the largest
+    int big = 0;
+    for (int i = 1; i < n; ++i)
+      if (share[i] > share[big]) big = i;
+    --share[big];
+    --used;
+  }
+  for (int i = 0; used < sm_count; i = (i + 1) % n, ++used) ++share[i];
+  WeightSideStreams* sd = nullptr;
+  qb_status st = weight_side_streams(&sd);
+  if (st != QB_OK) return st;
+  QB_CUDA_TRY(cudaEventRecord(sd->fork, stream));
+  for (int i = 1; i < n; ++i) QB_CUDA_TRY(cudaStreamWaitEvent(sd->stream[i - 1], sd->fork, 0));
+  qb_status first_error = QB_OK;
+  for (int i = 0; i < n; ++i) {
+    st = run_weight_job(jobs[i], ws, sm_count, share[i], i == 0 ? stream : sd->stream[i - 1]);
+    if (st != QB_OK && first_error == QB_OK) first_error = st;
+  }
+  for (int i = 1; i < n; ++i) {  // always join, also after an error
+    QB_CUDA_TRY(cudaEventRecord(sd->done[i - 1], sd->stream[i - 1]));
+    QB_CUDA_TRY(cudaStreamWaitEvent(stream, sd->done[i - 1], 0));
+  }
+  return first_error;
 }
 
 // Fake quantization of one matrix: the range kernel of the two-pass path, then weight_fake_kernel.
@@ -1129,6 +1248,7 @@ extern "C" qb_status qb_quantize_pack_weights_batch(const qb_weight_desc* descs,
   std::vector<int> order(count);
   for (int i = 0; i < count; ++i) order[i] = i;
   std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return descs[a].bits < descs[b].bits; });
+  std::vector<qb::WeightJob> jobs;
   int i = 0;
   while (i < count) {
     qb::HostWeight m[qb::kMaxWeightBatch];
@@ -1139,10 +1259,9 @@ extern "C" qb_status qb_quantize_pack_weights_batch(const qb_weight_desc* descs,
       m[n++] = qb::HostWeight{d.w, d.N, d.K, d.groups, d.range_lo, d.range_hi, d.packed, d.delta, d.q0};
       ++i;
     }
-    st = qb::launch_weight_batch(m, n, bits, ws, sms, (cudaStream_t)cuda_stream);
-    if (st != QB_OK) return st;
+    qb::plan_weight_batch(m, n, bits, sms, jobs);
   }
-  return QB_OK;
+  return qb::run_weight_jobs(jobs, ws, sms, (cudaStream_t)cuda_stream);
 }
 
 extern "C" qb_status qb_fake_quantize_weights(const float* w, int64_t N, int64_t K, int bits, int groups,
