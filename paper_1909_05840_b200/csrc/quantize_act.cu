@@ -37,7 +37,29 @@ struct ActBatch {
   void* ws;
   int64_t rows_total;
   int32_t count;
+  float keep_fraction;  // share of the launch's input that L2 is asked to keep between the two passes
 };
+
+// 16-byte load with an L2 eviction-priority policy (createpolicy): the maximum pass asks L2 to keep a
+// fraction of what it reads (the rounding pass reads the same tensors next), the rounding pass marks
+// its reads as the first to go.
+__device__ __forceinline__ float4 ldg_policy(const float4* p, uint64_t policy) {
+  float4 v;
+  asm volatile("ld.global.nc.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+               : "l"(p), "l"(policy));
+  return v;
+}
+__device__ __forceinline__ uint64_t policy_evict_last(float fraction) {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, %1;" : "=l"(pol) : "f"(fraction));
+  return pol;
+}
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
 
 __global__ void __launch_bounds__(kActThreads)
 act_absmax_kernel(const __grid_constant__ ActBatch b) {
@@ -47,12 +69,13 @@ act_absmax_kernel(const __grid_constant__ ActBatch b) {
   const float4* __restrict__ x = reinterpret_cast<const float4*>(t.x);
   const int64_t n4 = t.M * t.K / 4;
   uint32_t m = 0;
+  const uint64_t pol = policy_evict_last(b.keep_fraction);
   const int64_t stride = (int64_t)t.blocks * blockDim.x;
   int64_t i = (int64_t)((int)blockIdx.x - t.block_begin) * blockDim.x + threadIdx.x;
   // four independent 16-byte loads in flight per thread
   for (; i + 3 * stride < n4; i += 4 * stride) {
-    float4 a = __ldg(x + i), bb = __ldg(x + i + stride), c = __ldg(x + i + 2 * stride),
-           d = __ldg(x + i + 3 * stride);
+    float4 a = ldg_policy(x + i, pol), bb = ldg_policy(x + i + stride, pol), c = ldg_policy(x + i + 2 * stride, pol),
+           d = ldg_policy(x + i + 3 * stride, pol);
 #define QB_ABSMAX4(v)                                            \
   m = max(m, __float_as_uint(v.x) & 0x7fffffffu);                \
   m = max(m, __float_as_uint(v.y) & 0x7fffffffu);                \
@@ -61,7 +84,7 @@ act_absmax_kernel(const __grid_constant__ ActBatch b) {
     QB_ABSMAX4(a) QB_ABSMAX4(bb) QB_ABSMAX4(c) QB_ABSMAX4(d)
   }
   for (; i < n4; i += stride) {
-    float4 a = __ldg(x + i);
+    float4 a = ldg_policy(x + i, pol);
     QB_ABSMAX4(a)
   }
 #undef QB_ABSMAX4
@@ -103,6 +126,7 @@ act_quantize_kernel(const __grid_constant__ ActBatch b) {
   int it = 0;
   int cur = -1;
   float inv = 0.0f;
+  const uint64_t pol = policy_evict_first();
   for (int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); row < b.rows_total; row += warps) {
     while (it + 1 < b.count && row >= b.item[it + 1].row_begin) ++it;
     const ActItem& t = b.item[it];
@@ -122,7 +146,7 @@ act_quantize_kernel(const __grid_constant__ ActBatch b) {
     int sum = 0;
 #pragma unroll 4
     for (int64_t c = lane; c < k4; c += 32) {
-      const float4 v = __ldg(src + c);
+      const float4 v = ldg_policy(src + c, pol);
       const int q0 = quant_code(v.x, inv), q1 = quant_code(v.y, inv), q2 = quant_code(v.z, inv),
                 q3 = quant_code(v.w, inv);
       sum += (q0 + q1) + (q2 + q3);
@@ -178,6 +202,11 @@ static qb_status launch_act_batch(const qb_act_desc* d, int count, void* ws, uin
     blocks1 += (int)want;
   }
   b.rows_total = rows;
+  {
+    const double bytes = 16.0 * (double)total4;
+    const double keep = 96.0 * 1048576.0;  // what the 126 MB L2 holds of a stream besides the codes being written
+    b.keep_fraction = bytes <= keep ? 1.0f : (float)(keep / bytes);
+  }
   QB_CUDA_TRY(cudaMemsetAsync(absmax_slots, 0, sizeof(uint32_t) * (size_t)count, stream));
   act_absmax_kernel<<<(unsigned)blocks1, kActThreads, 0, stream>>>(b);
   QB_CUDA_TRY(cudaGetLastError());
