@@ -62,6 +62,34 @@ __device__ __forceinline__ float ordered_to_float(uint32_t e) {
   uint32_t b = (e & 0x80000000u) ? (e & 0x7fffffffu) : ~e;
   return __uint_as_float(b);
 }
+// 16-byte load with an L2 eviction-priority policy (createpolicy).  The two-pass quantizers use it: the
+// first pass asks L2 to keep a fraction of what it reads (the second pass reads the same tensor next),
+// the second pass marks its reads as the first to go.
+__device__ __forceinline__ float4 ldg_policy(const float4* p, uint64_t policy) {
+  float4 v;
+  asm volatile("ld.global.nc.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+               : "l"(p), "l"(policy));
+  return v;
+}
+__device__ __forceinline__ uint64_t policy_evict_last(float fraction) {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, %1;" : "=l"(pol) : "f"(fraction));
+  return pol;
+}
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+
+// Share of a first pass's input that L2 is asked to keep: all of it up to 96 MB (what the 126 MB L2 holds
+// of a stream besides what the second pass writes), else 96 MB worth.
+inline float l2_keep_fraction(double input_bytes) {
+  const double keep = 96.0 * 1048576.0;
+  return input_bytes <= keep ? 1.0f : (float)(keep / input_bytes);
+}
+
 #endif
 
 }  // namespace qb

@@ -25,8 +25,9 @@ __device__ __forceinline__ bool finite_f(float x) { return fabsf(x) <= 3.4028234
 // blockDim = (D/4) * slots: thread (slot, q) owns columns 4q..4q+3 of the rows slot, slot + slots, ... of the
 // block's share; the slots of a block are merged in shared memory, so that few blocks (two per SM) with
 // many loads in flight each take the place of many blocks that would queue on the same 2 D atomics.
-__global__ void emb_range_kernel(const float4* __restrict__ e, int64_t V, int d4, int slots,
+__global__ void emb_range_kernel(const float4* __restrict__ e, int64_t V, int d4, int slots, float keep_fraction,
                                  uint32_t* __restrict__ col_hi, uint32_t* __restrict__ col_lo_inv, void* ws) {
+  const uint64_t pol = policy_evict_last(keep_fraction);
   extern __shared__ uint32_t emb_smem[];  // [slots][2][4 * d4] encoded maxima / inverted minima
   const int q = threadIdx.x % d4, slot = threadIdx.x / d4;
   const float kInf = __int_as_float(0x7f800000);
@@ -37,7 +38,7 @@ __global__ void emb_range_kernel(const float4* __restrict__ e, int64_t V, int d4
   for (; r + 3 * step < V; r += 4 * step) {  // four rows in flight per thread
     float4 v[4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) v[j] = __ldg(e + (r + j * step) * d4 + q);
+    for (int j = 0; j < 4; ++j) v[j] = ldg_policy(e + (r + j * step) * d4 + q, pol);
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const float x[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
@@ -50,7 +51,7 @@ __global__ void emb_range_kernel(const float4* __restrict__ e, int64_t V, int d4
     }
   }
   for (; r < V; r += step) {
-    const float4 v = __ldg(e + r * d4 + q);
+    const float4 v = ldg_policy(e + r * d4 + q, pol);
     const float x[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -124,6 +125,7 @@ __global__ void emb_pack_kernel(const float4* __restrict__ e, int64_t V, int d4,
   constexpr int WORDS = 4 * BITS;  // output words per unit of 128 codes
   constexpr int NSRC = BITS == 8 ? 1 : (BITS == 4 ? 2 : 4);
   const int q = threadIdx.x, lane = threadIdx.x & 31, unit = threadIdx.x >> 5;
+  const uint64_t pol = policy_evict_first();
   ColParams p;
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
@@ -166,11 +168,11 @@ __global__ void emb_pack_kernel(const float4* __restrict__ e, int64_t V, int d4,
   for (; r + 3 * step < V; r += 4 * step) {  // four rows in flight
     float4 v[4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) v[j] = __ldg(e + (r + j * step) * d4 + q);
+    for (int j = 0; j < 4; ++j) v[j] = ldg_policy(e + (r + j * step) * d4 + q, pol);
 #pragma unroll
     for (int j = 0; j < 4; ++j) pack_row(r + j * step, v[j]);
   }
-  for (; r < V; r += step) pack_row(r, __ldg(e + r * d4 + q));
+  for (; r < V; r += step) pack_row(r, ldg_policy(e + r * d4 + q, pol));
 }
 
 template <int BITS>
@@ -274,7 +276,7 @@ extern "C" qb_status qb_quantize_embedding(const float* table, int64_t V, int64_
     if (rblocks * slots > V) rblocks = (V + slots - 1) / slots;
     // slots * D <= 4096 columns (blockDim <= 1024 threads of four columns each): at most 32 KB
     const size_t smem = (size_t)slots * 2 * (size_t)D * sizeof(uint32_t);
-    qb::emb_range_kernel<<<(unsigned)rblocks, threads * slots, smem, stream>>>(e4, V, threads, slots, col_hi, col_lo, ws);
+    qb::emb_range_kernel<<<(unsigned)rblocks, threads * slots, smem, stream>>>(e4, V, threads, slots, qb::l2_keep_fraction(4.0 * (double)V * (double)D), col_hi, col_lo, ws);
     QB_CUDA_TRY(cudaGetLastError());
   }
   const int cpg = (int)(D / groups);

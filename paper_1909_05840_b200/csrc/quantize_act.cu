@@ -40,27 +40,6 @@ struct ActBatch {
   float keep_fraction;  // share of the launch's input that L2 is asked to keep between the two passes
 };
 
-// 16-byte load with an L2 eviction-priority policy (createpolicy): the maximum pass asks L2 to keep a
-// fraction of what it reads (the rounding pass reads the same tensors next), the rounding pass marks
-// its reads as the first to go.
-__device__ __forceinline__ float4 ldg_policy(const float4* p, uint64_t policy) {
-  float4 v;
-  asm volatile("ld.global.nc.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
-               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
-               : "l"(p), "l"(policy));
-  return v;
-}
-__device__ __forceinline__ uint64_t policy_evict_last(float fraction) {
-  uint64_t pol;
-  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, %1;" : "=l"(pol) : "f"(fraction));
-  return pol;
-}
-__device__ __forceinline__ uint64_t policy_evict_first() {
-  uint64_t pol;
-  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
-  return pol;
-}
-
 __global__ void __launch_bounds__(kActThreads)
 act_absmax_kernel(const __grid_constant__ ActBatch b) {
   int it = 0;
@@ -202,11 +181,7 @@ static qb_status launch_act_batch(const qb_act_desc* d, int count, void* ws, uin
     blocks1 += (int)want;
   }
   b.rows_total = rows;
-  {
-    const double bytes = 16.0 * (double)total4;
-    const double keep = 96.0 * 1048576.0;  // what the 126 MB L2 holds of a stream besides the codes being written
-    b.keep_fraction = bytes <= keep ? 1.0f : (float)(keep / bytes);
-  }
+  b.keep_fraction = l2_keep_fraction(16.0 * (double)total4);
   QB_CUDA_TRY(cudaMemsetAsync(absmax_slots, 0, sizeof(uint32_t) * (size_t)count, stream));
   act_absmax_kernel<<<(unsigned)blocks1, kActThreads, 0, stream>>>(b);
   QB_CUDA_TRY(cudaGetLastError());

@@ -53,6 +53,7 @@ struct WeightBatch {
   int64_t units_total;
   int64_t units_per_warp;  // contiguous run per warp
   int32_t count;
+  float keep_fraction;     // share of the input that L2 is asked to keep between the range pass and the next
 };
 
 // Position of a warp in the launch's unit sequence.
@@ -108,6 +109,7 @@ __device__ __forceinline__ void flush_range(uint32_t* __restrict__ hi_enc, uint3
 __global__ void __launch_bounds__(kWqThreads)
 weight_range_kernel(const __grid_constant__ WeightBatch b) {
   const int lane = threadIdx.x & 31;
+  const uint64_t pol = policy_evict_last(b.keep_fraction);
   const int warp_in_block = threadIdx.x >> 5;
   const int64_t gwarp = (int64_t)blockIdx.x * kWqWarps + warp_in_block;
   int64_t u = gwarp * b.units_per_warp;
@@ -132,7 +134,7 @@ weight_range_kernel(const __grid_constant__ WeightBatch b) {
       float4 v[4];
 #pragma unroll
       for (int j = 0; j < 4; ++j)
-        if (j < nload) v[j] = __ldg(m.w + (pos.u_local + j) * 32 + lane);
+        if (j < nload) v[j] = ldg_policy(m.w + (pos.u_local + j) * 32 + lane, pol);
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         if (j < nload) {
@@ -276,6 +278,7 @@ weight_pack_kernel(const __grid_constant__ WeightBatch b) {
   if (u >= u_end) return;
 
   UnitWalk pos;
+  const uint64_t pol = policy_evict_first();
   pos.seek(b, u);
   int cur_g = -1;
   GroupParams gp{0.f, 0.f, 1.f};
@@ -289,7 +292,7 @@ weight_pack_kernel(const __grid_constant__ WeightBatch b) {
     float4 v[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j)
-      if (j < nload) v[j] = __ldg(m.w + (pos.u_local + j) * 32 + lane);
+      if (j < nload) v[j] = ldg_policy(m.w + (pos.u_local + j) * 32 + lane, pol);
     uint32_t* const out_base = m.packed + pos.u_local * WORDS;
     const int group_begin = m.group_begin;
     const float* const rlo = m.range_lo;
@@ -327,6 +330,7 @@ weight_fake_kernel(const __grid_constant__ WeightBatch b, int levels) {
   if (u_end > b.units_total) u_end = b.units_total;
   if (u >= u_end) return;
   UnitWalk pos;
+  const uint64_t pol = policy_evict_first();
   pos.seek(b, u);
   int cur_g = -1;
   GroupParams gp{0.f, 0.f, 1.f};
@@ -337,7 +341,7 @@ weight_fake_kernel(const __grid_constant__ WeightBatch b, int levels) {
     float4 v[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j)
-      if (j < nload) v[j] = __ldg(m.w + (pos.u_local + j) * 32 + lane);
+      if (j < nload) v[j] = ldg_policy(m.w + (pos.u_local + j) * 32 + lane, pol);
     float4* const out_base = reinterpret_cast<float4*>(m.packed) + pos.u_local * 32;
     const int group_begin = m.group_begin;
 #pragma unroll
@@ -881,6 +885,7 @@ static qb_status launch_two_pass(const HostWeight* m, int count, int bits, void*
   b.hi_enc = reinterpret_cast<uint32_t*>(static_cast<char*>(ws) + kWsRangeOff);
   b.lo_inv = b.hi_enc + total_groups;
   b.units_total = units;
+  b.keep_fraction = l2_keep_fraction(512.0 * (double)units);
   QB_CUDA_TRY(cudaMemsetAsync(b.hi_enc, 0, sizeof(uint32_t) * 2 * (size_t)total_groups, stream));
 
   const int64_t max_warps = (int64_t)sm_count * 32;  // 4 blocks of 8 warps per SM
@@ -1163,6 +1168,7 @@ static qb_status launch_fake_quantize(const float* w, int64_t N, int64_t K, int 
   b.hi_enc = reinterpret_cast<uint32_t*>(static_cast<char*>(ws) + kWsRangeOff);
   b.lo_inv = b.hi_enc + groups;
   b.units_total = it.units;
+  b.keep_fraction = l2_keep_fraction(512.0 * (double)it.units);
   QB_CUDA_TRY(cudaMemsetAsync(b.hi_enc, 0, sizeof(uint32_t) * 2 * (size_t)groups, stream));
   const int64_t max_warps = (int64_t)sm_count * 32;
   int64_t upw = (it.units + max_warps - 1) / max_warps;
