@@ -40,10 +40,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # launches of one step), from an ncu capture; valid only for the kernel source it was taken on.
 NCU_GEMM_TRAFFIC = {
     # "<sha256 of csrc/gemm.cu + csrc/ptx.cuh>": {<config>: bytes per launch}
-    # profiles/qb_gemm_kernel_config1.md, _config2.md, _config3.md (launch averages of the fp32 kernels).
-    # The key is the source the counters were taken on plus one later edit of host code only (the
-    # token-tile width of launches with fewer tiles than SMs, which configs 1-3 are not).
-    "946abbd4a4a6a087": {"1": 78.1e6, "2": 8.18e6, "3": 4299.1e6},
+    # profiles/qb_gemm_kernel_config1.md, _config2.md, _config3.md (launch averages of the fp32 kernels)
+    "c24f063c4550350d": {"1": 79.0e6, "2": 8.18e6, "3": 4299.2e6},
 }
 
 

@@ -265,6 +265,11 @@ qb_status qb_gemm_i8(const int8_t* xq, const float* act_scale, const int32_t* ro
                      int64_t M, int64_t N, int64_t K, int bits, int groups, const float* out_scale,
                      int8_t* yq, void* ws, size_t ws_bytes, void* cuda_stream);
 qb_status qb_rowsum_i8(const int8_t* xq, int64_t M, int64_t K, int32_t* rowsum, void* cuda_stream);
+/* Stack form of qb_gemm_i8: `y` of descriptor i points to int8 [M][N] (cast to float*) and
+ * out_scales[i] (HOST array of `count` dev pointers) is its output scale; grouping and side-by-side
+ * launches as in qb_layer_linears; each result equals qb_gemm_i8 on the same arguments bit for bit. */
+qb_status qb_layer_linears_i8(const qb_linear_desc* descs /*host*/, const float* const* out_scales /*host*/,
+                              int32_t count, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
  * Quantization-aware fine-tuning (Section 3.1: gradients pass through Q by the straight-through

@@ -32,7 +32,7 @@ EXPORTS = (
     "qb_layer_linears", "qb_quantize_pack_weights_noalloc", "qb_probe_i8_mma", "qb_quantize_act_batch",
     "qb_quantize_pack_weights_batch", "qb_gemm_bf16", "qb_layer_linears_bf16",
     "qb_fake_quantize_weights", "qb_ste_backward", "qb_quantize_embedding", "qb_embedding_lookup",
-    "qb_gemm_i8", "qb_rowsum_i8",
+    "qb_gemm_i8", "qb_rowsum_i8", "qb_layer_linears_i8",
 )
 NOALLOC_MAX_GROUPS = 4096
 
@@ -120,6 +120,8 @@ def lib() -> ctypes.CDLL:
     L.qb_embedding_lookup.restype = i32
     L.qb_gemm_i8.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, ctypes.c_int, ctypes.c_int, vp, vp, vp, sz, vp]
     L.qb_gemm_i8.restype = i32
+    L.qb_layer_linears_i8.argtypes = [ctypes.POINTER(LinearDescC), ctypes.POINTER(vp), i32, vp, sz, vp]
+    L.qb_layer_linears_i8.restype = i32
     L.qb_rowsum_i8.argtypes = [vp, i64, i64, vp, vp]
     L.qb_rowsum_i8.restype = i32
     L.qb_gemm_bf16.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, ctypes.c_int, ctypes.c_int, vp, vp, sz, vp]
@@ -394,6 +396,14 @@ def layer_linears(descs, ws: torch.Tensor) -> None:
     """``qb_layer_linears`` over a list of ``LinearDesc`` (or an array from ``make_desc_array``)."""
     arr = descs if isinstance(descs, ctypes.Array) else make_desc_array(descs)
     _check(lib().qb_layer_linears(arr, len(arr), ws.data_ptr(), ws.numel(), _stream()), "qb_layer_linears")
+
+
+def layer_linears_i8(descs: Sequence[LinearDesc], out_scales: Sequence[torch.Tensor], ws: torch.Tensor) -> None:
+    """``qb_layer_linears_i8``: every ``y`` an int8 [M,N] tensor, ``out_scales[i]`` a device fp32 [1] tensor."""
+    assert len(descs) == len(out_scales) and all(d.y.dtype == torch.int8 for d in descs)
+    arr = make_desc_array(descs)
+    sc = (ctypes.c_void_p * len(descs))(*[t.data_ptr() for t in out_scales])
+    _check(lib().qb_layer_linears_i8(arr, sc, len(arr), ws.data_ptr(), ws.numel(), _stream()), "qb_layer_linears_i8")
 
 
 def layer_linears_bf16(descs, ws: torch.Tensor) -> None:

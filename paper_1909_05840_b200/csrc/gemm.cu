@@ -846,7 +846,8 @@ static qb_status validate_gemm(const int8_t* xq, const float* act_scale, const i
 // One launch over descriptors d[idx[0..count)] (count <= kMaxProblems), all with the same bit width, on at
 // most `max_ctas` CTAs.
 static qb_status launch_group(const qb_linear_desc* d, const int* idx, int count, int32_t* acc_out, void* ws,
-                              int max_ctas, cudaStream_t stream, int out, const float* out_scale = nullptr) {
+                              int max_ctas, cudaStream_t stream, int out,
+                              const float* const* out_scales = nullptr) {
   const int sm_count = max_ctas;
   const int bits = d[idx[0]].bits;
   const int bt = choose_token_tile(d, idx, count, sm_count);
@@ -875,7 +876,7 @@ static qb_status launch_group(const qb_linear_desc* d, const int* idx, int count
     p.q0 = q.q0;
     p.bias = q.bias;
     p.y = q.y;
-    p.out_scale = out_scale;
+    p.out_scale = out_scales ? out_scales[idx[i]] : nullptr;
     p.acc_out = acc_out;
     p.M = (int32_t)q.M;
     p.N = (int32_t)q.N;
@@ -972,8 +973,7 @@ static qb_status side_streams(SideStreams** out) {
 // the start-up and the drain of the pipelines overlap instead of adding up; the launches join the
 // caller's stream before the call returns.  Large stacks keep one launch after the other on all SMs.
 static qb_status launch_stack(const qb_linear_desc* d, int count, void* ws, int sm_count, cudaStream_t stream,
-                              bool bf16) {
-  const int out = bf16 ? kOutBf16 : kOutF32;
+                              int out, const float* const* out_scales = nullptr) {
   std::vector<int> order(count);
   for (int i = 0; i < count; ++i) order[i] = i;
   std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
@@ -1011,7 +1011,7 @@ static qb_status launch_stack(const qb_linear_desc* d, int count, void* ws, int 
                             all_tiles < (int64_t)16 * sm_count;
   if (!side_by_side) {
     for (const Group& g : groups) {
-      qb_status st = launch_group(d, order.data() + g.begin, g.count, nullptr, ws, sm_count, stream, out);
+      qb_status st = launch_group(d, order.data() + g.begin, g.count, nullptr, ws, sm_count, stream, out, out_scales);
       if (st != QB_OK) return st;
     }
     return QB_OK;
@@ -1052,7 +1052,7 @@ static qb_status launch_stack(const qb_linear_desc* d, int count, void* ws, int 
   qb_status first_error = QB_OK;
   for (int g = 0; g < n_groups; ++g) {
     cudaStream_t sg = g == 0 ? stream : side->stream[g - 1];
-    st = launch_group(d, order.data() + groups[g].begin, groups[g].count, nullptr, ws, share[g], sg, out);
+    st = launch_group(d, order.data() + groups[g].begin, groups[g].count, nullptr, ws, share[g], sg, out, out_scales);
     if (st != QB_OK && first_error == QB_OK) first_error = st;
   }
   // always join, also after an error: the caller's stream must not run ahead of the side streams
@@ -1090,11 +1090,11 @@ static qb_status gemm_entry(const int8_t* xq, const float* act_scale, const int3
   d.groups = groups;
   d.y = static_cast<float*>(y);
   const int idx = 0;
-  return qb::launch_group(&d, &idx, 1, acc_out, ws, sms, (cudaStream_t)cuda_stream, out, out_scale);
+  return qb::launch_group(&d, &idx, 1, acc_out, ws, sms, (cudaStream_t)cuda_stream, out, out_scale ? &out_scale : nullptr);
 }
 
 static qb_status stack_entry(const char* who, const qb_linear_desc* descs, int32_t count, void* ws, size_t ws_bytes,
-                             void* cuda_stream, bool bf16) {
+                             void* cuda_stream, int out, const float* const* out_scales = nullptr) {
   if (!descs || count <= 0) {
     qb::set_last_error("%s: descs null or count <= 0", who);
     return QB_ERR_INVALID;
@@ -1108,7 +1108,7 @@ static qb_status stack_entry(const char* who, const qb_linear_desc* descs, int32
   int sms = 0;
   qb_status st = qb::require_sm100(&sms);
   if (st != QB_OK) return st;
-  return qb::launch_stack(descs, count, ws, sms, (cudaStream_t)cuda_stream, bf16);
+  return qb::launch_stack(descs, count, ws, sms, (cudaStream_t)cuda_stream, out, out_scales);
 }
 
 extern "C" qb_status qb_gemm(const int8_t* xq, const float* act_scale, const int32_t* rowsum,
@@ -1182,10 +1182,24 @@ extern "C" qb_status qb_rowsum_i8(const int8_t* xq, int64_t M, int64_t K, int32_
 
 extern "C" qb_status qb_layer_linears(const qb_linear_desc* descs, int32_t count, void* ws, size_t ws_bytes,
                                       void* cuda_stream) {
-  return stack_entry("qb_layer_linears", descs, count, ws, ws_bytes, cuda_stream, false);
+  return stack_entry("qb_layer_linears", descs, count, ws, ws_bytes, cuda_stream, qb::kOutF32);
 }
 
 extern "C" qb_status qb_layer_linears_bf16(const qb_linear_desc* descs, int32_t count, void* ws, size_t ws_bytes,
                                            void* cuda_stream) {
-  return stack_entry("qb_layer_linears_bf16", descs, count, ws, ws_bytes, cuda_stream, true);
+  return stack_entry("qb_layer_linears_bf16", descs, count, ws, ws_bytes, cuda_stream, qb::kOutBf16);
+}
+
+extern "C" qb_status qb_layer_linears_i8(const qb_linear_desc* descs, const float* const* out_scales, int32_t count,
+                                         void* ws, size_t ws_bytes, void* cuda_stream) {
+  if (!out_scales) {
+    qb::set_last_error("qb_layer_linears_i8: out_scales is null");
+    return QB_ERR_INVALID;
+  }
+  for (int i = 0; i < count; ++i)
+    if (!out_scales[i]) {
+      qb::set_last_error("qb_layer_linears_i8: out_scales[%d] is null", i);
+      return QB_ERR_INVALID;
+    }
+  return stack_entry("qb_layer_linears_i8", descs, count, ws, ws_bytes, cuda_stream, qb::kOutI8, out_scales);
 }

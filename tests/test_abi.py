@@ -84,6 +84,7 @@ def test_argument_errors_are_returned_before_any_launch(lib):
     # re-quantized output and int8 row sums
     assert lib.qb_gemm_i8(A, A, A, A, A, A, None, 8, 12, 128, 4, 3, None, A, A, ws_bytes, None) == qb.QB_ERR_INVALID
     assert lib.qb_gemm_i8(A, A, A, A, A, A, None, 8, 12, 192, 4, 3, A, A, A, ws_bytes, None) == qb.QB_ERR_ALIGN
+    assert lib.qb_layer_linears_i8(None, None, 2, A, ws_bytes, None) == qb.QB_ERR_INVALID
     assert lib.qb_rowsum_i8(A, 8, 100, A, None) == qb.QB_ERR_ALIGN
     assert lib.qb_rowsum_i8(None, 8, 128, A, None) == qb.QB_ERR_INVALID
     # fake quantization and its straight-through backward

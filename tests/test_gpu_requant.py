@@ -82,3 +82,27 @@ def test_rowsum_i8_matches_oracle():
         xq = rng.integers(-127, 128, (M, K)).astype(np.int8)
         got = qb.rowsum_i8(torch.from_numpy(xq).cuda()).cpu().numpy()
         assert np.array_equal(got, oracle.rowsum_i8(xq))
+
+
+def test_layer_linears_i8_equals_single_calls(ws):
+    # a small mixed-precision stack (side-by-side launches) with one output scale per linear
+    M = 128
+    shapes = [(256, 256, 2, 4), (384, 512, 4, 6), (128, 1024, 8, 2), (256, 256, 3, 1), (272, 384, 4, 17)]
+    descs, scales, singles = [], [], []
+    for i, (N, K, bits, G) in enumerate(shapes):
+        x = synth.activations(M, K, seed=300 + i)
+        w = synth.weights(N, K, seed=350 + i)
+        b = synth.bias(N, seed=390 + i)
+        xq, sc, rs = gu.gpu_quantize_act(x, ws)
+        packed, delta, q0 = gu.gpu_quantize_weights(w, bits, G, ws)
+        o = oracle.linear(x, w, b, bits, G)
+        s_out = torch.tensor([float(np.float32(np.abs(o["y"]).max() / (90.0 + 10 * i)))], device="cuda")
+        yq = gu.poison(torch.empty((M, N), dtype=torch.int8, device="cuda"))
+        descs.append(qb.LinearDesc(xq, sc, rs, packed, delta, q0, gu.dev(b), N, bits, G, yq))
+        scales.append(s_out)
+        singles.append(qb.gemm_i8(xq, sc, rs, packed, delta, q0, gu.dev(b), N, bits, G, s_out, ws))
+        _check_codes(singles[-1].cpu().numpy(), o["y"], float(s_out.item()))
+    qb.layer_linears_i8(descs, scales, ws)
+    assert qb.read_status(ws) == qb.QB_OK
+    for d, y1 in zip(descs, singles):
+        assert torch.equal(d.y, y1)
