@@ -44,3 +44,22 @@ def test_workload_arithmetic_matches_the_encoder_layer():
     assert bench.gemm_ops(wl) == 2.0 * 4096 * (2304 * 768 + 768 * 768 + 3072 * 768 + 768 * 3072)
     # fp32 outputs dominate the traffic of three of the four GEMMs
     assert 130e6 < bench.gemm_algorithmic_bytes(wl) < 145e6
+
+
+def test_reference_arm_prints_one_json_line_with_the_contract_keys():
+    # `bench.py --impl reference` times the CPU oracle on a bounded sample: no GPU needed
+    import json
+    import subprocess
+    r = subprocess.run([sys.executable, str(ROOT / "bench.py"), "--impl", "reference", "--steps", "1", "--ref-rows", "32"],
+                       capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-500:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    for key in ("impl", "metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better",
+                "scaling", "vs_baseline", "dtype", "data", "config", "cpu_baseline", "e2e"):
+        assert key in d, key
+    assert d["impl"] == "reference" and d["value"] > 0 and d["cpu_baseline"]["kind"] == "oracle"
+    assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["e2e"]["d2h_bytes_per_step"] == 0
+    assert d["e2e"]["value"] == d["value"] and d["vs_baseline"] is None
+
