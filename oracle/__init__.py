@@ -67,6 +67,8 @@ def _lib(omp: bool = False) -> ctypes.CDLL:
         lib.qo_rowsum_i8.restype = None
         lib.qo_ste_backward.argtypes = [vp, vp, i64, i64, i32, vp, vp, vp]
         lib.qo_ste_backward.restype = None
+        lib.qo_sensitivity_bits.argtypes = [vp, i32, i32, vp, i32, vp, vp, vp]
+        lib.qo_sensitivity_bits.restype = i32
         lib.qo_round_bf16.argtypes = [vp, i64, vp]
         lib.qo_round_bf16.restype = None
         lib.qo_quantize_act.argtypes = [vp, i64, i64, vp, vp, vp]
@@ -277,3 +279,17 @@ def rowsum_i8(xq) -> np.ndarray:
     out = np.empty(M, dtype=np.int32)
     _lib().qo_rowsum_i8(_p(xq), M, K, _p(out))
     return out
+
+
+def sensitivity_bits(lam, budget, reverse: bool = False):
+    """Eq. 2: ``(status, omega f64 [L], order i32 [L], bits i32 [L])`` from eigenvalue samples ``lam`` [L, S]
+    and ``budget``, the bit width for each rank of the descending order."""
+    lam = _c(np.asarray(lam), np.float64)
+    L, S = lam.shape
+    budget = _c(np.asarray(budget), np.int32)
+    assert budget.shape == (L,)
+    omega = np.empty(L, np.float64)
+    order = np.empty(L, np.int32)
+    bits = np.empty(L, np.int32)
+    st = _lib().qo_sensitivity_bits(_p(lam), L, S, _p(budget), int(reverse), _p(omega), _p(order), _p(bits))
+    return st, omega, order, bits

@@ -429,4 +429,54 @@ void qo_rowsum_i8(const int8_t* xq, int64_t M, int64_t K, int32_t* rowsum) {
   }
 }
 
+// ---------------------------------------------------------------------------
+// Section 3.2, Eq. 2: sensitivity of encoder layer i from the top Hessian eigenvalues lambda_i measured
+// on `samples` portions of the training data (the caller supplies them; the power iteration that finds
+// them is not part of this library):
+//     Omega_i = |mean(lambda_i)| + std(lambda_i)
+// and the paragraph after it: the layers are sorted by Omega in descending order and the order decides
+// the precision relative to the other layers.
+// Readings: std is the standard deviation of the empirical distribution of the given samples (divide by
+// the number of samples, not by one less); equal Omega keep the lower layer index first; the paper gives
+// no rule from rank to bit width, so the caller supplies `budget`, the bit width for rank 0 (most
+// sensitive), rank 1, ...; `reverse` deals the budget from the least sensitive layer instead (the
+// "MP-rev" ablation of the appendix).
+// lambda: [layers][samples] fp64.  Outputs: omega [layers], order [layers] (order[r] = layer of rank r),
+// bits [layers].  All arithmetic in fp64, sums taken in index order.
+int qo_sensitivity_bits(const double* lambda, int layers, int samples, const int* budget, int reverse,
+                        double* omega, int* order, int* bits) {
+  if (layers < 1 || samples < 1) return QO_ERR_INVALID;
+  for (int r = 0; r < layers; ++r)
+    if (!qo_valid_bits(budget[r])) return QO_ERR_INVALID;
+  for (int i = 0; i < layers; ++i) {
+    const double* l = lambda + (int64_t)i * samples;
+    double sum = 0.0;
+    for (int s = 0; s < samples; ++s) {
+      if (!std::isfinite(l[s])) return QO_ERR_NONFINITE;
+      sum += l[s];
+    }
+    const double mean = sum / (double)samples;
+    double sq = 0.0;
+    for (int s = 0; s < samples; ++s) {
+      const double d = l[s] - mean;
+      sq += d * d;
+    }
+    omega[i] = std::fabs(mean) + std::sqrt(sq / (double)samples);
+  }
+  // descending order by repeated selection of the largest remaining Omega; ties: lower index first
+  for (int i = 0; i < layers; ++i) order[i] = -1;
+  for (int r = 0; r < layers; ++r) {
+    int best = -1;
+    for (int i = 0; i < layers; ++i) {
+      bool taken = false;
+      for (int q = 0; q < r; ++q) taken = taken || order[q] == i;
+      if (taken) continue;
+      if (best < 0 || omega[i] > omega[best]) best = i;
+    }
+    order[r] = best;
+  }
+  for (int r = 0; r < layers; ++r) bits[order[r]] = budget[reverse ? layers - 1 - r : r];
+  return QO_OK;
+}
+
 }  // extern "C"

@@ -13,6 +13,8 @@
 // The array is shared by every call and keeps whatever the last call left in it, so each call
 // clears the parts that must start at zero, and two calls that overlap on the GPU (different
 // streams, or the same stream from two threads without ordering) would race on it.
+#include <atomic>
+
 #include "common.cuh"
 
 namespace qb {
@@ -31,24 +33,24 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratch
 // use: the device address is looked up once per device, with that device current.
 static qb_status noalloc_scratch_ptr(void** out) {
   constexpr int kMaxDev = 64;
-  static void* cached[kMaxDev] = {};
+  static std::atomic<void*> cached[kMaxDev] = {};  // two threads may look the address up at once: both find the same value
   int dev = 0;
   QB_CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= kMaxDev) {
     set_last_error("device ordinal %d out of range", dev);
     return QB_ERR_CUDA;
   }
-  if (cached[dev] == nullptr) {
-    void* p = nullptr;
+  void* p = cached[dev].load(std::memory_order_acquire);
+  if (p == nullptr) {
     cudaError_t e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
     if (e != cudaSuccess) return cuda_fail(e, "cudaGetSymbolAddress(g_noalloc_scratch)");
     if (p == nullptr) {
       set_last_error("cudaGetSymbolAddress returned a null address for the built-in scratch");
       return QB_ERR_CUDA;
     }
-    cached[dev] = p;
+    cached[dev].store(p, std::memory_order_release);
   }
-  *out = cached[dev];
+  *out = p;
   return QB_OK;
 }
 

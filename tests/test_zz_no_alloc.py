@@ -3,13 +3,17 @@
 Collected last on purpose (file name): a run that stops at the first failure has then already run
 every other test.  The entry point keeps its scratch in an array inside the library, shared by all
 calls, so the test makes two calls in a row -- the second on a different matrix, bit width and group
-count -- and compares each with qb_quantize_pack_weights (caller workspace) on the same input.  Packed
-words, Delta and q0 are integer / byte-exact results in this library's tests, so they must be equal.
+count -- and compares each with qb_quantize_pack_weights (caller workspace) on the same input and with
+the CPU oracle's quantizer and packer.  Packed words, Delta and q0 are integer / byte-exact results in
+this library's tests, so they must be equal.  The shapes are chosen so that the built-in scratch is used
+by each of the quantizer's kernels: groups kept in registers, groups streamed through the shared-memory
+ring, and the two-pass path.
 """
 import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_1909_05840_b200 as qb
 from paper_1909_05840_b200 import build as qb_build
 from paper_1909_05840_b200 import synth
@@ -30,8 +34,11 @@ def test_noalloc_matches_workspace_entry_point_twice_in_a_row():
     ws = qb.workspace(groups=qb.NOALLOC_MAX_GROUPS)
     status = torch.full((1,), 77, dtype=torch.int32, device="cuda")
     # second call: fewer groups, other width and shape, so that stale ranges of call 1 would show
-    for call, (N, K, bits, groups) in enumerate([(768, 768, 3, 768), (264, 384, 4, 11)]):
-        w = torch.from_numpy(synth.weights(N, K, seed=900 + call)).cuda()
+    # (3072, 768, 128 groups): 144 units of 128 weights per group, more groups than half the SMs -> the shared-memory ring
+    for call, (N, K, bits, groups) in enumerate([(768, 768, 3, 768), (264, 384, 4, 11), (3072, 768, 2, 128),
+                                                 (768, 3072, 8, 1)]):
+        w_host = synth.weights(N, K, seed=900 + call)
+        w = torch.from_numpy(w_host).cuda()
         ref_packed, ref_delta, ref_q0 = qb.quantize_pack_weights(w, bits, groups, ws)
         packed, delta, q0 = _outputs(N, K, bits, groups)
         qb.quantize_pack_weights_noalloc(w, bits, groups, packed, delta, q0, status_out=status)
@@ -39,6 +46,11 @@ def test_noalloc_matches_workspace_entry_point_twice_in_a_row():
         assert status.item() == qb.QB_OK
         assert torch.equal(packed, ref_packed), f"call {call}: packed words differ"
         assert torch.equal(delta, ref_delta) and torch.equal(q0, ref_q0), f"call {call}: group tables differ"
+        # and against the oracle directly, not only against the library's other entry point
+        st, codes, o_delta, o_q0 = oracle.quantize_weights(w_host, bits, groups, omp=True)
+        assert st == oracle.OK
+        assert np.array_equal(packed.cpu().numpy().view(np.uint32), oracle.pack(codes, bits)), f"call {call}: words vs oracle"
+        assert np.array_equal(delta.cpu().numpy(), o_delta) and np.array_equal(q0.cpu().numpy(), o_q0)
     assert qb.read_status(ws) == qb.QB_OK
 
     # a non-finite weight is reported through status_out for that call only; the next call is clean again
