@@ -330,6 +330,32 @@ qb_status qb_embedding_lookup(const int32_t* ids, int64_t T, const uint32_t* pac
                               float* out, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * Mixed-precision assignment from Hessian spectra (Section 3.2, Eq. 2 and the paragraph after it).
+ * Host-only: no GPU work, no stream, all pointers are HOST pointers.
+ *
+ *   Omega_i = | mean(lambda_i) | + std(lambda_i)
+ *
+ * where lambda_i are the top eigenvalues of the Hessian of encoder layer i measured on `samples`
+ * portions of the training data (the caller computes them; the power iteration is not part of this
+ * library).  The layers are sorted by Omega in descending order (equal Omega: lower layer first) and
+ * the layer of rank r receives budget_bits[r].  The paper fixes the ordering but no rule from rank to
+ * bit width, so the budget is the caller's (e.g. six 3s then six 2s for the 2/3-bit mixed setting of
+ * a 12-layer encoder).  std is the standard deviation of the empirical distribution of the samples
+ * (divisor `samples`).  All arithmetic in fp64, sums in index order.
+ *   lambda       host fp64 [layers][samples]                         (read)
+ *   budget_bits  host int32 [layers], each in {2,3,4,8}; entry r is the width for rank r (read)
+ *   reverse      0: as above; != 0: rank r receives budget_bits[layers-1-r] (the appendix's
+ *                "MP-rev" ablation: fewest bits to the most sensitive layer)
+ *   omega_out    host fp64 [layers] or NULL                          (written)
+ *   order_out    host int32 [layers] or NULL: order_out[r] = layer of rank r   (written)
+ *   bits_out     host int32 [layers]: bit width per layer, ready for qb_linear_desc.bits (written)
+ * Returns QB_ERR_INVALID for null pointers, sizes < 1 or a budget entry outside {2,3,4,8};
+ * QB_ERR_NONFINITE if a sample is NaN or Inf (nothing is written then).
+ */
+qb_status qb_sensitivity_bits(const double* lambda, int32_t layers, int32_t samples, const int32_t* budget_bits,
+                              int32_t reverse, double* omega_out, int32_t* order_out, int32_t* bits_out);
+
+/*
  * Diagnostic: the rate the tensor cores sustain for the GEMM's own instruction (tcgen05.mma kind::i8,
  * s8 x s8 -> s32, 128 x `tokens` x 32) with both operands resident in shared memory, no global
  * traffic, four K blocks in flight, one CTA per SM on the default stream.  (No counterpart in the

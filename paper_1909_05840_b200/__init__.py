@@ -32,7 +32,7 @@ EXPORTS = (
     "qb_layer_linears", "qb_quantize_pack_weights_noalloc", "qb_probe_i8_mma", "qb_quantize_act_batch",
     "qb_quantize_pack_weights_batch", "qb_gemm_bf16", "qb_layer_linears_bf16",
     "qb_fake_quantize_weights", "qb_ste_backward", "qb_quantize_embedding", "qb_embedding_lookup",
-    "qb_gemm_i8", "qb_rowsum_i8", "qb_layer_linears_i8",
+    "qb_gemm_i8", "qb_rowsum_i8", "qb_layer_linears_i8", "qb_sensitivity_bits",
 )
 NOALLOC_MAX_GROUPS = 4096
 
@@ -101,6 +101,8 @@ def lib() -> ctypes.CDLL:
     L.qb_quantize_pack_weights_noalloc.restype = i32
     L.qb_probe_i8_mma.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
     L.qb_probe_i8_mma.restype = i32
+    L.qb_sensitivity_bits.argtypes = [vp, i32, i32, vp, i32, vp, vp, vp]
+    L.qb_sensitivity_bits.restype = i32
     L.qb_quantize_act_batch.argtypes = [ctypes.POINTER(ActDescC), i32, vp, sz, vp]
     L.qb_quantize_act_batch.restype = i32
     L.qb_quantize_pack_weights_batch.argtypes = [ctypes.POINTER(WeightDescC), i32, vp, sz, vp]
@@ -310,6 +312,23 @@ def probe_i8_mma(tokens: int = 256, k_blocks: int = 20000):
     tops, cyc = ctypes.c_double(0.0), ctypes.c_double(0.0)
     _check(lib().qb_probe_i8_mma(tokens, k_blocks, ctypes.byref(tops), ctypes.byref(cyc)), "qb_probe_i8_mma")
     return tops.value, cyc.value
+
+
+def sensitivity_bits(lam, budget_bits, reverse: bool = False):
+    """``qb_sensitivity_bits`` (host only): ``lam`` [layers, samples] eigenvalue samples, ``budget_bits`` the bit
+    width for each rank of the descending Omega order.  Returns (omega f64 [L], order i32 [L], bits i32 [L])."""
+    import numpy as np
+    lam = np.ascontiguousarray(lam, dtype=np.float64)
+    budget = np.ascontiguousarray(budget_bits, dtype=np.int32)
+    layers, samples = lam.shape
+    if budget.shape != (layers,):
+        raise QbertError(QB_ERR_INVALID, "budget_bits must have one entry per layer")
+    omega = np.empty(layers, np.float64)
+    order = np.empty(layers, np.int32)
+    bits = np.empty(layers, np.int32)
+    _check(lib().qb_sensitivity_bits(lam.ctypes.data, layers, samples, budget.ctypes.data, int(reverse),
+                                     omega.ctypes.data, order.ctypes.data, bits.ctypes.data), "qb_sensitivity_bits")
+    return omega, order, bits
 
 
 def gemm(xq: torch.Tensor, act_scale: torch.Tensor, rowsum: torch.Tensor, packed: torch.Tensor,

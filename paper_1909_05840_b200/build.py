@@ -10,7 +10,7 @@ PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 INCLUDE = PKG.parent / "include"
 LIB = PKG / "libqbert.so"
-SOURCES = ["api.cu", "quantize_act.cu", "quantize_weights.cu", "quantize_weights_noalloc.cu", "gemm.cu", "probe.cu", "embedding.cu"]
+SOURCES = ["api.cu", "quantize_act.cu", "quantize_weights.cu", "quantize_weights_noalloc.cu", "gemm.cu", "probe.cu", "embedding.cu", "sensitivity.cu"]
 
 
 def _nvcc() -> str:
