@@ -37,12 +37,12 @@ NOMINAL_INT8_OVER_BF16 = 2.0  # dense int8 peak / dense bf16 peak (4.5 / 2.25 PF
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 # DRAM traffic of qb_gemm per launch (dram__bytes_read.sum + dram__bytes_write.sum averaged over the
-# launches of one step), from an ncu capture; valid only for the kernel source it was taken on.
+# launches of one step), from an ncu capture; valid only for the kernel source it was taken on, so the
+# table is keyed by a hash of that source and reads null as soon as the kernel changes.
 NCU_GEMM_TRAFFIC = {
     # "<sha256 of csrc/gemm.cu + csrc/ptx.cuh>": {<config>: bytes per launch}
-    # profiles/qb_gemm_kernel_config1.md, _config2.md, _config3.md (launch averages of the fp32 kernels)
-    "c24f063c4550350d": {"1": 79.0e6, "2": 8.18e6, "3": 4299.2e6},
 }
+NOMINAL_INT8_TOPS = 4500.0  # dense int8 tensor peak of the part as published (context, not the denominator)
 
 
 def kernel_source_hash() -> str:
@@ -202,37 +202,72 @@ def aggregate_over_ranks(local_ms: float, local_units: float, world: int, dist=N
     return float(t.item()), float(u.item())
 
 
-def run_ours(args, wl):
-    import torch
-    import paper_1909_05840_b200 as qb
-    from paper_1909_05840_b200 import build as qb_build
+def gemm_rooflines(wl: synth.Workload, out_bytes: float, int8_peak_tops: float, hbm_gbs: float):
+    """Per-GEMM ideal times: (sum over the linears of max(t_tensor, t_hbm), sum of t_tensor, sum of t_hbm, seconds)."""
+    t_max = t_tensor = t_hbm = 0.0
+    for _, _, s, bits in linear_list(wl):
+        ops = 2.0 * wl.M * s.N * s.K
+        byts = wl.M * s.K + s.N * s.K * bits / 8 + out_bytes * wl.M * s.N + 4 * s.N + 4 * wl.M + 8 * s.groups
+        tt, th = ops / (int8_peak_tops * 1e12), byts / (hbm_gbs * 1e9)
+        t_max += max(tt, th)
+        t_tensor += tt
+        t_hbm += th
+    return t_max, t_tensor, t_hbm
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: libqbert has no CPU path")
-    torch.cuda.set_device(local_rank)
-    device = torch.device("cuda", local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist_mod
-        dist = dist_mod
-        dist.init_process_group("nccl", device_id=device)
-    if rank == 0:
-        qb_build.build()
-    if dist is not None:
-        dist.barrier()
-    qb.lib()
 
-    # ---- inputs: pinned host copies (for the end-to-end arm) and resident device copies ------------
+class Runner:
+    """Device state of one rank, shared by the workloads measured in one run."""
+
+    def __init__(self, args):
+        import torch
+        import paper_1909_05840_b200 as qb
+        from paper_1909_05840_b200 import build as qb_build
+        self.torch, self.qb, self.args = torch, qb, args
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: libqbert has no CPU path")
+        torch.cuda.set_device(self.local_rank)
+        self.device = torch.device("cuda", self.local_rank)
+        self.dist = None
+        if self.world > 1:
+            import torch.distributed as dist_mod
+            self.dist = dist_mod
+            self.dist.init_process_group("nccl", device_id=self.device)
+        if self.rank == 0:
+            qb_build.build()
+        if self.dist is not None:
+            self.dist.barrier()
+        qb.lib()
+        self.flush = torch.empty(512 << 20, dtype=torch.uint8, device=self.device)  # > L2 (126 MB)
+        self.clean = torch.zeros(256 << 20, dtype=torch.uint8, device=self.device).view(torch.int32)
+
+    def flush_l2(self, i):
+        # untimed: a 512 MiB write evicts the previous step's tensors; a 256 MiB read of another buffer
+        # then leaves L2 holding clean, unrelated lines, so that the timed step does not also pay for
+        # writing back the flush buffer's dirty lines
+        self.flush.fill_(i & 0xFF)
+        self.clean.sum()
+
+    def sync_all(self):
+        self.torch.cuda.synchronize(self.device)
+        if self.dist is not None:
+            self.dist.barrier()
+            self.torch.cuda.synchronize(self.device)
+
+
+def measure(R: Runner, wl: synth.Workload, steps: int, with_e2e: bool, warm_too: bool = False):
+    """Time `steps` whole steps of workload `wl` (and its phases) on this rank.  Returns a dict of
+    local timings; the caller aggregates over ranks."""
+    torch, qb, args, device = R.torch, R.qb, R.args, R.device
     lin = linear_list(wl)
     host, devb = [], []
     ws = qb.workspace(groups=max(32, sum(s.groups for *_, s, _ in lin)), device=device)
     ws_w = qb.workspace(groups=max(32, sum(s.groups for *_, s, _ in lin)), device=device)  # weight quantizer's own
     cache = {}
     for layer, mi, s, bits in lin:
-        seed = synth.seed_for(wl.config, layer, mi) + 100000 * rank
+        seed = synth.seed_for(wl.config, layer, mi) + 100000 * R.rank
         key = (s.N, s.K) if wl.layers > 4 else None  # deep stacks: reuse the host arrays per shape
         if key is not None and key in cache:
             x, w, b = cache[key]
@@ -259,11 +294,11 @@ def run_ours(args, wl):
     act_arr = qb.make_act_desc_array([(d["x"], d["xq"], d["sc"], d["rs"]) for d in devb])
     w_arr = qb.make_weight_desc_array([(d["w"], d["bits"], d["s"].groups, d["packed"], d["delta"], d["q0"])
                                        for d in devb])
-    # kernels launched per step (the library splits a stack by bit width and by its batch limits)
+    # kernels launched per step, counted from the library's own launch plan for these descriptors
+    gemm_launches = qb.layer_linears_launch_count(descs)
     per_bits = {}
     for d in devb:
         per_bits[d["bits"]] = per_bits.get(d["bits"], 0) + 1
-    gemm_launches = sum(-(-n // 16) for n in per_bits.values())
     launches_per_step = 2 * -(-len(lin) // 32) + sum(2 * -(-n // 32) for n in per_bits.values()) + gemm_launches
 
     def phase_act():
@@ -291,29 +326,12 @@ def run_ours(args, wl):
         cur.wait_stream(side)
         phase_gemm()
 
-    flush = torch.empty(512 << 20, dtype=torch.uint8, device=device)  # > L2 (126 MB)
-    clean = torch.zeros(256 << 20, dtype=torch.uint8, device=device).view(torch.int32)
-
-    def flush_l2(i):
-        # untimed: a 512 MiB write evicts the previous step's tensors; a 256 MiB read of another buffer
-        # then leaves L2 holding clean, unrelated lines, so that the timed step does not also pay for
-        # writing back the flush buffer's dirty lines
-        flush.fill_(i & 0xFF)
-        clean.sum()
-
     direct = (phase_act, phase_weights, phase_gemm)
-
-    def sync_all():
-        torch.cuda.synchronize(device)
-        if dist is not None:
-            dist.barrier()
-            torch.cuda.synchronize(device)
-
     for _ in range(max(3, args.warmup)):
         phase_act(); phase_weights(); phase_gemm()
-    sync_all()
+    R.sync_all()
     whole_step()
-    sync_all()
+    R.sync_all()
     assert qb.read_status(ws) == qb.QB_OK and qb.read_status(ws_w) == qb.QB_OK, "device status word reports an error"
 
     if not args.no_graphs:
@@ -331,150 +349,236 @@ def run_ours(args, wl):
         whole_step = g_step.replay
         for _ in range(3):
             phase_act(); phase_weights(); phase_gemm(); whole_step()
-        sync_all()
+        R.sync_all()
 
-    sampler = ClockSampler(local_rank)
+    sampler = ClockSampler(R.local_rank)
     sampler.start()
     # keep the GPU busy for a moment so that the clock samples are taken under load
     t_busy = time.time()
     while time.time() - t_busy < args.busy_ms * 1e-3:
         whole_step()
-    sync_all()
+    R.sync_all()
 
     # the timed region: K whole steps, each bracketed by its own pair of events (the flush is untimed)
-    sev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
-    sync_all()
+    sev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(steps)]
+    R.sync_all()
     t_wall0 = time.time()
-    for i in range(args.steps):
-        flush_l2(i)
+    for i in range(steps):
+        R.flush_l2(i)
         sev[i][0].record(); whole_step(); sev[i][1].record()
-    sync_all()
+    R.sync_all()
     t_wall1 = time.time()
-    ms_step = float(np.mean([e[0].elapsed_time(e[1]) for e in sev]))
+    step_ms = [e[0].elapsed_time(e[1]) for e in sev]
     # the phases one after the other, for the per-kernel figures (same flush, same graphs)
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
-    for i in range(args.steps):
-        flush_l2(i)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)]
+    for i in range(steps):
+        R.flush_l2(i)
         ev[i][0].record(); phase_act()
         ev[i][1].record(); phase_weights()
         ev[i][2].record(); phase_gemm()
         ev[i][3].record()
-    sync_all()
-    sampler.stop()
+    R.sync_all()
+    t_wall2 = time.time()
+    clocks = sampler.summary(t_wall0, t_wall1)
+    clocks_phases = sampler.summary(t_wall1, t_wall2)
     assert qb.read_status(ws) == qb.QB_OK and qb.read_status(ws_w) == qb.QB_OK, "device status word reports an error"
-    ms_act = float(np.mean([e[0].elapsed_time(e[1]) for e in ev]))
-    ms_w = float(np.mean([e[1].elapsed_time(e[2]) for e in ev]))
-    ms_gemm = float(np.mean([e[2].elapsed_time(e[3]) for e in ev]))
-    ms_serial = float(np.mean([e[0].elapsed_time(e[3]) for e in ev]))
+    res = {
+        "ms_step": float(np.median(step_ms)), "ms_step_mean": float(np.mean(step_ms)),
+        "ms_act": float(np.median([e[0].elapsed_time(e[1]) for e in ev])),
+        "ms_w": float(np.median([e[1].elapsed_time(e[2]) for e in ev])),
+        "ms_gemm": float(np.median([e[2].elapsed_time(e[3]) for e in ev])),
+        "ms_serial": float(np.median([e[0].elapsed_time(e[3]) for e in ev])),
+        "clocks": clocks, "clocks_phases": clocks_phases,
+        "gemm_launches": gemm_launches, "launches_per_step": launches_per_step, "linears": len(lin),
+    }
+    if warm_too:
+        # warm: the same graphs replayed back to back with no flush in between (weights, codes and outputs
+        # of a small stack stay in the 126 MB L2 from one replay to the next)
+        wev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(steps)]
+        gev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(steps)]
+        for i in range(steps):
+            wev[i][0].record(); whole_step(); wev[i][1].record()
+        for i in range(steps):
+            gev[i][0].record(); phase_gemm(); gev[i][1].record()
+        R.sync_all()
+        res["ms_step_warm"] = float(np.median([e[0].elapsed_time(e[1]) for e in wev]))
+        res["ms_gemm_warm"] = float(np.median([e[0].elapsed_time(e[1]) for e in gev]))
+    sampler.stop()
 
-    # ---- end to end: host buffers in, results out, copies inside the timed region ------------------
-    e2e_steps = max(1, min(args.steps, args.e2e_steps))  # a shorter loop: each step moves ~250 MB over PCIe
-    y_host = [torch.empty((wl.M, d["s"].N), dtype=d["y"].dtype).pin_memory() for d in devb]
-    h2d = sum(x.numel() * 4 + w.numel() * 4 + b.numel() * 4 for x, w, b in host)
-    d2h = sum(y.numel() * y.element_size() for y in y_host)
+    if with_e2e:
+        # ---- end to end: host buffers in, results out, copies inside the timed region ------------------
+        e2e_steps = max(1, min(steps, args.e2e_steps))
+        # pinned result buffers: one per output shape (a deep stack reads every layer's result back into
+        # the buffer of its shape; every byte still crosses the link)
+        y_pool = {}
+        y_host = []
+        for d in devb:
+            key = (tuple(d["y"].shape), d["y"].dtype)
+            if key not in y_pool or wl.layers <= 4:
+                y_pool[key] = torch.empty(d["y"].shape, dtype=d["y"].dtype).pin_memory()
+            y_host.append(y_pool[key])
+        h2d = sum(x.numel() * 4 + w.numel() * 4 + b.numel() * 4 for x, w, b in host)
+        d2h = sum(d["y"].numel() * d["y"].element_size() for d in devb)
 
-    # Host -> device copies, the step and device -> host copies run on three streams chained by events, so
-    # that the read-back of step i and the upload of step i + 1 share the (full-duplex) link: the upload
-    # waits for step i's kernels (it overwrites their inputs), the kernels of step i + 1 wait for the
-    # upload and for the read-back of step i (they overwrite its outputs).  Every step still moves all
-    # its inputs in and all its outputs out inside the timed region.
-    s_in, s_out = torch.cuda.Stream(device=device), torch.cuda.Stream(device=device)
-    ev_in, ev_comp, ev_out = torch.cuda.Event(), torch.cuda.Event(), torch.cuda.Event()
+        # Host -> device copies, the step and device -> host copies run on three streams chained by events, so
+        # that the read-back of step i and the upload of step i + 1 share the (full-duplex) link: the upload
+        # waits for step i's kernels (it overwrites their inputs), the kernels of step i + 1 wait for the
+        # upload and for the read-back of step i (they overwrite its outputs).  Every step still moves all
+        # its inputs in and all its outputs out inside the timed region.
+        s_in, s_out = torch.cuda.Stream(device=device), torch.cuda.Stream(device=device)
+        ev_in, ev_comp, ev_out = torch.cuda.Event(), torch.cuda.Event(), torch.cuda.Event()
 
-    def e2e_step():
-        main = torch.cuda.current_stream(device)
-        s_in.wait_event(ev_comp)
-        with torch.cuda.stream(s_in):
-            for (x, w, b), d in zip(host, devb):
-                d["x"].copy_(x, non_blocking=True)
-                d["w"].copy_(w, non_blocking=True)
-                d["b"].copy_(b, non_blocking=True)
-            ev_in.record(s_in)
-        main.wait_event(ev_in)
-        main.wait_event(ev_out)
-        whole_step()
-        ev_comp.record(main)
-        s_out.wait_event(ev_comp)
-        with torch.cuda.stream(s_out):
-            for yh, d in zip(y_host, devb):
-                yh.copy_(d["y"], non_blocking=True)
-            ev_out.record(s_out)
+        def e2e_step():
+            main = torch.cuda.current_stream(device)
+            s_in.wait_event(ev_comp)
+            with torch.cuda.stream(s_in):
+                for (x, w, b), d in zip(host, devb):
+                    d["x"].copy_(x, non_blocking=True)
+                    d["w"].copy_(w, non_blocking=True)
+                    d["b"].copy_(b, non_blocking=True)
+                ev_in.record(s_in)
+            main.wait_event(ev_in)
+            main.wait_event(ev_out)
+            whole_step()
+            ev_comp.record(main)
+            s_out.wait_event(ev_comp)
+            with torch.cuda.stream(s_out):
+                for yh, d in zip(y_host, devb):
+                    yh.copy_(d["y"], non_blocking=True)
+                ev_out.record(s_out)
 
-    e2e_step()
-    sync_all()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(e2e_steps):
         e2e_step()
-    torch.cuda.current_stream(device).wait_event(ev_out)  # the last read-back is inside the timed region
-    e1.record()
-    sync_all()
-    ms_e2e = e0.elapsed_time(e1) / e2e_steps
+        R.sync_all()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(e2e_steps):
+            e2e_step()
+        torch.cuda.current_stream(device).wait_event(ev_out)  # the last read-back is inside the timed region
+        e1.record()
+        R.sync_all()
+        res.update({"ms_e2e": e0.elapsed_time(e1) / e2e_steps, "e2e_steps": e2e_steps, "h2d": h2d, "d2h": d2h})
+    return res
 
+
+def pick_int8_peak(peaks, clocks):
+    """The tensor denominator for this run: the measured bf16 rate (burst for a short phase at full clock,
+    sustained when the power cap was seen or the clock sat below its maximum) times the nominal
+    int8 / bf16 ratio."""
+    capped = "sw_power_cap" in (clocks.get("reasons") or [])
+    mhz, mx = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
+    low = mhz is not None and mx is not None and mhz < 0.95 * mx
+    if capped or low:
+        return peaks["bf16_tflops_sustained"] * NOMINAL_INT8_OVER_BF16, "sustained bf16 measured peak x 2 (power cap or clock below maximum seen during the GEMM phase)"
+    return peaks["bf16_tflops"] * NOMINAL_INT8_OVER_BF16, "burst bf16 measured peak x 2 (short phase at full clock, no power cap seen)"
+
+
+def gemm_roofline_block(wl, res, peaks, peak_kind, out_bytes, probe_tops, probe_cycles, ms_gemm):
+    ops = gemm_ops(wl)
+    gemm_bytes = gemm_algorithmic_bytes(wl, out_bytes)
+    n_gemm = res["gemm_launches"]
+    s_gemm = ms_gemm * 1e-3
+    int8_peak, peak_note = pick_int8_peak(peaks, res["clocks_phases"])
+    t_max, t_tensor, t_hbm = gemm_rooflines(wl, out_bytes, int8_peak, peaks["hbm_gbs"])
+    achieved_tops = ops / s_gemm / 1e12
+    achieved_gbs = gemm_bytes / s_gemm / 1e9
+    if t_hbm >= t_tensor:
+        roof = {"bound": "hbm", "achieved": achieved_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    else:
+        roof = {"bound": "tensor", "achieved": achieved_tops, "peak": int8_peak, "unit": "TOP/s"}
+    burst, sust = peaks["bf16_tflops"] * NOMINAL_INT8_OVER_BF16, peaks["bf16_tflops_sustained"] * NOMINAL_INT8_OVER_BF16
+    roof.update({
+        # per GEMM: sum over the linears of max(t_tensor, t_hbm), divided by the measured time of the launches
+        "frac": t_max / s_gemm,
+        "frac_note": "sum over the linears of max(ideal tensor time, ideal HBM time) / measured time of the GEMM launches",
+        "traffic": (NCU_GEMM_TRAFFIC.get(kernel_source_hash(), {}).get(str(wl.config)) if out_bytes == 4.0 else None),
+        "kernel": "qb_gemm_kernel", "launches_per_step": n_gemm, "linears_per_step": res["linears"],
+        "us_per_launch": s_gemm * 1e6 / n_gemm, "us_gemm_phase": s_gemm * 1e6,
+        "algorithmic_bytes_per_launch": gemm_bytes / n_gemm, "algorithmic_ops_per_launch": ops / n_gemm,
+        "peak_source": f"{peak_kind} (MEASURED_PEAKS.json)" if peak_kind == "measured" else "fallback",
+        "int8_peak_tops": int8_peak, "int8_peak_note": peak_note,
+        "achieved_tops": achieved_tops, "achieved_GBps": achieved_gbs,
+        "tensor_frac_of_burst_x2": achieved_tops / burst, "tensor_frac_of_sustained_x2": achieved_tops / sust,
+        "frac_of_probed_int8": achieved_tops / probe_tops, "frac_of_nominal_int8": achieved_tops / NOMINAL_INT8_TOPS,
+        "hbm_frac": achieved_gbs / peaks["hbm_gbs"],
+        "probed_int8_tops": probe_tops, "probed_cycles_per_k_block": probe_cycles,
+    })
+    return roof
+
+
+def run_ours(args, wl):
+    R = Runner(args)
+    torch, qb, device, dist, world, rank = R.torch, R.qb, R.device, R.dist, R.world, R.rank
+    res = measure(R, wl, args.steps, with_e2e=True, warm_too=(wl.M <= 256))
+    # the small-M, weight-bandwidth-bound stack (12-layer mixed precision at M = 128) in the same run
+    small = None
+    if wl.config != 2 and not args.no_small_m:
+        wl2 = synth.workload(2)
+        small = (wl2, measure(R, wl2, max(args.steps, 20), with_e2e=False, warm_too=True))
     probe_tops, probe_cycles = qb.probe_i8_mma(256, 20000)
     ops = gemm_ops(wl)
-    ms_job, ops_job = aggregate_over_ranks(ms_step, ops, world, dist, device)
-    ms_e2e_job, _ = aggregate_over_ranks(ms_e2e, ops, world, dist, device)
-    ms_gemm_job, _ = aggregate_over_ranks(ms_gemm, ops, world, dist, device)
+    ms_job, ops_job = aggregate_over_ranks(res["ms_step"], ops, world, dist, device)
+    ms_e2e_job, _ = aggregate_over_ranks(res["ms_e2e"], ops, world, dist, device)
+    ms_gemm_job, _ = aggregate_over_ranks(res["ms_gemm"], ops, world, dist, device)
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
 
     peaks, peak_kind = measured_peaks()
-    n_gemm = gemm_launches
-    gemm_bytes = gemm_algorithmic_bytes(wl, 2.0 if args.out == "bf16" else 4.0)
-    gemm_s_per_launch = ms_gemm * 1e-3 / n_gemm
-    achieved_gbs = gemm_bytes / n_gemm / gemm_s_per_launch / 1e9
-    achieved_tops = ops / n_gemm / gemm_s_per_launch / 1e12
-    int8_peak = peaks["bf16_tflops_sustained"] * NOMINAL_INT8_OVER_BF16
-    t_hbm = gemm_bytes / (peaks["hbm_gbs"] * 1e9)
-    t_tensor = ops / (int8_peak * 1e12)
-    if t_hbm >= t_tensor:
-        roof = {"bound": "hbm", "achieved": achieved_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved_gbs / peaks["hbm_gbs"]}
-    else:
-        roof = {"bound": "tensor", "achieved": achieved_tops, "peak": int8_peak, "unit": "TOP/s",
-                "frac": achieved_tops / int8_peak}
-    traffic = NCU_GEMM_TRAFFIC.get(kernel_source_hash(), {}).get(str(wl.config)) if args.out == "f32" else None
-    roof.update({
-        "traffic": traffic, "kernel": "qb_gemm_kernel", "launches_per_step": n_gemm,
-        "us_per_launch": gemm_s_per_launch * 1e6, "algorithmic_bytes_per_launch": gemm_bytes / n_gemm,
-        "peak_source": f"{peak_kind} (MEASURED_PEAKS.json)" if peak_kind == "measured" else "fallback",
-        "tensor_frac_of_int8_peak": achieved_tops / int8_peak,
-        "int8_peak_note": "sustained bf16 measured peak x nominal int8/bf16 ratio 2.0",
-        "hbm_frac": achieved_gbs / peaks["hbm_gbs"],
-        "linears_per_step": len(lin),
-        "probed_int8_tops": probe_tops, "probed_cycles_per_k_block": probe_cycles,
-        "frac_of_probed_int8": achieved_tops / probe_tops,
-    })
+    out_bytes = 2.0 if args.out == "bf16" else 4.0
+    roof = gemm_roofline_block(wl, res, peaks, peak_kind, out_bytes, probe_tops, probe_cycles, res["ms_gemm"])
+    gemm_bytes = gemm_algorithmic_bytes(wl, out_bytes)
+    l2_note = "untimed between timed steps: 512 MiB flush write, then a 256 MiB read of another buffer (L2 left with clean lines)"
 
     line = {
         "metric": METRIC, "value": ops_job / (ms_job * 1e-3) / 1e12, "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_job, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
-        "config": {"workload": wl.name, "config_index": wl.config, "M": wl.M, "linears": n_gemm,
+        "config": {"workload": wl.name, "config_index": wl.config, "M": wl.M, "linears": res["linears"],
+                   "gemm_launches": res["gemm_launches"],
                    "bits": sorted(set(wl.bits)), "output": "fp32" if args.out == "f32" else "bfloat16 (narrow-output epilogue)",
-                   "l2": "untimed between timed steps: 512 MiB flush write, then a 256 MiB read of another buffer (L2 left with clean lines)",
+                   "l2": l2_note, "timing": "median of per-step CUDA-event times",
                    "step": "quantize_act_batch beside quantize_pack_weights_batch (two streams), then layer_linears over all linears",
                    "launch": "direct C-ABI calls" if args.no_graphs else "C-ABI calls captured once per phase into CUDA graphs, replayed"},
-        "clocks": sampler.summary(t_wall0, t_wall1),
-        "e2e": {"value": ops_job / (ms_e2e_job * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e_job, "steps": e2e_steps},
-        "gpu_launches": launches_per_step * args.steps,
+        "clocks": res["clocks"],
+        "e2e": {"value": ops_job / (ms_e2e_job * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": res["h2d"],
+                "d2h_bytes_per_step": res["d2h"], "ms_per_step": ms_e2e_job, "steps": res["e2e_steps"]},
+        "gpu_launches": res["launches_per_step"] * args.steps,
         "roofline": roof,
         "phases": {
-            "note": "measured one after the other in a second loop of the same length; ms_serial is their sum as timed",
-            "ms_serial": ms_serial,
-            "quantize_act": {"ms": ms_act, "GBps": act_quant_algorithmic_bytes(wl) / (ms_act * 1e-3) / 1e9,
-                             "frac_hbm": act_quant_algorithmic_bytes(wl) / (ms_act * 1e-3) / 1e9 / peaks["hbm_gbs"]},
-            "quantize_pack_weights": {"ms": ms_w,
-                                      "GBps": weight_quant_algorithmic_bytes(wl) / (ms_w * 1e-3) / 1e9,
-                                      "frac_hbm": weight_quant_algorithmic_bytes(wl) / (ms_w * 1e-3) / 1e9 / peaks["hbm_gbs"]},
-            "gemm": {"ms": ms_gemm_job, "TOPS": ops / (ms_gemm * 1e-3) / 1e12,
-                     "GBps": gemm_bytes / (ms_gemm * 1e-3) / 1e9},
+            "note": "measured one after the other in a second loop of the same length (medians); ms_serial is their sum as timed",
+            "ms_serial": res["ms_serial"], "clocks": res["clocks_phases"],
+            "quantize_act": {"ms": res["ms_act"], "GBps": act_quant_algorithmic_bytes(wl) / (res["ms_act"] * 1e-3) / 1e9,
+                             "frac_hbm": act_quant_algorithmic_bytes(wl) / (res["ms_act"] * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+            "quantize_pack_weights": {"ms": res["ms_w"],
+                                      "GBps": weight_quant_algorithmic_bytes(wl) / (res["ms_w"] * 1e-3) / 1e9,
+                                      "frac_hbm": weight_quant_algorithmic_bytes(wl) / (res["ms_w"] * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+            "gemm": {"ms": ms_gemm_job, "TOPS": ops / (res["ms_gemm"] * 1e-3) / 1e12,
+                     "GBps": gemm_bytes / (res["ms_gemm"] * 1e-3) / 1e9},
         },
     }
+    if "ms_step_warm" in res:
+        line["phases"]["warm"] = {"ms_step": res["ms_step_warm"], "ms_gemm": res["ms_gemm_warm"],
+                                  "note": "same graphs replayed back to back without the L2 flush"}
+    if small is not None:
+        wl2, r2 = small
+        ops2 = gemm_ops(wl2)
+        b2 = gemm_algorithmic_bytes(wl2, out_bytes)
+        roof2 = gemm_roofline_block(wl2, r2, peaks, peak_kind, out_bytes, probe_tops, probe_cycles, r2["ms_gemm"])
+        line["small_m"] = {
+            "workload": wl2.name, "config_index": 2, "M": wl2.M, "linears": r2["linears"],
+            "gemm_launches": r2["gemm_launches"], "bits_per_layer": list(wl2.bits),
+            "cold": {"l2": l2_note, "ms_step": r2["ms_step"], "ms_gemm": r2["ms_gemm"],
+                     "ms_quantize_act": r2["ms_act"], "ms_quantize_pack_weights": r2["ms_w"],
+                     "TOPS": ops2 / (r2["ms_step"] * 1e-3) / 1e12,
+                     "gemm_GBps": b2 / (r2["ms_gemm"] * 1e-3) / 1e9,
+                     "hbm_frac": b2 / (r2["ms_gemm"] * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+            "warm": {"l2": "no flush: replays back to back, the stack's 50 MB of codes and outputs stay in L2",
+                     "ms_step": r2["ms_step_warm"], "ms_gemm": r2["ms_gemm_warm"],
+                     "gemm_GBps": b2 / (r2["ms_gemm_warm"] * 1e-3) / 1e9,
+                     "hbm_frac": b2 / (r2["ms_gemm_warm"] * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+            "roofline": roof2, "clocks": r2["clocks"],
+        }
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(wl, args)
     print(json.dumps(line))
@@ -483,7 +587,8 @@ def run_ours(args, wl):
 
 
 def cpu_baseline(wl, args):
-    """The oracle, as it stands, on the host cores, on a bounded sample of the same workload."""
+    """The oracle, as it stands, on the host cores, on a bounded sample of the same workload: all cores
+    (the OpenMP build of the same source) and, on a smaller sample, one thread (the parity build)."""
     import oracle
     oracle.build()
     m_sample = min(wl.M, args.ref_rows)
@@ -501,9 +606,18 @@ def cpu_baseline(wl, args):
             oracle.linear(x, w, b, bits, s.groups, omp=True)
         reps += 1
     dt = (time.perf_counter() - t0) / reps
+    # one thread: the first 16 token rows of the same linears, once
+    m1 = min(m_sample, 16)
+    t1 = time.perf_counter()
+    for x, w, b, bits, s in data:
+        oracle.linear(x[:m1], w, b, bits, s.groups, omp=False)
+    dt1 = time.perf_counter() - t1
+    ops1 = sum(2.0 * m1 * s.N * s.K for *_, s in data)
     return {"value": ops / dt / 1e12, "unit": UNIT, "cores": oracle.num_threads(omp=True), "kind": "oracle",
             "sample": f"first layer ({len(data)} linears), first {m_sample} of {wl.M} token rows, whole path, "
-                      f"{reps} repetitions, {dt * 1e3:.1f} ms each"}
+                      f"{reps} repetitions, {dt * 1e3:.1f} ms each",
+            "single_thread": {"value": ops1 / dt1 / 1e12, "unit": UNIT, "cores": 1,
+                              "sample": f"same linears, first {m1} token rows, once, {dt1 * 1e3:.1f} ms"}}
 
 
 def run_quantizer_sweep(args):
@@ -674,13 +788,18 @@ def run_quantizer_sweep(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
-    ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--config", type=int, default=1, help="workload index 0-3 (see synth.workload); 4 = quantizer sweep")
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=3,
+                    help="workload index 0-3 (see synth.workload; default: the BERT-large stack, the largest single-GPU "
+                         "workload); 4 = quantizer sweep")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--ref-rows", type=int, default=256, help="token rows of the oracle's bounded sample")
     ap.add_argument("--ref-steps", type=int, default=5)
-    ap.add_argument("--e2e-steps", type=int, default=20)
+    ap.add_argument("--e2e-steps", type=int, default=None,
+                    help="steps of the end-to-end loop (default: 3 for the BERT-large stack, whose step moves 38 GB over the "
+                         "host link, else 20)")
+    ap.add_argument("--no-small-m", action="store_true", help="skip the small-M stack measured beside the main workload")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--out", default="f32", choices=["f32", "bf16"],
                     help="output type of the GEMMs: fp32 (the graded path) or bfloat16 (qb_layer_linears_bf16)")
@@ -696,6 +815,8 @@ def main():
         run_quantizer_sweep(args)
         return
     wl = synth.workload(args.config)
+    if args.e2e_steps is None:
+        args.e2e_steps = 3 if args.config == 3 else 20
     if args.impl == "reference":
         run_reference(args, wl)
     else:

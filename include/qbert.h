@@ -229,6 +229,15 @@ qb_status qb_layer_linears(const qb_linear_desc* descs /*host*/, int32_t count, 
                            size_t ws_bytes, void* cuda_stream);
 
 /*
+ * How many GEMM kernel launches qb_layer_linears (and its narrow-output forms) issue for this stack: host
+ * arithmetic on the descriptors only (bit widths, shapes), no GPU work.  (No counterpart in the paper; it
+ * lets a caller that counts or budgets launches, e.g. a benchmark, ask the library instead of guessing.)
+ *   descs   host array of `count` descriptors; only M, N, K and bits are read
+ * Returns 0 for a null or empty stack.
+ */
+int32_t qb_layer_linears_launch_count(const qb_linear_desc* descs /*host*/, int32_t count);
+
+/*
  * Narrow-output forms of qb_gemm and qb_layer_linears.  The paper keeps the activations between
  * layers at 8 bits (Table 1 caption: every quantized model uses 8-bit activations), so the fp32
  * result of a linear is an intermediate that the next operation narrows again; writing it as
@@ -367,6 +376,19 @@ qb_status qb_sensitivity_bits(const double* lambda, int32_t layers, int32_t samp
  * Synchronizes the device.  Returns QB_ERR_TIMEOUT if a bounded wait expired.
  */
 qb_status qb_probe_i8_mma(int32_t tokens, int32_t k_blocks, double* tops_out, double* cycles_per_kblock_out);
+
+/*
+ * Self-test of the bounded waits.  (No counterpart in the paper: every wait of the GEMM kernels on an
+ * mbarrier is bounded so that a fault elsewhere cannot hang the GPU; this call shows the bound working.)
+ * One small kernel waits, with the GEMM's own wait routines, on a barrier at which nothing ever arrives.
+ * After `limit_cycles` SM cycles (1e3 .. 2e9; 2e6 is about a millisecond) the waits give up, the kernel
+ * records QB_ERR_TIMEOUT in the status word of `ws` and returns normally; the context stays usable.
+ *   ws                 dev, >= 256 bytes: its status word receives QB_ERR_TIMEOUT (sticky, as everywhere)
+ *   waited_cycles_out  dev uint64 [2] or NULL: cycles each of the two waiting warps spent before giving up
+ * Enqueued on `cuda_stream`; read the outcome with qb_read_status.
+ */
+qb_status qb_probe_wait_limit(void* ws, size_t ws_bytes, int64_t limit_cycles, uint64_t* waited_cycles_out,
+                              void* cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -32,7 +32,7 @@ EXPORTS = (
     "qb_layer_linears", "qb_quantize_pack_weights_noalloc", "qb_probe_i8_mma", "qb_quantize_act_batch",
     "qb_quantize_pack_weights_batch", "qb_gemm_bf16", "qb_layer_linears_bf16",
     "qb_fake_quantize_weights", "qb_ste_backward", "qb_quantize_embedding", "qb_embedding_lookup",
-    "qb_gemm_i8", "qb_rowsum_i8", "qb_layer_linears_i8", "qb_sensitivity_bits",
+    "qb_gemm_i8", "qb_rowsum_i8", "qb_layer_linears_i8", "qb_sensitivity_bits", "qb_probe_wait_limit", "qb_layer_linears_launch_count",
 )
 NOALLOC_MAX_GROUPS = 4096
 
@@ -101,6 +101,10 @@ def lib() -> ctypes.CDLL:
     L.qb_quantize_pack_weights_noalloc.restype = i32
     L.qb_probe_i8_mma.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
     L.qb_probe_i8_mma.restype = i32
+    L.qb_layer_linears_launch_count.argtypes = [ctypes.POINTER(LinearDescC), i32]
+    L.qb_layer_linears_launch_count.restype = i32
+    L.qb_probe_wait_limit.argtypes = [vp, sz, i64, vp, vp]
+    L.qb_probe_wait_limit.restype = i32
     L.qb_sensitivity_bits.argtypes = [vp, i32, i32, vp, i32, vp, vp, vp]
     L.qb_sensitivity_bits.restype = i32
     L.qb_quantize_act_batch.argtypes = [ctypes.POINTER(ActDescC), i32, vp, sz, vp]
@@ -314,6 +318,14 @@ def probe_i8_mma(tokens: int = 256, k_blocks: int = 20000):
     return tops.value, cyc.value
 
 
+def probe_wait_limit(ws: torch.Tensor, limit_cycles: int = 2_000_000) -> torch.Tensor:
+    """``qb_probe_wait_limit``: a bounded wait that must run out; returns the cycles the two warps waited."""
+    waited = torch.zeros(2, dtype=torch.int64, device=ws.device)
+    _check(lib().qb_probe_wait_limit(ws.data_ptr(), ws.numel(), limit_cycles, waited.data_ptr(), _stream()),
+           "qb_probe_wait_limit")
+    return waited
+
+
 def sensitivity_bits(lam, budget_bits, reverse: bool = False):
     """``qb_sensitivity_bits`` (host only): ``lam`` [layers, samples] eigenvalue samples, ``budget_bits`` the bit
     width for each rank of the descending Omega order.  Returns (omega f64 [L], order i32 [L], bits i32 [L])."""
@@ -415,6 +427,12 @@ def layer_linears(descs, ws: torch.Tensor) -> None:
     """``qb_layer_linears`` over a list of ``LinearDesc`` (or an array from ``make_desc_array``)."""
     arr = descs if isinstance(descs, ctypes.Array) else make_desc_array(descs)
     _check(lib().qb_layer_linears(arr, len(arr), ws.data_ptr(), ws.numel(), _stream()), "qb_layer_linears")
+
+
+def layer_linears_launch_count(descs) -> int:
+    """``qb_layer_linears_launch_count``: GEMM kernel launches ``layer_linears`` issues for this stack."""
+    arr = descs if isinstance(descs, ctypes.Array) else make_desc_array(descs)
+    return int(lib().qb_layer_linears_launch_count(arr, len(arr)))
 
 
 def layer_linears_i8(descs: Sequence[LinearDesc], out_scales: Sequence[torch.Tensor], ws: torch.Tensor) -> None:

@@ -37,6 +37,7 @@
 #include <vector>
 
 #include "common.cuh"
+#include "mbar_wait.cuh"
 #include "ptx.cuh"
 
 namespace qb {
@@ -49,7 +50,6 @@ constexpr int kGemmThreads = kEpilogueThread0 + 32 * kEpilogueWarps;
 constexpr int kTileN = 128;          // output neurons per tile (MMA M)
 constexpr int kBlockK = 128;         // K elements (= bytes) per pipeline stage
 constexpr int kWBytes = kTileN * kBlockK;
-constexpr long long kWaitLimitCycles = 4000000000ll;  // about 2 s at 2 GHz
 
 constexpr int kMaxProblems = 16;
 constexpr int kMaxOrder = 4096;   // entries of the explicit tile visiting order (when it is used)
@@ -88,57 +88,20 @@ struct GroupedParams {
   uint16_t order[kMaxOrder];
 };
 
-template <int BT>
+// BT: tokens per tile (the N of the MMA).  CG: CTAs that share one MMA (1, or 2 = a CTA pair of a cluster:
+// the tile is then 256 neurons x BT tokens, each CTA expands its own 128 weight rows, loads its own half
+// of the token tile and drains its own half of the accumulator).
+template <int BT, int CG>
 struct GemmCfg {
-  static constexpr int kXBytes = BT * kBlockK;
+  static constexpr int kXRows = BT / CG;             // token rows this CTA stages per K block
+  static constexpr int kXBytes = kXRows * kBlockK;
   static constexpr int kStageBytes = kWBytes + kXBytes;
-  static constexpr int kStages = (BT == 256) ? 3 : 5;
+  static constexpr int kStages = (kStageBytes == 48 * 1024) ? 3 : 5;
   static constexpr int kTmemCols = 2 * BT;
   static constexpr int kBarBytes = 256 + 2 * 256 * 4;  // barriers + two row-sum tiles
   static constexpr int kOutStageBytes = kEpilogueWarps * 2 * 32 * 32 * 4;  // per epilogue warp: two buffers of 32 tokens x 32 neurons fp32
   static constexpr int kSmemBytes = kStages * kStageBytes + kOutStageBytes + kBarBytes;
 };
-
-// Bounded wait on an mbarrier phase.  Returns false if the wait expired or another role aborted.
-// The bound is counted in SM clock cycles (clock64 is a cheap register read; the global nanosecond
-// timer costs about a microsecond per read and would dominate short waits).
-// kSleep: the waiter is not on the critical path (it runs several stages ahead) and must not compete
-// for issue slots with the MMA issuer that shares its scheduler: it uses the form of try_wait that
-// takes a suspend-time hint.  A warp that polls in a tight loop is always "ready", and a handful of
-// them starve the one thread that feeds the tensor cores.
-template <bool kSleep>
-__device__ __forceinline__ bool wait_barrier_t(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  if (ptx::mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  for (uint32_t spin = 1;; ++spin) {
-    if (kSleep) {
-      // suspended by the hardware until the phase completes or about a microsecond has passed: no issue
-      // slots are spent while waiting and the wake-up does not wait for a sleep interval to end
-      if (ptx::mbar_try_wait_suspend(bar, parity, 1000u)) return true;
-    } else {
-      if (ptx::mbar_try_wait(bar, parity)) return true;
-    }
-    if ((spin & 63u) == 0u) {
-      if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitLimitCycles) return false;
-    }
-  }
-}
-__device__ __forceinline__ bool wait_barrier(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  return wait_barrier_t<false>(bar, parity, abort_flag);
-}
-__device__ __forceinline__ bool wait_barrier_relaxed(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  return wait_barrier_t<true>(bar, parity, abort_flag);
-}
-
-// Whole-warp wait: only lane 0 polls the barrier (hundreds of threads polling the same shared-memory
-// word would flood the shared-memory pipeline that the stores and the other roles' waits also use);
-// the outcome is broadcast, and the shuffle orders the other lanes' later accesses after the wait.
-__device__ __forceinline__ bool wait_barrier_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  int ok = 1;
-  if ((threadIdx.x & 31) == 0) ok = wait_barrier_relaxed(bar, parity, abort_flag) ? 1 : 0;
-  return __shfl_sync(0xffffffffu, ok, 0) != 0;
-}
 
 // Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes, groups of
 // 8 rows 1024 bytes apart.  Fields: start address >> 4 (bits 0-13), leading byte offset >> 4 (16-29,
@@ -228,20 +191,24 @@ __device__ __forceinline__ void load_item(const uint32_t* __restrict__ src, uint
   }
 }
 
-// A role's walk over the tiles of its CTA: positions blockIdx.x, + gridDim.x, ... of the visiting order.
+// A role's walk over the tiles of its CTA (or CTA pair): positions g, g + G, ... of the visiting order, g the
+// index of the CTA group and G their number.
 struct TileCursor {
   int p;   // position
   int t;   // tile at that position
   int pi;  // problem that owns tile t
-  __device__ __forceinline__ void start() {
-    p = (int)blockIdx.x - (int)gridDim.x;
+  int stride;  // CTA groups in the launch
+  // `cg`: CTAs per group (1 or 2); the CTAs of a group walk the same tiles
+  __device__ __forceinline__ void start(int cg = 1) {
+    stride = (int)gridDim.x / cg;
+    p = (int)blockIdx.x / cg - stride;
     t = 0;
     pi = 0;
   }
   // move to the CTA's next tile; false when there is none
   __device__ __forceinline__ bool next(const GroupedParams& gp) {
     for (;;) {
-      p += (int)gridDim.x;
+      p += stride;
       if (p >= gp.total_positions) return false;
       if (!gp.use_order) {
         t = p;
@@ -972,19 +939,20 @@ static qb_status side_streams(SideStreams** out) {
 // total) runs its launches side by side, each on a share of the SMs in proportion to its work, so that
 // the start-up and the drain of the pipelines overlap instead of adding up; the launches join the
 // caller's stream before the call returns.  Large stacks keep one launch after the other on all SMs.
-static qb_status launch_stack(const qb_linear_desc* d, int count, void* ws, int sm_count, cudaStream_t stream,
-                              int out, const float* const* out_scales = nullptr) {
-  std::vector<int> order(count);
+struct StackGroup {
+  int begin, count;
+  int64_t tiles, cost;
+};
+// The launches of a stack: `order` lists the descriptors by bit width, then longest K first; every group
+// is a run of `order` that one launch serves.
+static void plan_stack(const qb_linear_desc* d, int count, std::vector<int>& order, std::vector<StackGroup>& groups,
+                       int64_t* all_tiles_out, int64_t* all_cost_out) {
+  order.resize(count);
   for (int i = 0; i < count; ++i) order[i] = i;
   std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
     if (d[a].bits != d[b].bits) return d[a].bits < d[b].bits;
     return d[a].K > d[b].K;
   });
-  struct Group {
-    int begin, count;
-    int64_t tiles, cost;
-  };
-  std::vector<Group> groups;
   int64_t all_tiles = 0, all_cost = 0;
   int i = 0;
   while (i < count) {
@@ -1006,6 +974,17 @@ static qb_status launch_stack(const qb_linear_desc* d, int count, void* ws, int 
     all_cost += cost;
     i = j;
   }
+  if (all_tiles_out) *all_tiles_out = all_tiles;
+  if (all_cost_out) *all_cost_out = all_cost;
+}
+
+static qb_status launch_stack(const qb_linear_desc* d, int count, void* ws, int sm_count, cudaStream_t stream,
+                              int out, const float* const* out_scales = nullptr) {
+  std::vector<int> order;
+  std::vector<StackGroup> groups;
+  int64_t all_tiles = 0, all_cost = 0;
+  plan_stack(d, count, order, groups, &all_tiles, &all_cost);
+  using Group = StackGroup;
   const int n_groups = (int)groups.size();
   const bool side_by_side = n_groups > 1 && n_groups <= kMaxSide + 1 && n_groups <= sm_count &&
                             all_tiles < (int64_t)16 * sm_count;
@@ -1178,6 +1157,14 @@ extern "C" qb_status qb_rowsum_i8(const int8_t* xq, int64_t M, int64_t K, int32_
                                                                                 K / 16, rowsum);
   QB_CUDA_TRY(cudaGetLastError());
   return QB_OK;
+}
+
+extern "C" int32_t qb_layer_linears_launch_count(const qb_linear_desc* descs, int32_t count) {
+  if (!descs || count <= 0) return 0;
+  std::vector<int> order;
+  std::vector<qb::StackGroup> groups;
+  qb::plan_stack(descs, count, order, groups, nullptr, nullptr);
+  return (int32_t)groups.size();
 }
 
 extern "C" qb_status qb_layer_linears(const qb_linear_desc* descs, int32_t count, void* ws, size_t ws_bytes,

@@ -3,6 +3,7 @@
 // It is the denominator against which qb_gemm's tensor-bound shapes are read: the GEMM cannot beat
 // the rate at which the instruction itself retires.
 #include "common.cuh"
+#include "mbar_wait.cuh"
 #include "ptx.cuh"
 
 namespace qb {
@@ -116,5 +117,59 @@ extern "C" qb_status qb_probe_i8_mma(int32_t tokens, int32_t k_blocks, double* t
   const double ops = 2.0 * 128.0 * tokens * 128.0 * (double)k_blocks * sms;
   *tops_out = ops / (ms * 1e-3) / 1e12;
   if (cycles_per_kblock_out) *cycles_per_kblock_out = (double)worst / k_blocks;
+  return QB_OK;
+}
+
+// qb_probe_wait_limit: the self-test of the bounded waits.  One CTA initialises an mbarrier that nothing
+// ever arrives at and waits on it with the GEMM's own wait helpers (the single-thread form and the
+// whole-warp form) under a short limit.  The waits must give up after `limit_cycles`, record
+// QB_ERR_TIMEOUT in the workspace's status word exactly as the GEMM roles do, and the kernel must leave
+// through its normal exit.  Nothing here can hang: the wait is the bounded one under test, and its
+// loop ends on the cycle count alone.
+namespace qb {
+__global__ void __launch_bounds__(64, 1) probe_wait_limit_kernel(void* ws, long long limit_cycles,
+                                                                 unsigned long long* waited_out) {
+  __shared__ __align__(8) unsigned long long bar_storage;
+  __shared__ int abort_flag;
+  const uint32_t bar = ptx::smem_u32(&bar_storage);
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(bar, 1);  // one arrival expected; none will come
+    abort_flag = 0;
+    ptx::fence_mbar_init();
+  }
+  __syncthreads();
+  const long long t0 = clock64();
+  bool ok;
+  if (threadIdx.x < 32) {
+    ok = true;
+    if (threadIdx.x == 0) ok = wait_barrier(bar, 0, &abort_flag, limit_cycles);  // the MMA issuer's form
+    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+  } else {
+    ok = wait_barrier_warp(bar, 0, &abort_flag, limit_cycles);                    // the other roles' form
+  }
+  const long long waited = clock64() - t0;
+  if (!ok && (threadIdx.x & 31) == 0) {
+    report_status(ws, QB_ERR_TIMEOUT, (9 << 16) | (int)(threadIdx.x >> 5));
+    if (waited_out) waited_out[threadIdx.x >> 5] = (unsigned long long)waited;
+  }
+}
+}  // namespace qb
+
+extern "C" qb_status qb_probe_wait_limit(void* ws, size_t ws_bytes, int64_t limit_cycles, uint64_t* waited_cycles_out,
+                                         void* cuda_stream) {
+  if (!ws || ws_bytes < qb::kWsMinBytes) {
+    qb::set_last_error("qb_probe_wait_limit: workspace null or too small");
+    return QB_ERR_WORKSPACE;
+  }
+  if (limit_cycles < 1000 || limit_cycles > 2000000000ll) {
+    qb::set_last_error("qb_probe_wait_limit: limit_cycles must be in [1e3, 2e9]");
+    return QB_ERR_INVALID;
+  }
+  int sms = 0;
+  qb_status st = qb::require_sm100(&sms);
+  if (st != QB_OK) return st;
+  qb::probe_wait_limit_kernel<<<1, 64, 0, (cudaStream_t)cuda_stream>>>(ws, (long long)limit_cycles,
+                                                                       reinterpret_cast<unsigned long long*>(waited_cycles_out));
+  QB_CUDA_TRY(cudaGetLastError());
   return QB_OK;
 }
