@@ -33,6 +33,8 @@
 #include <cuda_bf16.h>
 
 #include <algorithm>
+#include <atomic>
+#include <cstdlib>
 #include <cstring>
 #include <vector>
 
@@ -42,11 +44,29 @@
 
 namespace qb {
 
+#ifndef QB_LOAD_AFTER
+#define QB_LOAD_AFTER 1
+#endif
+// Roles sit on warpgroup boundaries (four consecutive warps) so that registers can be moved between them
+// with setmaxnreg: warpgroup 0 holds the two single-thread roles (and two idle warps) and gives its
+// registers away, warpgroups 1-3 are the expander teams, warpgroups 4-5 the epilogue.
 constexpr int kExpandTeams = 3;     // teams of 128 expander threads
 constexpr int kEpilogueWarps = 8;
-constexpr int kFirstEpilogueWarp = 2 + 4 * kExpandTeams;
+constexpr int kFirstExpandWarp = 4;
+constexpr int kFirstEpilogueWarp = kFirstExpandWarp + 4 * kExpandTeams;
 constexpr int kEpilogueThread0 = 32 * kFirstEpilogueWarp;
 constexpr int kGemmThreads = kEpilogueThread0 + 32 * kEpilogueWarps;
+// Registers per thread: the launch gives every thread kRegsLaunch (65,536 / 768 rounded down to a multiple
+// of 8); the shares below add up to at most kGemmThreads * kRegsLaunch, which setmaxnreg.inc needs in order
+// not to wait forever.
+constexpr int kRegsLaunch = 80;
+constexpr int kRegsLight = 56;      // producer / issuer warpgroup
+constexpr int kRegsExpand = 72;
+constexpr int kRegsEpilogue = 104;
+static_assert(128 * kRegsLight + 128 * kExpandTeams * kRegsExpand + 32 * kEpilogueWarps * kRegsEpilogue <=
+                  kGemmThreads * kRegsLaunch,
+              "register shares exceed what the launch allocates");
+static_assert(kGemmThreads * kRegsLaunch <= 65536, "launch allocation exceeds the register file");
 constexpr int kTileN = 128;          // output neurons per tile (MMA M)
 constexpr int kBlockK = 128;         // K elements (= bytes) per pipeline stage
 constexpr int kWBytes = kTileN * kBlockK;
@@ -226,15 +246,31 @@ struct TileCursor {
   }
 };
 
+// Barrier over the epilogue warps (named barrier 1) that also ORs a predicate over them.
+__device__ __forceinline__ bool epilogue_sync_or(bool pred) {
+  uint32_t res;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.or.pred p, 1, %2, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(res)
+      : "r"((uint32_t)pred), "n"(32 * kEpilogueWarps)
+      : "memory");
+  return res != 0;
+}
+
 // OUT selects what the epilogue writes: the fp32 result; that result rounded to bfloat16 (round to nearest
 // even), Y bfloat16 [M][N]; or that result re-quantized to the 8-bit activation grid of step *out_scale,
 // clamp(round_half_even(y * (1 / out_scale)), -127, 127), Y int8 [M][N].
 enum { kOutF32 = 0, kOutBf16 = 1, kOutI8 = 2 };
-template <int BT, int BITS, int OUT>
+template <int BT, int BITS, int OUT, int CG>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
-  using Cfg = GemmCfg<BT>;
+  using Cfg = GemmCfg<BT, CG>;
   constexpr int kStages = Cfg::kStages;
+  // CG == 2: this CTA's rank in its pair (rank 0 issues the MMAs for both and owns the barriers the issuer
+  // waits on); the pair's tile is 2 * kTileN neurons x BT tokens, rank r owns neurons 128 r .. 128 r + 127
+  // and stages token rows (BT / 2) r .. of the tile
+  const uint32_t cta_rank = CG == 2 ? ptx::cluster_ctarank() : 0u;
+  constexpr int kGroupN = kTileN * CG;  // neurons per tile of the CTA group
   // 128-byte swizzle patterns repeat every 1024 bytes: stage bases must be 1024-byte aligned.  The
   // kernel has no static shared memory, so the dynamic segment starts at offset 0 of the CTA's window.
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -265,29 +301,38 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
-      ptx::mbar_init(full(s), 1 + 4);
+      ptx::mbar_init(full(s), 1 + 4 * CG);  // the producer's expect-tx arrival + the expander warps of every CTA of the group
       ptx::mbar_init(empty(s), 1);
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(acc_full(a), 1);
-      ptx::mbar_init(acc_empty(a), kEpilogueWarps);  // one arrival per epilogue warp
+      ptx::mbar_init(acc_empty(a), kEpilogueWarps * CG);  // one arrival per epilogue warp of the group
     }
     ptx::mbar_init(drain_bar, 1);
     *abort_flag = 0;
     ptx::fence_mbar_init();
   }
   if (warp == 1) {
-    ptx::tmem_alloc(ptx::smem_u32(tmem_slot), Cfg::kTmemCols);
-    ptx::tmem_relinquish_alloc_permit();
+    ptx::tmem_alloc_cg<CG>(ptx::smem_u32(tmem_slot), Cfg::kTmemCols);
+    ptx::tmem_relinquish_cg<CG>();
   }
   ptx::tcgen05_fence_before_sync();
   __syncthreads();
+  // a pair: no arrival or copy may reach the other CTA's barriers before it has initialised them
+  if constexpr (CG == 2) ptx::cluster_sync_all();
   ptx::tcgen05_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  // the barriers the MMA issuer waits on live in the group's first CTA
+  auto full_lead = [&](int s) { return CG == 2 ? ptx::map_to_cta(full(s), 0) : full(s); };
+  auto acc_empty_lead = [&](int a) { return CG == 2 ? ptx::map_to_cta(acc_empty(a), 0) : acc_empty(a); };
 
   bool timed_out = false;
   int where = 0;
 
+  // Each warpgroup first sets its register share: the light warpgroup (and the expanders, a little) hand
+  // registers to the epilogue warps.
+  if (warp < kFirstExpandWarp) {
+  ptx::setmaxnreg_dec<kRegsLight>();
   if (warp == 0) {
     // ---------------- TMA producer: token tiles -------------------------------------------------
     if (ptx::elect_one()) {
@@ -298,16 +343,18 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
       // CTA's next tile when the current one ends) so that the loads themselves hit L2.
       constexpr int kL2Ahead = 8;
       TileCursor c;
-      c.start();
+      c.start(CG);
       bool have = c.next(gp);
+      constexpr int kMyRow0 = 0;
+      const int row_off = (int)cta_rank * Cfg::kXRows + kMyRow0;  // this CTA's rows inside the token tile
       if (have) {
         const Problem& pr = gp.prob[c.pi];
-        const int m0 = ((c.t - pr.tile_begin) / pr.n_tiles) * BT;
+        const int m0 = ((c.t - pr.tile_begin) / pr.n_tiles) * BT + row_off;
         for (int kb = 0; kb < kL2Ahead && kb < pr.K / kBlockK; ++kb) ptx::tma_prefetch_l2_2d(&gp.tmx[c.pi], kb * kBlockK, m0);
       }
       while (have && !timed_out) {
         const Problem& pr = gp.prob[c.pi];
-        const int m0 = ((c.t - pr.tile_begin) / pr.n_tiles) * BT;
+        const int m0 = ((c.t - pr.tile_begin) / pr.n_tiles) * BT + row_off;
         const int k_blocks = pr.K / kBlockK;
         const CUtensorMap* tm = &gp.tmx[c.pi];
         // the CTA's next tile, for prefetches that run past the end of this one
@@ -318,7 +365,7 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
         if (have_nx) {
           const Problem& pn = gp.prob[nx.pi];
           tm_nx = &gp.tmx[nx.pi];
-          m0_nx = ((nx.t - pn.tile_begin) / pn.n_tiles) * BT;
+          m0_nx = ((nx.t - pn.tile_begin) / pn.n_tiles) * BT + row_off;
           kblocks_nx = pn.K / kBlockK;
         }
         for (int kb = 0; kb < k_blocks; ++kb) {
@@ -333,8 +380,14 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
             where = (0 << 16) | stage;
             break;
           }
-          ptx::mbar_arrive_expect_tx(full(stage), Cfg::kXBytes);
-          ptx::tma_load_2d(stage_x(stage), tm, full(stage), kb * kBlockK, m0);
+          if constexpr (CG == 2) {
+            // the first CTA announces the bytes of both halves; each CTA's copy completes on that barrier
+            if (cta_rank == 0) ptx::mbar_arrive_expect_tx(full(stage), CG * Cfg::kXBytes);
+            ptx::tma_load_2d_pair(stage_x(stage), tm, full_lead(stage), kb * kBlockK, m0);
+          } else {
+            ptx::mbar_arrive_expect_tx(full(stage), Cfg::kXBytes);
+            ptx::tma_load_2d(stage_x(stage), tm, full(stage), kb * kBlockK, m0);
+          }
           if (++stage == kStages) {
             stage = 0;
             phase ^= 1u;
@@ -351,13 +404,13 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
       }
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer ----------------------------------------------------------------
-    if (ptx::elect_one()) {
+    // ---------------- MMA issuer (of a pair: in its first CTA only) -------------------------------
+    if (cta_rank == 0 && ptx::elect_one()) {
       // This one thread must issue a K block's work in well under the 512 cycles the tensor cores need
       // for it, and every instruction here is long-latency and serial.  So: one barrier wait per K
       // block, and the loop is unrolled over the ring so that barrier addresses and both operand
       // descriptors of a stage are compile-time offsets from loop-invariant values.
-      constexpr uint32_t idesc = make_idesc_i8(kTileN, BT);
+      constexpr uint32_t idesc = make_idesc_i8(kGroupN, BT);
       const uint64_t a_desc0 = make_kmajor_sw128_desc(stage_w(0));
       const uint64_t b_desc0 = make_kmajor_sw128_desc(stage_x(0));
       constexpr uint32_t kStageDescStep = Cfg::kStageBytes >> 4;  // start-address field counts 16-byte units
@@ -365,7 +418,7 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
       int it = 0, kb = 0, k_blocks = 0, a = 0;
       uint32_t d_tmem = 0;
       TileCursor c;
-      c.start();
+      c.start(CG);
       bool active = c.next(gp);
       while (active) {
 #pragma unroll
@@ -393,10 +446,10 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
               const uint64_t b_desc = b_desc0 + (uint64_t)(stage * kStageDescStep);
 #pragma unroll
               for (int j = 0; j < kBlockK / 32; ++j)  // 32 bytes of K per instruction: +2 in the address field
-                ptx::mma_i8_ss(d_tmem, a_desc + 2u * j, b_desc + 2u * j, idesc, j != 0 ? 1u : (kb != 0 ? 1u : 0u));
-              ptx::mma_commit(empty(stage));
+                ptx::mma_i8_ss_cg<CG>(d_tmem, a_desc + 2u * j, b_desc + 2u * j, idesc, j != 0 ? 1u : (kb != 0 ? 1u : 0u));
+              ptx::mma_commit_cg<CG>(empty(stage));
               if (++kb == k_blocks) {  // tile done: hand the accumulator to the epilogue
-                ptx::mma_commit(acc_full(a));
+                ptx::mma_commit_cg<CG>(acc_full(a));
                 kb = 0;
                 ++it;
                 active = c.next(gp);
@@ -408,25 +461,28 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
       }
       if (timed_out) {
         // wait (bounded) for the MMAs already issued before tensor memory is freed
-        ptx::mma_commit(drain_bar);
+        ptx::mma_commit_cg<CG>(drain_bar);
         const long long t0 = clock64();
         while (!ptx::mbar_try_wait(drain_bar, 0) && clock64() - t0 < 400000000ll) {
         }
       }
     }
+  }
+  // (warps 2 and 3 of warpgroup 0 have nothing to do but to give their registers away)
   } else if (warp < kFirstEpilogueWarp) {
+    ptx::setmaxnreg_dec<kRegsExpand>();
     // ---------------- weight expanders ------------------------------------------------------------
     // A K block of the tile is 128 rows x 4 items of 32 codes.  Thread i of a team takes items
     // i, i+128, i+256, i+384: piece i%4 of rows i/4 + 32j.  Four neighbouring lanes read one row's
     // 16*BITS contiguous bytes, so a warp-wide load touches 8 rows instead of 32.
     // The K blocks of all tiles of this CTA form one sequence; team g takes those with index g mod 3.
-    const int team = (warp - 2) >> 2;
-    const int i_team = (threadIdx.x - 64) & 127;
+    const int team = (warp - kFirstExpandWarp) >> 2;
+    const int i_team = (threadIdx.x - 32 * kFirstExpandWarp) & 127;
     const int piece = i_team & 3;
     const int row0 = i_team >> 2;
     // fetch cursor: tile, K block inside it, and the tile's weight rows
     TileCursor c;
-    c.start();
+    c.start(CG);
     int ld_kb = team;
     int ld_kblocks = 0, ld_n0 = 0, ld_N = 0, ld_wpr = 0;
     const uint32_t* ld_packed = nullptr;
@@ -434,7 +490,7 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
     auto enter_tile = [&]() {  // fields of the tile the cursor stands on
       const Problem& pr = gp.prob[c.pi];
       ld_kblocks = pr.K / kBlockK;
-      ld_n0 = ((c.t - pr.tile_begin) % pr.n_tiles) * kTileN;
+      ld_n0 = ((c.t - pr.tile_begin) % pr.n_tiles) * kGroupN + (int)cta_rank * kTileN;
       ld_N = pr.N;
       ld_wpr = pr.K / 32 * BITS;
       ld_packed = pr.packed;
@@ -488,7 +544,9 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
 #pragma unroll
         for (int i = 0; i < 4 * BITS; ++i) pre[d][i] = pre[d + 1][i];
       }
+#if !QB_LOAD_AFTER
       pre_valid[kPrefetch - 1] = load_next(pre[kPrefetch - 1]);
+#endif
       if (!wait_barrier_warp(empty(stage), phase ^ 1u, abort_flag)) {
         timed_out = true;
         where = (2 << 16) | stage;
@@ -507,7 +565,15 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
       }
       ptx::fence_proxy_async_smem();  // every lane: its own stores -> visible to the tensor cores
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(full(stage));
+      if (lane == 0) {
+        if (CG == 2 && cta_rank != 0) ptx::mbar_arrive_remote(full_lead(stage));
+        else ptx::mbar_arrive(full(stage));
+      }
+#if QB_LOAD_AFTER
+      // the next fetch goes out after the proxy fence, not before it: the fence waits for the thread's loads
+      // in flight, and a fetch issued first would put its whole latency into every K block
+      pre_valid[kPrefetch - 1] = load_next(pre[kPrefetch - 1]);
+#endif
       stage += kExpandTeams;
       if (stage >= kStages) {
         stage -= kStages;
@@ -515,112 +581,159 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
       }
     }
   } else {
+    ptx::setmaxnreg_inc<kRegsEpilogue>();
     // ---------------- epilogue --------------------------------------------------------------------
+    // Two warps per TMEM lane quarter; the warps of a quarter take alternate chunks of 32 tokens.  Per tile:
+    // wait for the accumulator, then for every chunk: tcgen05.ld, convert and two fused multiply-adds per
+    // output (two outputs per instruction), 32 x 32 tile into shared memory, one TMA store.  The accumulator is handed back to the issuer as soon as the warp's last
+    // chunk is in registers.  The next tile's dequantization constants and row sums are fetched while
+    // this tile drains.
+    const int ew = warp - kFirstEpilogueWarp;
     const int quarter = warp & 3;              // TMEM lanes this warp may access: 32*quarter ..
-    const int r = quarter * 32 + lane;         // output neuron inside the tile
+    const int half = ew >> 2;                  // which of the quarter's two warps
+    const int r = quarter * 32 + lane;         // output neuron inside the CTA's 128 rows
+    const int e = threadIdx.x - kEpilogueThread0;  // 0..255: the token whose row sum this thread stages
     constexpr int c_code = 1 << (BITS - 1);
-    int it = 0;
+    float* const warp_bufs = out_stage + ew * (2 * 32 * 32);
     int out_flip = 0;
+
+    // per-tile values: the tile being drained, and the CTA's next tile (prefetched)
+    struct TileVals {
+      int pi, n_base, m0;
+      float alpha, beta, b, rs;  // rs: row sum of token m0 + e (as fp32, exact), 0 past M
+    };
+    auto fetch = [&](const TileCursor& tc, TileVals& tv) {
+      const Problem& pr = gp.prob[tc.pi];
+      const int local = tc.t - pr.tile_begin;
+      tv.pi = tc.pi;
+      tv.n_base = (local % pr.n_tiles) * kGroupN + (int)cta_rank * kTileN;
+      tv.m0 = (local / pr.n_tiles) * BT;
+      const int n = tv.n_base + r;
+      tv.alpha = tv.beta = tv.b = 0.f;
+      if (n < pr.N) {
+        const float s_a = __ldg(pr.act_scale);
+        const int g = n / pr.rows_per_group;
+        const float dlt = __ldg(pr.delta + g);
+        const float z = __ldg(pr.q0 + g);
+        const float zc = __fmaf_rn(dlt, (float)c_code, z);
+        tv.alpha = __fmul_rn(s_a, dlt);
+        tv.beta = __fmul_rn(s_a, zc);
+        tv.b = pr.bias ? __ldg(pr.bias + n) : 0.0f;
+      }
+      tv.rs = (e < BT && tv.m0 + e < pr.M) ? (float)__ldg(pr.rowsum + tv.m0 + e) : 0.0f;  // exact: |rowsum| < 2^24
+    };
+
     TileCursor c;
-    c.start();
-    for (; !timed_out && c.next(gp); ++it) {
-      const Problem& pr = gp.prob[c.pi];
-      const CUtensorMap* tmy = &gp.tmy[c.pi];
-      const int local = c.t - pr.tile_begin;
+    c.start(CG);
+    bool have = c.next(gp);
+    TileVals cur;
+    if (have) {
+      fetch(c, cur);
+      if (e < BT) rs_tile[e] = cur.rs;  // accumulator 0's row sums; published by the barrier below
+    }
+    for (int it = 0; have; ++it) {
+      const Problem& pr = gp.prob[cur.pi];
+      const CUtensorMap* tmy = &gp.tmy[cur.pi];
       const int pM = pr.M, pN = pr.N;
       const int a = it & 1;
       const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
-      const int n_base = (local % pr.n_tiles) * kTileN;
+      const int n_base = cur.n_base, m0 = cur.m0;
       const int n = n_base + r;
-      const int m0 = (local / pr.n_tiles) * BT;
       const bool nvalid = n < pN;
       const bool tma_store = pr.tma_store != 0;
+      const float alpha = cur.alpha, beta = cur.beta, b = cur.b;
+      // alpha * 2^-(8-BITS), used when that scaling loses no bits in any lane of the warp
+      const float alpha_s = __fmul_rn(alpha, 1.0f / (float)(1 << (8 - BITS)));
+      const bool fold_shift = __all_sync(0xffffffffu, __fmul_rn(alpha_s, (float)(1 << (8 - BITS))) == alpha);
       float* const y_ptr = reinterpret_cast<float*>(pr.y);
       uint16_t* const y16_ptr = reinterpret_cast<uint16_t*>(pr.y);
       int8_t* const y8_ptr = reinterpret_cast<int8_t*>(pr.y);
       float out_inv = 0.0f;
       if constexpr (OUT == kOutI8) out_inv = __fdiv_rn(1.0f, __ldg(pr.out_scale));
       int32_t* const acc_ptr = pr.acc_out;
-      float alpha = 0.f, beta = 0.f, b = 0.f;
-      if (nvalid) {
-        const float s_a = __ldg(pr.act_scale);
-        const int g = n / pr.rows_per_group;
-        const float dlt = __ldg(pr.delta + g);
-        const float z = __ldg(pr.q0 + g);
-        const float zc = __fmaf_rn(dlt, (float)c_code, z);
-        alpha = __fmul_rn(s_a, dlt);
-        beta = __fmul_rn(s_a, zc);
-        b = pr.bias ? __ldg(pr.bias + n) : 0.0f;
-      }
-      // row sums of this tile's tokens -> shared memory (zero past M), visible to the epilogue warps
-      {
-        const int e = threadIdx.x - kEpilogueThread0;
-        if (e < BT)
-          rs_tile[a * 256 + e] = (m0 + e < pM) ? (float)__ldg(pr.rowsum + m0 + e) : 0.0f;  // exact: |rowsum| < 2^24
-        asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpilogueWarps) : "memory");
-      }
-      if (!wait_barrier_warp(acc_full(a), aphase, abort_flag)) {
+
+      const bool ok = wait_barrier_warp(acc_full(a), aphase, abort_flag);
+      // One barrier over the epilogue warps per tile: it publishes the row sums staged for this tile and
+      // makes the decision to give up the same in all eight warps (a warp that left alone would leave
+      // the others waiting at this barrier).
+      if (epilogue_sync_or(!ok)) {
         timed_out = true;
         where = (3 << 16) | a;
         break;
       }
       ptx::tcgen05_fence_after_sync();
+
+      // the CTA's next tile: its constants are fetched now and used after this tile's chunks
+      TileCursor nx = c;
+      const bool have_nx = nx.next(gp);
+      TileVals nxt;
+      if (have_nx) fetch(nx, nxt);
+
       const uint32_t t_base = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * BT);
       const int n_chunks = min(BT / 32, (pM - m0 + 31) / 32);  // chunks of 32 tokens, warp-uniform
-      float* const warp_bufs = out_stage + (warp - kFirstEpilogueWarp) * (2 * 32 * 32);
       const int x0 = n_base + quarter * 32;
-      // the two warps of a lane quarter take alternate chunks
-#pragma unroll 1
-      for (int ch = (warp - kFirstEpilogueWarp) >> 2; ch < n_chunks; ch += kEpilogueWarps / 4) {
-        uint32_t v[32];
-        ptx::tmem_ld_32x32b_x32(t_base + (uint32_t)(ch * 32), v);
-        ptx::tmem_ld_wait();
-        ptx::tmem_ld_regs_ready(v);
+      const float* const rs_a = rs_tile + a * 256;
+
+      auto release_acc = [&]() {  // this warp has read all it needs from the accumulator
+        ptx::tcgen05_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) {
+          if (CG == 2 && cta_rank != 0) ptx::mbar_arrive_remote(acc_empty_lead(a));
+          else ptx::mbar_arrive(acc_empty(a));
+        }
+      };
+      auto process = [&](uint32_t (&v)[32], int ch) {
         const int mc = m0 + ch * 32;
-        const float4* rs4 = reinterpret_cast<const float4*>(rs_tile + a * 256 + ch * 32);
+        const float4* rs4 = reinterpret_cast<const float4*>(rs_a + ch * 32);
         float* buf = warp_bufs + (out_flip & 1) * (32 * 32);  // alternate between the warp's two staging buffers
         ++out_flip;
         if (tma_store) {
           // 32 tokens x 32 neurons of this warp -> shared memory [token][neuron] -> one TMA store.
           // Lanes write consecutive words of a row: conflict-free.  Rows past M and neurons past N
-          // are clipped by the tensor map.  Loads, then arithmetic, then stores, in halves of 16
-          // tokens; the wait for the warp's previous store comes as late as possible.
+          // are clipped by the tensor map.  All 32 results are formed first (in the registers that held
+          // the accumulators), two per instruction: y = fma(alpha, (float)Ac, fma(beta, rowsum, b)) with
+          // Ac = v >> (8 - BITS).  When alpha * 2^-(8-BITS) is exact (always, short of underflow) the
+          // shift is folded into alpha: (float)v = 2^(8-BITS) * (float)Ac exactly, so the product, and
+          // with it the fused result, is the same real number rounded once.
+          float yv[32];
+          if (fold_shift) {
 #pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            float rsv[16], yv[16];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              const float4 rv = rs4[4 * h + q];  // same address in every lane: one broadcast read
-              rsv[4 * q] = rv.x;
-              rsv[4 * q + 1] = rv.y;
-              rsv[4 * q + 2] = rv.z;
-              rsv[4 * q + 3] = rv.w;
+            for (int q = 0; q < 8; ++q) {
+              const float4 rv = rs4[q];  // same address in every lane: one broadcast read
+              float t0, t1, t2, t3;
+              ptx::fma_f32x2(t0, t1, beta, beta, rv.x, rv.y, b, b);
+              ptx::fma_f32x2(t2, t3, beta, beta, rv.z, rv.w, b, b);
+              ptx::fma_f32x2(yv[4 * q], yv[4 * q + 1], alpha_s, alpha_s, (float)(int)v[4 * q], (float)(int)v[4 * q + 1], t0, t1);
+              ptx::fma_f32x2(yv[4 * q + 2], yv[4 * q + 3], alpha_s, alpha_s, (float)(int)v[4 * q + 2], (float)(int)v[4 * q + 3], t2, t3);
             }
+          } else {
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              const int ac = ((int)v[16 * h + j]) >> (8 - BITS);
-              yv[j] = __fmaf_rn(alpha, (float)ac, __fmaf_rn(beta, rsv[j], b));
-            }
-            if (h == 0) {
-              if (lane == 0) ptx::tma_store_wait_read1();  // the store before last (same buffer) has read it
-              __syncwarp();
-            }
-            if constexpr (OUT == kOutBf16) {  // rows of 32 bfloat16 (64 bytes): the first half of the fp32 buffer
-              uint16_t* buf16 = reinterpret_cast<uint16_t*>(buf);
+            for (int q = 0; q < 8; ++q) {
+              const float4 rv = rs4[q];
+              const float rsv[4] = {rv.x, rv.y, rv.z, rv.w};
 #pragma unroll
-              for (int j = 0; j < 16; ++j)
-                buf16[(16 * h + j) * 32 + lane] = __bfloat16_as_ushort(__float2bfloat16_rn(yv[j]));
-            } else if constexpr (OUT == kOutI8) {  // rows of 32 codes (32 bytes): the first quarter of the buffer
-              int8_t* buf8 = reinterpret_cast<int8_t*>(buf);
-#pragma unroll
-              for (int j = 0; j < 16; ++j) {
-                const int c = __float2int_rn(__fmul_rn(yv[j], out_inv));
-                buf8[(16 * h + j) * 32 + lane] = (int8_t)min(max(c, -127), 127);
+              for (int i = 0; i < 4; ++i) {
+                const int ac = ((int)v[4 * q + i]) >> (8 - BITS);
+                yv[4 * q + i] = __fmaf_rn(alpha, (float)ac, __fmaf_rn(beta, rsv[i], b));
               }
-            } else {
-#pragma unroll
-              for (int j = 0; j < 16; ++j) buf[(16 * h + j) * 32 + lane] = yv[j];
             }
+          }
+          if (lane == 0) ptx::tma_store_wait_read1();  // the store before last (same buffer) has read it
+          __syncwarp();
+          if constexpr (OUT == kOutBf16) {  // rows of 32 bfloat16 (64 bytes): the first half of the fp32 buffer
+            uint16_t* buf16 = reinterpret_cast<uint16_t*>(buf);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) buf16[j * 32 + lane] = __bfloat16_as_ushort(__float2bfloat16_rn(yv[j]));
+          } else if constexpr (OUT == kOutI8) {  // rows of 32 codes (32 bytes): the first quarter of the buffer
+            int8_t* buf8 = reinterpret_cast<int8_t*>(buf);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const int q = __float2int_rn(__fmul_rn(yv[j], out_inv));
+              buf8[j * 32 + lane] = (int8_t)min(max(q, -127), 127);
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) buf[j * 32 + lane] = yv[j];
           }
           ptx::fence_proxy_async_smem();
           __syncwarp();
@@ -658,10 +771,25 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
             }
           }
         }
+      };
+
+      // the warp's chunks: half, half + 2, ...
+      if (half >= n_chunks) release_acc();
+#pragma unroll 1
+      for (int ch = half; ch < n_chunks; ch += kEpilogueWarps / 4) {
+        uint32_t v[32];
+        ptx::tmem_ld_32x32b_x32(t_base + (uint32_t)(ch * 32), v);
+        ptx::tmem_ld_wait();
+        ptx::tmem_ld_regs_ready(v);
+        if (ch + kEpilogueWarps / 4 >= n_chunks) release_acc();  // the warp's last chunk is in registers
+        process(v, ch);
       }
-      ptx::tcgen05_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(acc_empty(a));
+      // stage the next tile's row sums for the other accumulator (its previous readers all passed this
+      // tile's barrier) and move on
+      if (have_nx && e < BT) rs_tile[(a ^ 1) * 256 + e] = nxt.rs;
+      c = nx;
+      cur = nxt;
+      have = have_nx;
     }
   }
 
@@ -673,14 +801,24 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
   // ---------------- teardown ----------------------------------------------------------------------
   ptx::tcgen05_fence_before_sync();
   __syncthreads();
+  // a pair: the other CTA's MMAs write this CTA's tensor memory and its roles arrive on this CTA's barriers;
+  // neither CTA may free anything or exit before both are done
+  if constexpr (CG == 2) ptx::cluster_sync_all();
   if (warp == 1) {
     __syncwarp();
     ptx::tcgen05_fence_after_sync();
-    ptx::tmem_dealloc(tmem_base, Cfg::kTmemCols);
+    ptx::tmem_dealloc_cg<CG>(tmem_base, Cfg::kTmemCols);
   }
 }
 
 // ---- host side -----------------------------------------------------------------------------------
+// 1 (default): launches with enough 256 x 256 tiles run as CTA pairs; 0: single-CTA tiles everywhere.
+// Read once from the environment (QBERT_PAIR=0 switches the pairs off, for comparisons).
+static const int g_pair_mode = [] {
+  const char* e = std::getenv("QBERT_PAIR");
+  return (e && e[0] == '0') ? 0 : 1;
+}();
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -746,29 +884,41 @@ static qb_status make_y_tensormap(CUtensorMap* tm, void* y, int64_t M, int64_t N
   return QB_OK;
 }
 
-template <int BT, int BITS, int OUT>
+// `grid` CTAs; with CG == 2 they are launched as clusters of two (grid is even).
+template <int BT, int BITS, int OUT, int CG>
 static qb_status launch_group_inst(const GroupedParams& gp, int grid, cudaStream_t stream) {
-  using Cfg = GemmCfg<BT>;
-  auto kernel = qb_gemm_kernel<BT, BITS, OUT>;
-  static bool attr_set[64] = {};
+  using Cfg = GemmCfg<BT, CG>;
+  auto kernel = qb_gemm_kernel<BT, BITS, OUT, CG>;
+  static std::atomic<bool> attr_set[64] = {};
   int dev = 0;
   QB_CUDA_TRY(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+  if (dev < 0 || dev >= 64 || !attr_set[dev].load(std::memory_order_acquire)) {
     QB_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
-    if (dev >= 0 && dev < 64) attr_set[dev] = true;
+    if (dev >= 0 && dev < 64) attr_set[dev].store(true, std::memory_order_release);
   }
-  kernel<<<grid, kGemmThreads, Cfg::kSmemBytes, stream>>>(gp);
-  QB_CUDA_TRY(cudaGetLastError());
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid, 1, 1);
+  cfg.blockDim = dim3(kGemmThreads, 1, 1);
+  cfg.dynamicSmemBytes = Cfg::kSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CG;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = CG == 2 ? 1 : 0;
+  QB_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, gp));
   return QB_OK;
 }
 
-template <int BT, int OUT>
+template <int BT, int OUT, int CG>
 static qb_status launch_group_bits(int bits, const GroupedParams& gp, int grid, cudaStream_t stream) {
   switch (bits) {
-    case 2: return launch_group_inst<BT, 2, OUT>(gp, grid, stream);
-    case 3: return launch_group_inst<BT, 3, OUT>(gp, grid, stream);
-    case 4: return launch_group_inst<BT, 4, OUT>(gp, grid, stream);
-    case 8: return launch_group_inst<BT, 8, OUT>(gp, grid, stream);
+    case 2: return launch_group_inst<BT, 2, OUT, CG>(gp, grid, stream);
+    case 3: return launch_group_inst<BT, 3, OUT, CG>(gp, grid, stream);
+    case 4: return launch_group_inst<BT, 4, OUT, CG>(gp, grid, stream);
+    case 8: return launch_group_inst<BT, 8, OUT, CG>(gp, grid, stream);
     default: return QB_ERR_INVALID;
   }
 }
@@ -777,12 +927,21 @@ static qb_status launch_group_bits(int bits, const GroupedParams& gp, int grid, 
 // small to give every SM a 256-token tile.  The 128-wide instruction takes as long as the 256-wide one
 // (measured with qb_probe_i8_mma: 498 vs 512 cycles per K block), so narrow tiles halve the tensor rate
 // and double the weight expansion per token; they pay only when SMs would otherwise idle.
-static int choose_token_tile(const qb_linear_desc* d, const int* idx, int count, int sm_count) {
+// `cg_out`: CTAs per tile.  A launch with at least one 256 x 256 tile per pair of SMs runs as CTA pairs: each
+// CTA then stages half of the token tile (half the L2 and shared-memory traffic per MMA) and the ring is
+// five K blocks deep instead of three.
+static int choose_token_tile(const qb_linear_desc* d, const int* idx, int count, int sm_count, int* cg_out) {
   bool wide = false;
-  int64_t tiles256 = 0;
+  int64_t tiles256 = 0, tiles_pair = 0;
   for (int i = 0; i < count; ++i) {
     if (d[idx[i]].M > 128) wide = true;
     tiles256 += ((d[idx[i]].N + kTileN - 1) / kTileN) * ((d[idx[i]].M + 255) / 256);
+    tiles_pair += ((d[idx[i]].N + 2 * kTileN - 1) / (2 * kTileN)) * ((d[idx[i]].M + 255) / 256);
+  }
+  *cg_out = 1;
+  if (wide && sm_count >= 2 && tiles_pair >= sm_count / 2 && g_pair_mode != 0) {
+    *cg_out = 2;
+    return 256;
   }
   // a launch that cannot give every SM a 256-token tile uses 128-token tiles: twice the CTAs at work,
   // half the epilogue per tile
@@ -817,7 +976,9 @@ static qb_status launch_group(const qb_linear_desc* d, const int* idx, int count
                               const float* const* out_scales = nullptr) {
   const int sm_count = max_ctas;
   const int bits = d[idx[0]].bits;
-  const int bt = choose_token_tile(d, idx, count, sm_count);
+  int cg = 1;
+  const int bt = choose_token_tile(d, idx, count, sm_count, &cg);
+  const int group_n = kTileN * cg;
   GroupedParams gp;
   memset(&gp, 0, sizeof(gp));
   gp.ws = ws;
@@ -825,7 +986,7 @@ static qb_status launch_group(const qb_linear_desc* d, const int* idx, int count
   int tile = 0;
   for (int i = 0; i < count; ++i) {
     const qb_linear_desc& q = d[idx[i]];
-    qb_status st = make_x_tensormap(&gp.tmx[i], q.xq, q.M, q.K, bt);
+    qb_status st = make_x_tensormap(&gp.tmx[i], q.xq, q.M, q.K, bt / cg);
     if (st != QB_OK) return st;
     // Y rows 16-byte aligned: the epilogue stages tiles in shared memory and stores them with TMA
     const bool tma_store = (q.N % (out == kOutF32 ? 4 : (out == kOutBf16 ? 8 : 16)) == 0) && aligned16(q.y);
@@ -849,14 +1010,15 @@ static qb_status launch_group(const qb_linear_desc* d, const int* idx, int count
     p.N = (int32_t)q.N;
     p.K = (int32_t)q.K;
     p.rows_per_group = (int32_t)(q.N / q.groups);
-    p.n_tiles = (int32_t)((q.N + kTileN - 1) / kTileN);
+    p.n_tiles = (int32_t)((q.N + group_n - 1) / group_n);
     p.m_tiles = (int32_t)((q.M + bt - 1) / bt);
     p.tile_begin = tile;
     p.tma_store = tma_store ? 1 : 0;
     tile += p.n_tiles * p.m_tiles;
   }
   gp.total_tiles = tile;
-  const int grid = tile < sm_count ? tile : sm_count;
+  const int max_groups = sm_count / cg;
+  const int grid = tile < max_groups ? tile : max_groups;  // CTA groups
   gp.total_positions = tile;
   gp.use_order = 0;
   // Tiles of different problems differ in length (K blocks).  When the launch is small enough for the
@@ -893,14 +1055,19 @@ static qb_status launch_group(const qb_linear_desc* d, const int* idx, int count
       }
     }
   }
+  if (cg == 2) {
+    if (out == kOutBf16) return launch_group_bits<256, kOutBf16, 2>(bits, gp, 2 * grid, stream);
+    if (out == kOutI8) return launch_group_bits<256, kOutI8, 2>(bits, gp, 2 * grid, stream);
+    return launch_group_bits<256, kOutF32, 2>(bits, gp, 2 * grid, stream);
+  }
   if (out == kOutBf16)
-    return bt == 256 ? launch_group_bits<256, kOutBf16>(bits, gp, grid, stream)
-                     : launch_group_bits<128, kOutBf16>(bits, gp, grid, stream);
+    return bt == 256 ? launch_group_bits<256, kOutBf16, 1>(bits, gp, grid, stream)
+                     : launch_group_bits<128, kOutBf16, 1>(bits, gp, grid, stream);
   if (out == kOutI8)
-    return bt == 256 ? launch_group_bits<256, kOutI8>(bits, gp, grid, stream)
-                     : launch_group_bits<128, kOutI8>(bits, gp, grid, stream);
-  return bt == 256 ? launch_group_bits<256, kOutF32>(bits, gp, grid, stream)
-                   : launch_group_bits<128, kOutF32>(bits, gp, grid, stream);
+    return bt == 256 ? launch_group_bits<256, kOutI8, 1>(bits, gp, grid, stream)
+                     : launch_group_bits<128, kOutI8, 1>(bits, gp, grid, stream);
+  return bt == 256 ? launch_group_bits<256, kOutF32, 1>(bits, gp, grid, stream)
+                   : launch_group_bits<128, kOutF32, 1>(bits, gp, grid, stream);
 }
 
 // Side streams and events for launches of one stack that run side by side (host objects, created once per

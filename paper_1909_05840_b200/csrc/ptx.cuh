@@ -134,6 +134,30 @@ __device__ __forceinline__ void tma_store_wait_read1() {
   asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
 }
 
+// Two IEEE fused multiply-adds in one instruction: d0 = fma(a0, b0, c0), d1 = fma(a1, b1, c1), each rounded
+// to nearest even exactly as fma.rn.f32 would.
+__device__ __forceinline__ void fma_f32x2(float& d0, float& d1, float a0, float a1, float b0, float b1, float c0,
+                                          float c1) {
+  asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
+      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%6, %7};\n\t"
+      "fma.rn.f32x2 rd, ra, rb, rc;\n\t"
+      "mov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d0), "=f"(d1)
+      : "f"(a0), "f"(a1), "f"(b0), "f"(b1), "f"(c0), "f"(c1));
+}
+
+// ---- register reallocation between warpgroups ------------------------------------------------------
+// Executed by all warps of a warpgroup (four consecutive warps).  dec releases registers down to N per
+// thread; inc waits until the CTA's pool (threads x registers at launch) has N per thread to give.
+template <int N>
+__device__ __forceinline__ void setmaxnreg_dec() {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N>
+__device__ __forceinline__ void setmaxnreg_inc() {
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+}
+
 // ---- tensor memory -----------------------------------------------------------------------------
 // Allocate `ncols` (power of two, >= 32) columns; the base address is written to shared memory.
 // Must be executed by one whole warp.
@@ -184,9 +208,13 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
   return r;
 }
-// Arrive on an mbarrier given by a shared::cluster address (this CTA's or another's); release at cluster scope.
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+// Arrive on an mbarrier of another CTA of the cluster, given by its shared::cluster address.  Default
+// semantics (release at CTA scope): the writes this arrival publishes are this CTA's own shared-memory
+// writes, made visible to the tensor cores by fence.proxy.async before the arrival is sent, and they are read
+// through this CTA's own shared memory; no cluster-scope fence (which would also wait for the thread's
+// global loads in flight) is needed, and none is paid.
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // 2-D tiled load whose completion is counted on an mbarrier that may live in the peer CTA of the pair
 // (`bar_cluster` is a shared::cluster address).  No multicast: the data goes to this CTA only.
