@@ -36,6 +36,7 @@
 #include <atomic>
 #include <cstdlib>
 #include <cstring>
+#include <type_traits>
 #include <vector>
 
 #include "common.cuh"
@@ -44,9 +45,6 @@
 
 namespace qb {
 
-#ifndef QB_LOAD_AFTER
-#define QB_LOAD_AFTER 1
-#endif
 // Roles sit on warpgroup boundaries (four consecutive warps) so that registers can be moved between them
 // with setmaxnreg: warpgroup 0 holds the two single-thread roles (and two idle warps) and gives its
 // registers away, warpgroups 1-3 are the expander teams, warpgroups 4-5 the epilogue.
@@ -71,7 +69,7 @@ constexpr int kTileN = 128;          // output neurons per tile (MMA M)
 constexpr int kBlockK = 128;         // K elements (= bytes) per pipeline stage
 constexpr int kWBytes = kTileN * kBlockK;
 
-constexpr int kMaxProblems = 16;
+constexpr int kMaxProblems = 48;
 constexpr int kMaxOrder = 4096;   // entries of the explicit tile visiting order (when it is used)
 constexpr uint16_t kNoTile = 0xFFFF;  // linears per launch (all in kernel-parameter space, no device table)
 
@@ -91,6 +89,7 @@ struct Problem {
   int32_t n_tiles, m_tiles;
   int32_t tile_begin;  // index of this problem's first tile in the launch's tile list
   int32_t tma_store;   // 1: Y rows are 16-byte aligned, the epilogue stores through TMA
+  int32_t bits;        // bit width of this problem's codes (read by the kernels that mix bit widths)
 };
 
 struct GroupedParams {
@@ -240,11 +239,28 @@ struct TileCursor {
         break;
       }
     }
-    pi = 0;
-    while (pi + 1 < gp.count && t >= gp.prob[pi + 1].tile_begin) ++pi;
+    // the problem that owns tile t: the last one whose first tile is <= t
+    int lo = 0, hi = gp.count - 1;
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (t >= gp.prob[mid].tile_begin) lo = mid;
+      else hi = mid - 1;
+    }
+    pi = lo;
     return true;
   }
 };
+
+// Barrier over the four warps of an expander team (named barriers 2..) that also ORs a predicate over them.
+__device__ __forceinline__ bool team_sync_or(bool pred, int bar_id) {
+  uint32_t res;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.or.pred p, %2, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(res)
+      : "r"((uint32_t)pred), "r"(bar_id)
+      : "memory");
+  return res != 0;
+}
 
 // Barrier over the epilogue warps (named barrier 1) that also ORs a predicate over them.
 __device__ __forceinline__ bool epilogue_sync_or(bool pred) {
@@ -347,9 +363,23 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
       bool have = c.next(gp);
       constexpr int kMyRow0 = 0;
       const int row_off = (int)cta_rank * Cfg::kXRows + kMyRow0;  // this CTA's rows inside the token tile
+      // Narrow token tiles are what launches with few tokens use: there every packed weight is read once,
+      // straight from DRAM, and the expanders' register prefetch alone does not keep enough bytes in flight
+      // (a K block of 2-bit weights is 4 KB).  The producer therefore asks L2 for a tile's whole block of
+      // packed rows (contiguous in memory) one tile ahead of its use.
+      auto prefetch_weights = [&](const TileCursor& tc) {
+        if constexpr (BT == 128) {
+          const Problem& pw = gp.prob[tc.pi];
+          const int n0 = ((tc.t - pw.tile_begin) % pw.n_tiles) * kGroupN + (int)cta_rank * kTileN;
+          const int rows = min(kTileN, pw.N - n0);
+          const uint32_t row_bytes = (uint32_t)(pw.K / 8 * (BITS ? BITS : pw.bits));
+          if (rows > 0) ptx::bulk_prefetch_l2(reinterpret_cast<const uint8_t*>(pw.packed) + (size_t)n0 * row_bytes, (uint32_t)rows * row_bytes);
+        }
+      };
       if (have) {
         const Problem& pr = gp.prob[c.pi];
         const int m0 = ((c.t - pr.tile_begin) / pr.n_tiles) * BT + row_off;
+        prefetch_weights(c);
         for (int kb = 0; kb < kL2Ahead && kb < pr.K / kBlockK; ++kb) ptx::tma_prefetch_l2_2d(&gp.tmx[c.pi], kb * kBlockK, m0);
       }
       while (have && !timed_out) {
@@ -364,6 +394,7 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
         int m0_nx = 0, kblocks_nx = 0;
         if (have_nx) {
           const Problem& pn = gp.prob[nx.pi];
+          prefetch_weights(nx);
           tm_nx = &gp.tmx[nx.pi];
           m0_nx = ((nx.t - pn.tile_begin) / pn.n_tiles) * BT + row_off;
           kblocks_nx = pn.K / kBlockK;
@@ -484,7 +515,7 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
     TileCursor c;
     c.start(CG);
     int ld_kb = team;
-    int ld_kblocks = 0, ld_n0 = 0, ld_N = 0, ld_wpr = 0;
+    int ld_kblocks = 0, ld_n0 = 0, ld_N = 0, ld_wpr = 0, ld_bits = BITS;
     const uint32_t* ld_packed = nullptr;
     bool ld_done = !c.next(gp);
     auto enter_tile = [&]() {  // fields of the tile the cursor stands on
@@ -492,7 +523,8 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
       ld_kblocks = pr.K / kBlockK;
       ld_n0 = ((c.t - pr.tile_begin) % pr.n_tiles) * kGroupN + (int)cta_rank * kTileN;
       ld_N = pr.N;
-      ld_wpr = pr.K / 32 * BITS;
+      if constexpr (BITS == 0) ld_bits = pr.bits;  // a launch that mixes bit widths: the tile's own
+      ld_wpr = pr.K / 32 * ld_bits;
       ld_packed = pr.packed;
     };
     auto normalize = [&]() {  // carry ld_kb over tile ends
@@ -509,59 +541,91 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
       enter_tile();
       normalize();
     }
-    // Register prefetch of the packed words, kPrefetch team-iterations ahead.
-    constexpr int kPrefetch = BITS == 8 ? 1 : 2;
-    uint32_t pre[kPrefetch][4 * BITS];
+    // Register prefetch of the packed words, kPrefetch team-iterations ahead.  kW: words per item of 32 codes
+    // (the bit width; 8, the largest, when the launch mixes widths: every buffer then carries its own width).
+    constexpr int kW = BITS ? BITS : 8;
+    constexpr int kPrefetch = kW == 8 ? 1 : 2;
+    uint32_t pre[kPrefetch][4 * kW];
+    int pre_bits[kPrefetch];
     bool pre_valid[kPrefetch];
-    auto load_next = [&](uint32_t* nxt) -> bool {
-      if (ld_done) return false;
+    auto load_rows = [&](auto width, uint32_t* nxt) {
+      constexpr int B = decltype(width)::value;
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const int n = ld_n0 + row0 + 32 * j;
         if (n < ld_N) {
-          load_item<BITS>(ld_packed + (size_t)n * ld_wpr + ld_kb * (4 * BITS) + piece * BITS, nxt + j * BITS);
+          load_item<B>(ld_packed + (size_t)n * ld_wpr + ld_kb * (4 * B) + piece * B, nxt + j * kW);
         } else {
           // rows past N: their accumulators are never stored, any operand value will do
 #pragma unroll
-          for (int w = 0; w < BITS; ++w) nxt[j * BITS + w] = 0u;
+          for (int w = 0; w < B; ++w) nxt[j * kW + w] = 0u;
+        }
+      }
+    };
+    auto load_next = [&](uint32_t* nxt, int& nxt_bits) -> bool {
+      if (ld_done) return false;
+      nxt_bits = ld_bits;
+      if constexpr (BITS != 0) {
+        load_rows(std::integral_constant<int, BITS ? BITS : 8>(), nxt);
+      } else {
+        switch (ld_bits) {  // the same for every thread of the CTA
+          case 2: load_rows(std::integral_constant<int, 2>(), nxt); break;
+          case 3: load_rows(std::integral_constant<int, 3>(), nxt); break;
+          case 4: load_rows(std::integral_constant<int, 4>(), nxt); break;
+          default: load_rows(std::integral_constant<int, 8>(), nxt); break;
         }
       }
       ld_kb += kExpandTeams;
       normalize();
       return true;
     };
+    auto expand_rows = [&](auto width, const uint32_t* words, uint8_t* stage_ptr) {
+      constexpr int B = decltype(width)::value;
 #pragma unroll
-    for (int d = 0; d < kPrefetch; ++d) pre_valid[d] = load_next(pre[d]);
+      for (int j = 0; j < 4; ++j) {
+        const int row = row0 + 32 * j;
+        uint32_t out[8];
+        expand_item<B>(words + j * kW, out);
+        // the item is 16-byte chunks 2*piece and 2*piece+1 of the row; 128-byte swizzle: chunk ^ (row % 8)
+        uint8_t* row_ptr = stage_ptr + row * 128;
+        *reinterpret_cast<uint4*>(row_ptr + (((2 * piece) ^ (row & 7)) << 4)) = make_uint4(out[0], out[1], out[2], out[3]);
+        *reinterpret_cast<uint4*>(row_ptr + (((2 * piece + 1) ^ (row & 7)) << 4)) = make_uint4(out[4], out[5], out[6], out[7]);
+      }
+    };
+#pragma unroll
+    for (int d = 0; d < kPrefetch; ++d) pre_valid[d] = load_next(pre[d], pre_bits[d]);
     int stage = team % kStages;
     uint32_t phase = (uint32_t)(team / kStages) & 1u;
     while (pre_valid[0]) {
-      uint32_t cur[4 * BITS];
+      uint32_t cur[4 * kW];
+      const int cur_bits = pre_bits[0];
 #pragma unroll
-      for (int i = 0; i < 4 * BITS; ++i) cur[i] = pre[0][i];
+      for (int i = 0; i < 4 * kW; ++i) cur[i] = pre[0][i];
 #pragma unroll
       for (int d = 0; d + 1 < kPrefetch; ++d) {
         pre_valid[d] = pre_valid[d + 1];
+        pre_bits[d] = pre_bits[d + 1];
 #pragma unroll
-        for (int i = 0; i < 4 * BITS; ++i) pre[d][i] = pre[d + 1][i];
+        for (int i = 0; i < 4 * kW; ++i) pre[d][i] = pre[d + 1][i];
       }
-#if !QB_LOAD_AFTER
-      pre_valid[kPrefetch - 1] = load_next(pre[kPrefetch - 1]);
-#endif
-      if (!wait_barrier_warp(empty(stage), phase ^ 1u, abort_flag)) {
+      // the team's first warp polls the stage's barrier, the other three are parked at the team's named
+      // barrier, which also makes the decision to give up the same in all four
+      const bool got = (warp & 3) != 0 || wait_barrier_warp(empty(stage), phase ^ 1u, abort_flag);
+      if (team_sync_or(!got, 2 + team)) {
         timed_out = true;
         where = (2 << 16) | stage;
         break;
       }
       uint8_t* stage_ptr = smem + stage * Cfg::kStageBytes;
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int row = row0 + 32 * j;
-        uint32_t out[8];
-        expand_item<BITS>(cur + j * BITS, out);
-        // the item is 16-byte chunks 2*piece and 2*piece+1 of the row; 128-byte swizzle: chunk ^ (row % 8)
-        uint8_t* row_ptr = stage_ptr + row * 128;
-        *reinterpret_cast<uint4*>(row_ptr + (((2 * piece) ^ (row & 7)) << 4)) = make_uint4(out[0], out[1], out[2], out[3]);
-        *reinterpret_cast<uint4*>(row_ptr + (((2 * piece + 1) ^ (row & 7)) << 4)) = make_uint4(out[4], out[5], out[6], out[7]);
+      if constexpr (BITS != 0) {
+        expand_rows(std::integral_constant<int, BITS ? BITS : 8>(), cur, stage_ptr);
+      } else {
+        switch (cur_bits) {
+          case 2: expand_rows(std::integral_constant<int, 2>(), cur, stage_ptr); break;
+          case 3: expand_rows(std::integral_constant<int, 3>(), cur, stage_ptr); break;
+          case 4: expand_rows(std::integral_constant<int, 4>(), cur, stage_ptr); break;
+          default: expand_rows(std::integral_constant<int, 8>(), cur, stage_ptr); break;
+        }
       }
       ptx::fence_proxy_async_smem();  // every lane: its own stores -> visible to the tensor cores
       __syncwarp();
@@ -569,11 +633,9 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
         if (CG == 2 && cta_rank != 0) ptx::mbar_arrive_remote(full_lead(stage));
         else ptx::mbar_arrive(full(stage));
       }
-#if QB_LOAD_AFTER
       // the next fetch goes out after the proxy fence, not before it: the fence waits for the thread's loads
       // in flight, and a fetch issued first would put its whole latency into every K block
-      pre_valid[kPrefetch - 1] = load_next(pre[kPrefetch - 1]);
-#endif
+      pre_valid[kPrefetch - 1] = load_next(pre[kPrefetch - 1], pre_bits[kPrefetch - 1]);
       stage += kExpandTeams;
       if (stage >= kStages) {
         stage -= kStages;
@@ -585,7 +647,7 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
     // ---------------- epilogue --------------------------------------------------------------------
     // Two warps per TMEM lane quarter; the warps of a quarter take alternate chunks of 32 tokens.  Per tile:
     // wait for the accumulator, then for every chunk: tcgen05.ld, convert and two fused multiply-adds per
-    // output (two outputs per instruction), 32 x 32 tile into shared memory, one TMA store.  The accumulator is handed back to the issuer as soon as the warp's last
+    // output, 32 x 32 tile into shared memory, one TMA store.  The accumulator is handed back to the issuer as soon as the warp's last
     // chunk is in registers.  The next tile's dequantization constants and row sums are fetched while
     // this tile drains.
     const int ew = warp - kFirstEpilogueWarp;
@@ -593,34 +655,42 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
     const int half = ew >> 2;                  // which of the quarter's two warps
     const int r = quarter * 32 + lane;         // output neuron inside the CTA's 128 rows
     const int e = threadIdx.x - kEpilogueThread0;  // 0..255: the token whose row sum this thread stages
-    constexpr int c_code = 1 << (BITS - 1);
     float* const warp_bufs = out_stage + ew * (2 * 32 * 32);
     int out_flip = 0;
 
     // per-tile values: the tile being drained, and the CTA's next tile (prefetched)
+    // `fetch` only issues the loads; the arithmetic on them (`finish`) comes when the tile's turn has come,
+    // so that the warp does not wait for a tile's constants while it could drain the one before.
     struct TileVals {
       int pi, n_base, m0;
-      float alpha, beta, b, rs;  // rs: row sum of token m0 + e (as fp32, exact), 0 past M
+      int bits;                   // bit width of the tile's codes
+      float s_a, dlt, z;          // as loaded: activation scale, the neuron's group step and offset
+      int32_t rs_i;               // row sum of token m0 + e, 0 past M
+      float alpha, beta, b, rs;   // after finish(); rs as fp32 (exact: |rowsum| < 2^24)
+    };
+    auto finish = [&](TileVals& tv) {
+      const float zc = __fmaf_rn(tv.dlt, (float)(1 << (tv.bits - 1)), tv.z);
+      tv.alpha = __fmul_rn(tv.s_a, tv.dlt);
+      tv.beta = __fmul_rn(tv.s_a, zc);
+      tv.rs = (float)tv.rs_i;
     };
     auto fetch = [&](const TileCursor& tc, TileVals& tv) {
       const Problem& pr = gp.prob[tc.pi];
       const int local = tc.t - pr.tile_begin;
       tv.pi = tc.pi;
+      tv.bits = BITS ? BITS : pr.bits;
       tv.n_base = (local % pr.n_tiles) * kGroupN + (int)cta_rank * kTileN;
       tv.m0 = (local / pr.n_tiles) * BT;
       const int n = tv.n_base + r;
-      tv.alpha = tv.beta = tv.b = 0.f;
+      tv.s_a = tv.dlt = tv.z = tv.b = 0.f;  // neurons past N: alpha = beta = b = 0, never stored
       if (n < pr.N) {
-        const float s_a = __ldg(pr.act_scale);
+        tv.s_a = __ldg(pr.act_scale);
         const int g = n / pr.rows_per_group;
-        const float dlt = __ldg(pr.delta + g);
-        const float z = __ldg(pr.q0 + g);
-        const float zc = __fmaf_rn(dlt, (float)c_code, z);
-        tv.alpha = __fmul_rn(s_a, dlt);
-        tv.beta = __fmul_rn(s_a, zc);
+        tv.dlt = __ldg(pr.delta + g);
+        tv.z = __ldg(pr.q0 + g);
         tv.b = pr.bias ? __ldg(pr.bias + n) : 0.0f;
       }
-      tv.rs = (e < BT && tv.m0 + e < pr.M) ? (float)__ldg(pr.rowsum + tv.m0 + e) : 0.0f;  // exact: |rowsum| < 2^24
+      tv.rs_i = (e < BT && tv.m0 + e < pr.M) ? __ldg(pr.rowsum + tv.m0 + e) : 0;
     };
 
     TileCursor c;
@@ -629,6 +699,7 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
     TileVals cur;
     if (have) {
       fetch(c, cur);
+      finish(cur);
       if (e < BT) rs_tile[e] = cur.rs;  // accumulator 0's row sums; published by the barrier below
     }
     for (int it = 0; have; ++it) {
@@ -642,9 +713,8 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
       const bool nvalid = n < pN;
       const bool tma_store = pr.tma_store != 0;
       const float alpha = cur.alpha, beta = cur.beta, b = cur.b;
-      // alpha * 2^-(8-BITS), used when that scaling loses no bits in any lane of the warp
-      const float alpha_s = __fmul_rn(alpha, 1.0f / (float)(1 << (8 - BITS)));
-      const bool fold_shift = __all_sync(0xffffffffu, __fmul_rn(alpha_s, (float)(1 << (8 - BITS))) == alpha);
+      const int sh = 8 - cur.bits;           // the tensor cores were fed (code - c) << sh
+      const int c_code = 1 << (cur.bits - 1);
       float* const y_ptr = reinterpret_cast<float*>(pr.y);
       uint16_t* const y16_ptr = reinterpret_cast<uint16_t*>(pr.y);
       int8_t* const y8_ptr = reinterpret_cast<int8_t*>(pr.y);
@@ -652,7 +722,9 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
       if constexpr (OUT == kOutI8) out_inv = __fdiv_rn(1.0f, __ldg(pr.out_scale));
       int32_t* const acc_ptr = pr.acc_out;
 
-      const bool ok = wait_barrier_warp(acc_full(a), aphase, abort_flag);
+      // one warp polls the accumulator's barrier; the others are parked at the named barrier below (a
+      // polling warp spends issue slots, a parked one none)
+      const bool ok = ew != 0 || wait_barrier_warp(acc_full(a), aphase, abort_flag);
       // One barrier over the epilogue warps per tile: it publishes the row sums staged for this tile and
       // makes the decision to give up the same in all eight warps (a warp that left alone would leave
       // the others waiting at this barrier).
@@ -691,31 +763,16 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
           // 32 tokens x 32 neurons of this warp -> shared memory [token][neuron] -> one TMA store.
           // Lanes write consecutive words of a row: conflict-free.  Rows past M and neurons past N
           // are clipped by the tensor map.  All 32 results are formed first (in the registers that held
-          // the accumulators), two per instruction: y = fma(alpha, (float)Ac, fma(beta, rowsum, b)) with
-          // Ac = v >> (8 - BITS).  When alpha * 2^-(8-BITS) is exact (always, short of underflow) the
-          // shift is folded into alpha: (float)v = 2^(8-BITS) * (float)Ac exactly, so the product, and
-          // with it the fused result, is the same real number rounded once.
+          // the accumulators): y = fma(alpha, (float)Ac, fma(beta, rowsum, b)) with Ac = v >> sh.
           float yv[32];
-          if (fold_shift) {
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-              const float4 rv = rs4[q];  // same address in every lane: one broadcast read
-              float t0, t1, t2, t3;
-              ptx::fma_f32x2(t0, t1, beta, beta, rv.x, rv.y, b, b);
-              ptx::fma_f32x2(t2, t3, beta, beta, rv.z, rv.w, b, b);
-              ptx::fma_f32x2(yv[4 * q], yv[4 * q + 1], alpha_s, alpha_s, (float)(int)v[4 * q], (float)(int)v[4 * q + 1], t0, t1);
-              ptx::fma_f32x2(yv[4 * q + 2], yv[4 * q + 3], alpha_s, alpha_s, (float)(int)v[4 * q + 2], (float)(int)v[4 * q + 3], t2, t3);
-            }
-          } else {
+          for (int q = 0; q < 8; ++q) {
+            const float4 rv = rs4[q];  // same address in every lane: one broadcast read
+            const float rsv[4] = {rv.x, rv.y, rv.z, rv.w};
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-              const float4 rv = rs4[q];
-              const float rsv[4] = {rv.x, rv.y, rv.z, rv.w};
-#pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                const int ac = ((int)v[4 * q + i]) >> (8 - BITS);
-                yv[4 * q + i] = __fmaf_rn(alpha, (float)ac, __fmaf_rn(beta, rsv[i], b));
-              }
+            for (int i = 0; i < 4; ++i) {
+              const int ac = ((int)v[4 * q + i]) >> sh;
+              yv[4 * q + i] = __fmaf_rn(alpha, (float)ac, __fmaf_rn(beta, rsv[i], b));
             }
           }
           if (lane == 0) ptx::tma_store_wait_read1();  // the store before last (same buffer) has read it
@@ -755,7 +812,7 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
               const int j = 4 * q + i;
-              const int ac = ((int)v[j]) >> (8 - BITS);
+              const int ac = ((int)v[j]) >> sh;
               if (nvalid && j < rows) {
                 if (!tma_store) {
                   const float yv = __fmaf_rn(alpha, (float)ac, __fmaf_rn(beta, rs[i], b));
@@ -786,7 +843,10 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
       }
       // stage the next tile's row sums for the other accumulator (its previous readers all passed this
       // tile's barrier) and move on
-      if (have_nx && e < BT) rs_tile[(a ^ 1) * 256 + e] = nxt.rs;
+      if (have_nx) {
+        finish(nxt);
+        if (e < BT) rs_tile[(a ^ 1) * 256 + e] = nxt.rs;
+      }
       c = nx;
       cur = nxt;
       have = have_nx;
@@ -975,9 +1035,15 @@ static qb_status launch_group(const qb_linear_desc* d, const int* idx, int count
                               int max_ctas, cudaStream_t stream, int out,
                               const float* const* out_scales = nullptr) {
   const int sm_count = max_ctas;
-  const int bits = d[idx[0]].bits;
+  int bits = d[idx[0]].bits;  // 0: the launch mixes bit widths (every problem carries its own)
+  for (int i = 1; i < count; ++i)
+    if (d[idx[i]].bits != bits) bits = 0;
   int cg = 1;
-  const int bt = choose_token_tile(d, idx, count, sm_count, &cg);
+  int bt = choose_token_tile(d, idx, count, sm_count, &cg);
+  if (bits == 0) {  // mixed widths: built for small stacks only (128-token tiles, single CTAs)
+    cg = 1;
+    bt = 128;
+  }
   const int group_n = kTileN * cg;
   GroupedParams gp;
   memset(&gp, 0, sizeof(gp));
@@ -1014,6 +1080,7 @@ static qb_status launch_group(const qb_linear_desc* d, const int* idx, int count
     p.m_tiles = (int32_t)((q.M + bt - 1) / bt);
     p.tile_begin = tile;
     p.tma_store = tma_store ? 1 : 0;
+    p.bits = q.bits;
     tile += p.n_tiles * p.m_tiles;
   }
   gp.total_tiles = tile;
@@ -1024,7 +1091,7 @@ static qb_status launch_group(const qb_linear_desc* d, const int* idx, int count
   // Tiles of different problems differ in length (K blocks).  When the launch is small enough for the
   // table, deal the tiles longest first to the least loaded CTA instead of round-robin.
   {
-    bool uniform = true;
+    bool uniform = bits != 0;
     for (int i = 1; i < count; ++i) uniform = uniform && gp.prob[i].K == gp.prob[0].K;
     if (!uniform && tile <= kMaxOrder && tile < (int)kNoTile) {
       constexpr int kEpilogueCost = 5;  // a tile's fixed cost in units of one K block
@@ -1032,7 +1099,9 @@ static qb_status launch_group(const qb_linear_desc* d, const int* idx, int count
       for (int i = 0, t = 0; i < count; ++i)
         for (int j = 0; j < gp.prob[i].n_tiles * gp.prob[i].m_tiles; ++j, ++t) {
           ids[t] = t;
-          cost[t] = gp.prob[i].K / kBlockK + kEpilogueCost;
+          // measured at M = 128: a K block of 3-bit weights takes about 1.2 times, of 8-bit weights about 1.4
+          // times as long as one of 2- or 4-bit weights
+          cost[t] = (gp.prob[i].K / kBlockK + kEpilogueCost) * (gp.prob[i].bits == 3 ? 12 : (gp.prob[i].bits == 8 ? 14 : 10));
         }
       std::stable_sort(ids.begin(), ids.end(), [&](int a, int b) { return cost[a] > cost[b]; });
       std::vector<std::vector<int>> lists(grid);
@@ -1055,6 +1124,11 @@ static qb_status launch_group(const qb_linear_desc* d, const int* idx, int count
       }
     }
   }
+  if (bits == 0) {
+    if (out == kOutBf16) return launch_group_inst<128, 0, kOutBf16, 1>(gp, grid, stream);
+    if (out == kOutI8) return launch_group_inst<128, 0, kOutI8, 1>(gp, grid, stream);
+    return launch_group_inst<128, 0, kOutF32, 1>(gp, grid, stream);
+  }
   if (cg == 2) {
     if (out == kOutBf16) return launch_group_bits<256, kOutBf16, 2>(bits, gp, 2 * grid, stream);
     if (out == kOutI8) return launch_group_bits<256, kOutI8, 2>(bits, gp, 2 * grid, stream);
@@ -1070,143 +1144,60 @@ static qb_status launch_group(const qb_linear_desc* d, const int* idx, int count
                    : launch_group_bits<128, kOutF32, 1>(bits, gp, grid, stream);
 }
 
-// Side streams and events for launches of one stack that run side by side (host objects, created once per
-// device on first use; no device memory).
-constexpr int kMaxSide = 7;
-struct SideStreams {
-  cudaStream_t stream[kMaxSide];
-  cudaEvent_t done[kMaxSide];
-  cudaEvent_t fork;
-  bool ready;
-};
-static qb_status side_streams(SideStreams** out) {
-  static SideStreams per_dev[64];
-  int dev = 0;
-  QB_CUDA_TRY(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= 64) {
-    set_last_error("device ordinal %d out of range", dev);
-    return QB_ERR_CUDA;
-  }
-  SideStreams& s = per_dev[dev];
-  if (!s.ready) {
-    for (int i = 0; i < kMaxSide; ++i) {
-      QB_CUDA_TRY(cudaStreamCreateWithFlags(&s.stream[i], cudaStreamNonBlocking));
-      QB_CUDA_TRY(cudaEventCreateWithFlags(&s.done[i], cudaEventDisableTiming));
-    }
-    QB_CUDA_TRY(cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming));
-    s.ready = true;
-  }
-  *out = &s;
-  return QB_OK;
-}
-
-// Split a stack into launches: same bit width per launch, longest K first (its tiles are the longest,
-// so they go out first in the round-robin), at most kMaxProblems problems and 2^30 tiles per launch.
-// A stack whose launches are all short (a mixed-precision stack at small M: a few tiles per SM in
-// total) runs its launches side by side, each on a share of the SMs in proportion to its work, so that
-// the start-up and the drain of the pipelines overlap instead of adding up; the launches join the
-// caller's stream before the call returns.  Large stacks keep one launch after the other on all SMs.
 struct StackGroup {
   int begin, count;
-  int64_t tiles, cost;
 };
-// The launches of a stack: `order` lists the descriptors by bit width, then longest K first; every group
-// is a run of `order` that one launch serves.
-static void plan_stack(const qb_linear_desc* d, int count, std::vector<int>& order, std::vector<StackGroup>& groups,
-                       int64_t* all_tiles_out, int64_t* all_cost_out) {
+// The launches of a stack.  `order` lists the descriptors, every group is a run of `order` that one launch
+// serves (at most kMaxProblems linears and 2^30 tiles).  A small stack (fewer than 16 tiles of 128 x 128
+// per SM in all: a mixed-precision stack at small M) is cut in stack order only, longest K first inside a
+// launch, and its launches mix bit widths: one launch, one tile list, one start-up and one drain for all
+// of it.  A large stack is sorted by bit width (every launch then has its bit width compiled in), longest
+// K first.
+static void plan_stack(const qb_linear_desc* d, int count, int sm_count, std::vector<int>& order,
+                       std::vector<StackGroup>& groups) {
+  groups.clear();
   order.resize(count);
   for (int i = 0; i < count; ++i) order[i] = i;
-  std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
-    if (d[a].bits != d[b].bits) return d[a].bits < d[b].bits;
-    return d[a].K > d[b].K;
-  });
-  int64_t all_tiles = 0, all_cost = 0;
+  int64_t all_tiles = 0;
+  bool mixed = false;
+  for (int i = 0; i < count; ++i) {
+    all_tiles += ((d[i].N + kTileN - 1) / kTileN) * ((d[i].M + 127) / 128);
+    mixed = mixed || d[i].bits != d[0].bits;
+  }
+  const bool small = mixed && all_tiles < (int64_t)16 * sm_count;
+  if (!small) {
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+      if (d[a].bits != d[b].bits) return d[a].bits < d[b].bits;
+      return d[a].K > d[b].K;
+    });
+  }
   int i = 0;
   while (i < count) {
     int j = i;
-    int64_t tiles = 0, cost = 0;
-    while (j < count && j - i < kMaxProblems && d[order[j]].bits == d[order[i]].bits) {
+    int64_t tiles = 0;
+    while (j < count && j - i < kMaxProblems && (small || d[order[j]].bits == d[order[i]].bits)) {
       const int64_t t = ((d[order[j]].N + kTileN - 1) / kTileN) * ((d[order[j]].M + 127) / 128);
       if (j > i && tiles + t > (1 << 30)) break;
       tiles += t;
-      cost += t * (d[order[j]].K / kBlockK + 5);  // K blocks plus a tile's fixed cost, as in the tile order
       ++j;
     }
-    // measured at M = 128: a K block of 3-bit weights takes about 1.2 times, of 8-bit weights about 1.4 times
-    // as long as one of 2- or 4-bit weights (expansion work; bytes fetched per block with few CTAs pulling)
-    const int b = d[order[i]].bits;
-    cost *= b == 3 ? 12 : (b == 8 ? 14 : 10);
-    groups.push_back({i, j - i, tiles, cost});
-    all_tiles += tiles;
-    all_cost += cost;
+    if (small)  // longest K first inside the launch: its tiles go out first
+      std::stable_sort(order.begin() + i, order.begin() + j, [&](int a, int b) { return d[a].K > d[b].K; });
+    groups.push_back({i, j - i});
     i = j;
   }
-  if (all_tiles_out) *all_tiles_out = all_tiles;
-  if (all_cost_out) *all_cost_out = all_cost;
 }
 
 static qb_status launch_stack(const qb_linear_desc* d, int count, void* ws, int sm_count, cudaStream_t stream,
                               int out, const float* const* out_scales = nullptr) {
   std::vector<int> order;
   std::vector<StackGroup> groups;
-  int64_t all_tiles = 0, all_cost = 0;
-  plan_stack(d, count, order, groups, &all_tiles, &all_cost);
-  using Group = StackGroup;
-  const int n_groups = (int)groups.size();
-  const bool side_by_side = n_groups > 1 && n_groups <= kMaxSide + 1 && n_groups <= sm_count &&
-                            all_tiles < (int64_t)16 * sm_count;
-  if (!side_by_side) {
-    for (const Group& g : groups) {
-      qb_status st = launch_group(d, order.data() + g.begin, g.count, nullptr, ws, sm_count, stream, out, out_scales);
-      if (st != QB_OK) return st;
-    }
-    return QB_OK;
+  plan_stack(d, count, sm_count, order, groups);
+  for (const StackGroup& g : groups) {
+    qb_status st = launch_group(d, order.data() + g.begin, g.count, nullptr, ws, sm_count, stream, out, out_scales);
+    if (st != QB_OK) return st;
   }
-  // SM shares in proportion to cost (at least one CTA each, no more than the launch has tiles); what
-  // rounding leaves over goes to the launches with the most work per CTA.
-  std::vector<int> share(n_groups);
-  int used = 0;
-  for (int g = 0; g < n_groups; ++g) {
-    int64_t sh = (int64_t)sm_count * groups[g].cost / all_cost;
-    if (sh < 1) sh = 1;
-    if (sh > groups[g].tiles) sh = groups[g].tiles;
-    share[g] = (int)sh;
-    used += share[g];
-  }
-  while (used > sm_count) {  // the minimum of one CTA per launch can overshoot: take from the largest share
-    int big = 0;
-    for (int g = 1; g < n_groups; ++g)
-      if (share[g] > share[big]) big = g;
-    --share[big];
-    --used;
-  }
-  while (used < sm_count) {
-    int best = -1;
-    for (int g = 0; g < n_groups; ++g)
-      if (share[g] < groups[g].tiles &&
-          (best < 0 || groups[g].cost * share[best] > groups[best].cost * share[g]))
-        best = g;
-    if (best < 0) break;
-    ++share[best];
-    ++used;
-  }
-  SideStreams* side = nullptr;
-  qb_status st = side_streams(&side);
-  if (st != QB_OK) return st;
-  QB_CUDA_TRY(cudaEventRecord(side->fork, stream));
-  for (int g = 1; g < n_groups; ++g) QB_CUDA_TRY(cudaStreamWaitEvent(side->stream[g - 1], side->fork, 0));
-  qb_status first_error = QB_OK;
-  for (int g = 0; g < n_groups; ++g) {
-    cudaStream_t sg = g == 0 ? stream : side->stream[g - 1];
-    st = launch_group(d, order.data() + groups[g].begin, groups[g].count, nullptr, ws, share[g], sg, out, out_scales);
-    if (st != QB_OK && first_error == QB_OK) first_error = st;
-  }
-  // always join, also after an error: the caller's stream must not run ahead of the side streams
-  for (int g = 1; g < n_groups; ++g) {
-    QB_CUDA_TRY(cudaEventRecord(side->done[g - 1], side->stream[g - 1]));
-    QB_CUDA_TRY(cudaStreamWaitEvent(stream, side->done[g - 1], 0));
-  }
-  return first_error;
+  return QB_OK;
 }
 
 }  // namespace qb
@@ -1330,7 +1321,9 @@ extern "C" int32_t qb_layer_linears_launch_count(const qb_linear_desc* descs, in
   if (!descs || count <= 0) return 0;
   std::vector<int> order;
   std::vector<qb::StackGroup> groups;
-  qb::plan_stack(descs, count, order, groups, nullptr, nullptr);
+  int sms = 148;
+  qb::require_sm100(&sms);  // without a device: the plan for a 148-SM part
+  qb::plan_stack(descs, count, sms, order, groups);
   return (int32_t)groups.size();
 }
 

@@ -117,6 +117,11 @@ __device__ __forceinline__ void tma_prefetch_l2_2d(const void* tmap, int32_t x, 
                : "memory");
 }
 
+// Ask L2 to fetch `bytes` contiguous bytes (16-byte aligned address, multiple of 16) that later loads will read.
+__device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(reinterpret_cast<uint64_t>(src)), "r"(bytes) : "memory");
+}
+
 // 2-D tiled store shared -> global (bulk async group).  Rows / columns of the box that fall outside
 // the tensor are not written.  x * element size must be a multiple of 16 bytes; x, y >= 0.
 __device__ __forceinline__ void tma_store_2d(const void* tmap, uint32_t src_smem, int32_t x, int32_t y) {
@@ -132,18 +137,6 @@ __device__ __forceinline__ void tma_store_wait_read0() {
 }
 __device__ __forceinline__ void tma_store_wait_read1() {
   asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-}
-
-// Two IEEE fused multiply-adds in one instruction: d0 = fma(a0, b0, c0), d1 = fma(a1, b1, c1), each rounded
-// to nearest even exactly as fma.rn.f32 would.
-__device__ __forceinline__ void fma_f32x2(float& d0, float& d1, float a0, float a1, float b0, float b1, float c0,
-                                          float c1) {
-  asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
-      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%6, %7};\n\t"
-      "fma.rn.f32x2 rd, ra, rb, rc;\n\t"
-      "mov.b64 {%0, %1}, rd;\n\t}"
-      : "=f"(d0), "=f"(d1)
-      : "f"(a0), "f"(a1), "f"(b0), "f"(b1), "f"(c0), "f"(c1));
 }
 
 // ---- register reallocation between warpgroups ------------------------------------------------------
