@@ -41,6 +41,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # table is keyed by a hash of that source and reads null as soon as the kernel changes.
 NCU_GEMM_TRAFFIC = {
     # "<sha256 of csrc/gemm.cu + csrc/ptx.cuh>": {<config>: bytes per launch}
+    # config 3: counters of a one-layer slice at M = 8192 (307.7 MB per launch) scaled by the units of a full
+    # launch (12 layers at three times the tokens: x 36); config 2: the whole stack in its one launch
+    "4e92f555469ecfec": {"3": 11.08e9, "2": 43.8e6},
 }
 NOMINAL_INT8_TOPS = 4500.0  # dense int8 tensor peak of the part as published (context, not the denominator)
 
@@ -800,6 +803,10 @@ def main():
                     help="steps of the end-to-end loop (default: 3 for the BERT-large stack, whose step moves 38 GB over the "
                          "host link, else 20)")
     ap.add_argument("--no-small-m", action="store_true", help="skip the small-M stack measured beside the main workload")
+    ap.add_argument("--slice-m", type=int, default=None,
+                    help="profiling slice: run the workload with this many token rows instead of its own M")
+    ap.add_argument("--slice-layers", type=int, default=None,
+                    help="profiling slice: run only the first layers of the workload")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--out", default="f32", choices=["f32", "bf16"],
                     help="output type of the GEMMs: fp32 (the graded path) or bfloat16 (qb_layer_linears_bf16)")
@@ -815,6 +822,13 @@ def main():
         run_quantizer_sweep(args)
         return
     wl = synth.workload(args.config)
+    if args.slice_m is not None or args.slice_layers is not None:
+        # a slice of the workload for profiler captures (small enough for multi-pass counters); its line is
+        # labelled as a slice and is not the benchmark's figure
+        layers = min(wl.layers, args.slice_layers or wl.layers)
+        m = args.slice_m or wl.M
+        wl = synth.Workload(wl.config, f"SLICE ({layers} of {wl.layers} layers, M={m}) of: {wl.name}", m, layers,
+                            wl.linears, wl.bits[:layers])
     if args.e2e_steps is None:
         args.e2e_steps = 3 if args.config == 3 else 20
     if args.impl == "reference":

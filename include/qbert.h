@@ -140,7 +140,9 @@ typedef struct {
  * its own scale (per-tensor quantization).  Weight matrices of different bit widths may be mixed;
  * each bit width gets its own launches, and when these are several small single-read launches (a
  * mixed-precision stack) they run side by side on streams the library creates once per device
- * (host objects only), forking from and joining `cuda_stream` inside the call as in qb_layer_linears.
+ * (host objects only), forking from and joining `cuda_stream` inside the call (after the fork every
+ * side stream is joined, also when a launch in between fails; the fork / launch / join sequence is
+ * serialised per device, so concurrent calls from several host threads are safe).
  * Workspace: qb_workspace_bytes(0, 0, 0, 0, G) bytes with G = max(32, sum of `groups` over the batch).
  */
 qb_status qb_quantize_act_batch(const qb_act_desc* descs /*host*/, int32_t count, void* ws, size_t ws_bytes,
@@ -218,12 +220,11 @@ typedef struct {
  * descriptors, e.g. four per encoder layer in the order QKV, attention output, FFN1, FFN2; each is
  * an independent problem with its own input, and the result of each equals qb_gemm on the same
  * arguments bit for bit.  All descriptors are validated before anything is launched.
- * Descriptors of equal bit width share a launch; a stack that mixes bit widths and is small (a few
- * tiles per SM in total) runs its launches side by side on streams the library creates once per
- * device (host objects only, no device memory).  They fork from and join `cuda_stream` inside the
- * call, so to the caller the work is ordered on `cuda_stream` as for every other call, and the call may
- * be captured into a CUDA graph.  The first such call on a device creates the streams and is not
- * safe to issue from two host threads at once.
+ * Up to 48 descriptors share one launch.  A large stack is cut into launches by bit width; a stack
+ * that mixes bit widths and is small (fewer than 16 tiles of 128 x 128 per SM in all: a mixed-precision
+ * stack at a few hundred tokens) goes out as launches that mix bit widths, so that the whole stack pays
+ * one start-up and one drain.  All launches are enqueued on `cuda_stream`, in order; the call uses no
+ * other stream, creates no host or device object, and may be captured into a CUDA graph.
  */
 qb_status qb_layer_linears(const qb_linear_desc* descs /*host*/, int32_t count, void* ws,
                            size_t ws_bytes, void* cuda_stream);

@@ -15,20 +15,27 @@
 // shift makes the expansion a mask and an xor per word; the epilogue shifts the exact int32 sum
 // back.  |sum| <= 127 * 128 * K < 2^31 for K <= 65536.
 //
-// One persistent CTA per SM, 22 warps:
+// One persistent CTA per SM, 24 warps, roles on warpgroup boundaries (registers are moved between the
+// warpgroups with setmaxnreg):
 //   warp 0        TMA producer for the token tiles               (one lane)
 //   warp 1        tcgen05.mma issuer, owns the TMEM allocation   (one lane)
-//   warps 2..13   weight expanders in three teams of four warps; team g fills the K blocks whose
+//   warps 2..3    idle (they complete the warpgroup that gives its registers away)
+//   warps 4..15   weight expanders in three teams of four warps; team g fills the K blocks whose
 //                 running index is g mod 3, thread r of a team owns weight row r of the tile
-//   warps 14..21  epilogue: TMEM -> registers -> fp32 -> shared memory -> TMA store; two warps per
+//   warps 16..23  epilogue: TMEM -> registers -> fp32 -> shared memory -> TMA store; two warps per
 //                 TMEM lane quarter, each taking every other chunk of 32 tokens
-// One launch serves up to kMaxProblems independent linears that share the bit width and the token
-// tile: their tiles form one list (longest K first) that the CTAs walk round-robin, so the start-up
-// and the drain of the pipeline are paid once per launch, not once per linear.
-// Shared-memory ring of STAGES stages (16 KB weights + BT*128 B tokens each, 128-byte swizzle, K
-// block of 128), two accumulator tiles in TMEM so the epilogue of tile i overlaps the MMAs of tile
-// i+1.  Every wait is bounded: on expiry the CTA records QB_ERR_TIMEOUT and leaves through the
-// normal exit path (TMEM freed).
+// Large launches run as CTA pairs (clusters of two, tcgen05 cta_group::2): the tile is 256 neurons x 256
+// tokens, each CTA expands its own 128 weight rows and stages its own 128 tokens, the pair's first CTA
+// issues one MMA for both.  That halves the token bytes each SM pulls from L2 and writes to and reads from
+// shared memory per MMA, and lets the ring be five K blocks deep instead of three.  No load is multicast.
+// One launch serves up to kMaxProblems independent linears that share the token tile: their tiles form
+// one list that the CTAs (or pairs) walk, so the start-up and the drain of the pipeline are paid once
+// per launch, not once per linear.  The bit width is a template argument, or (BITS = 0, small stacks
+// that mix widths) a field of every problem that the expanders and the epilogue read per tile.
+// Shared-memory ring of kStages stages (16 KB expanded weights + the CTA's token rows x 128 B each,
+// 128-byte swizzle, K block of 128), two accumulator tiles in TMEM so the epilogue of tile i overlaps
+// the MMAs of tile i+1.  Every wait is bounded: on expiry the CTA records QB_ERR_TIMEOUT and leaves
+// through the normal exit path (TMEM freed).
 #include <cuda.h>
 #include <cuda_bf16.h>
 

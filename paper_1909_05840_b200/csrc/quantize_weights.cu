@@ -14,6 +14,7 @@
 //                                shuffles so that the stores are contiguous 16k-byte runs.
 #include <algorithm>
 #include <cstring>
+#include <mutex>
 #include <vector>
 
 #include "common.cuh"
@@ -1070,6 +1071,7 @@ struct WeightSideStreams {
   cudaEvent_t done[kMaxSideJobs - 1];
   cudaEvent_t fork;
   bool ready;
+  std::mutex mu;  // one fork / launch / join sequence at a time per device: the events are shared
 };
 static qb_status weight_side_streams(WeightSideStreams** out) {
   static WeightSideStreams per_dev[64];
@@ -1080,6 +1082,7 @@ static qb_status weight_side_streams(WeightSideStreams** out) {
     return QB_ERR_CUDA;
   }
   WeightSideStreams& s = per_dev[dev];
+  std::lock_guard<std::mutex> lock(s.mu);
   if (!s.ready) {
     for (int i = 0; i < kMaxSideJobs - 1; ++i) {
       QB_CUDA_TRY(cudaStreamCreateWithFlags(&s.stream[i], cudaStreamNonBlocking));
@@ -1131,16 +1134,26 @@ static qb_status run_weight_jobs(const std::vector<WeightJob>& jobs, void* ws, i
   WeightSideStreams* sd = nullptr;
   qb_status st = weight_side_streams(&sd);
   if (st != QB_OK) return st;
-  QB_CUDA_TRY(cudaEventRecord(sd->fork, stream));
-  for (int i = 1; i < n; ++i) QB_CUDA_TRY(cudaStreamWaitEvent(sd->stream[i - 1], sd->fork, 0));
+  // Two host threads on one device would interleave their records of the shared events: serialise the
+  // whole fork / launch / join sequence.  After the fork every side stream is joined whatever fails in
+  // between, so that the caller's stream never runs ahead of work the call put on a side stream.
+  std::lock_guard<std::mutex> lock(sd->mu);
   qb_status first_error = QB_OK;
-  for (int i = 0; i < n; ++i) {
+  auto note = [&](cudaError_t e, const char* what) {
+    if (e != cudaSuccess && first_error == QB_OK) first_error = cuda_fail(e, what);
+    return e == cudaSuccess;
+  };
+  if (!note(cudaEventRecord(sd->fork, stream), "cudaEventRecord(fork)")) return first_error;  // nothing forked yet
+  bool forked[kMaxSideJobs] = {};
+  for (int i = 1; i < n; ++i) forked[i] = note(cudaStreamWaitEvent(sd->stream[i - 1], sd->fork, 0), "cudaStreamWaitEvent(fork)");
+  for (int i = 0; i < n && first_error == QB_OK; ++i) {
     st = run_weight_job(jobs[i], ws, sm_count, share[i], i == 0 ? stream : sd->stream[i - 1]);
     if (st != QB_OK && first_error == QB_OK) first_error = st;
   }
-  for (int i = 1; i < n; ++i) {  // always join, also after an error
-    QB_CUDA_TRY(cudaEventRecord(sd->done[i - 1], sd->stream[i - 1]));
-    QB_CUDA_TRY(cudaStreamWaitEvent(stream, sd->done[i - 1], 0));
+  for (int i = 1; i < n; ++i) {  // always join what was forked, also after an error
+    if (!forked[i]) continue;
+    if (note(cudaEventRecord(sd->done[i - 1], sd->stream[i - 1]), "cudaEventRecord(done)"))
+      note(cudaStreamWaitEvent(stream, sd->done[i - 1], 0), "cudaStreamWaitEvent(done)");
   }
   return first_error;
 }
