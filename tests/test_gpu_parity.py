@@ -204,6 +204,47 @@ def test_linear_wide_token_tiles(ws, bits):
     gu.check_linear(x, w, b, bits, groups, ws, use_omp=True)
 
 
+@pytest.mark.parametrize("bits", BITS)
+def test_linear_cta_pairs_ragged_tiles_through_tma_stores(ws, bits):
+    # enough 256 x 256 tiles for the CTA-pair kernel; the last neuron tile leaves the second CTA of the pair
+    # with 8 valid rows of 128, the last token tile is ragged (its second half partly outside M), K is
+    # five K blocks (the depth of the pair's ring); N % 4 == 0, so outputs leave through TMA stores
+    M, N, K, groups = 2500, 2440, 640, 10
+    x = synth.activations(M, K, seed=300 + bits)
+    w = synth.weights(N, K, seed=400 + bits)
+    b = synth.bias(N, seed=500 + bits) if bits != 3 else None
+    gu.check_linear(x, w, b, bits, groups, ws, use_omp=True)
+
+
+def test_small_mixed_stack_larger_than_one_launch(ws):
+    # 50 small linears of mixed bit widths and ragged shapes: more than one launch holds (48), every launch
+    # mixes bit widths; each result must equal the single call bit for bit and the oracle
+    rng = np.random.default_rng(77)
+    M = 96
+    descs, refs = [], []
+    for i in range(50):
+        N = int(rng.choice([24, 136, 264]))
+        K = int(rng.choice([128, 256, 640]))
+        bits = int(rng.choice(BITS))
+        G = int(rng.choice([1, 2, 4]))
+        x = synth.activations(M, K, seed=2000 + i)
+        w = synth.weights(N, K, seed=3000 + i)
+        b = synth.bias(N, seed=4000 + i)
+        xq, sc, rs = qb.quantize_act(gu.dev(x), ws)
+        packed, delta, q0 = qb.quantize_pack_weights(gu.dev(w), bits, G, ws)
+        y = gu.poison(torch.empty((M, N), dtype=torch.float32, device="cuda"))
+        descs.append(qb.LinearDesc(xq, sc, rs, packed, delta, q0, gu.dev(b), N, bits, G, y))
+        refs.append((x, w, b, bits, G))
+    assert qb.layer_linears_launch_count(descs) == 2
+    qb.layer_linears(descs, ws)
+    assert qb.read_status(ws) == qb.QB_OK
+    for d, (x, w, b, bits, G) in zip(descs, refs):
+        y1 = qb.gemm(d.xq, d.act_scale, d.rowsum, d.packed, d.delta, d.q0, d.bias, d.N, bits, G, ws)
+        assert torch.equal(y1, d.y)
+        ref = oracle.linear(x, w, b, bits, G)
+        gu.assert_y_close(d.y.cpu().numpy(), ref["y"])
+
+
 def test_linear_without_bias_and_with_positive_activations(ws):
     M, N, K, groups = 200, 256, 512, 32
     x = np.abs(synth.activations(M, K, seed=5))   # large row sums: the offset term dominates
