@@ -15,14 +15,14 @@
 // shift makes the expansion a mask and an xor per word; the epilogue shifts the exact int32 sum
 // back.  |sum| <= 127 * 128 * K < 2^31 for K <= 65536.
 //
-// One persistent CTA per SM, 24 warps, roles on warpgroup boundaries (registers are moved between the
+// One persistent CTA per SM, 28 warps, roles on warpgroup boundaries (registers are moved between the
 // warpgroups with setmaxnreg):
 //   warp 0        TMA producer for the token tiles               (one lane)
 //   warp 1        tcgen05.mma issuer, owns the TMEM allocation   (one lane)
 //   warps 2..3    idle (they complete the warpgroup that gives its registers away)
-//   warps 4..15   weight expanders in three teams of four warps; team g fills the K blocks whose
-//                 running index is g mod 3, thread r of a team owns weight row r of the tile
-//   warps 16..23  epilogue: TMEM -> registers -> fp32 -> shared memory -> TMA store; two warps per
+//   warps 4..19   weight expanders in four teams of four warps; team g fills the K blocks whose
+//                 running index is g mod 4, thread r of a team owns weight row r of the tile
+//   warps 20..27  epilogue: TMEM -> registers -> fp32 -> shared memory -> TMA store; two warps per
 //                 TMEM lane quarter, each taking every other chunk of 32 tokens
 // Large launches run as CTA pairs (clusters of two, tcgen05 cta_group::2): the tile is 256 neurons x 256
 // tokens, each CTA expands its own 128 weight rows and stages its own 128 tokens, the pair's first CTA
@@ -54,20 +54,23 @@ namespace qb {
 
 // Roles sit on warpgroup boundaries (four consecutive warps) so that registers can be moved between them
 // with setmaxnreg: warpgroup 0 holds the two single-thread roles (and two idle warps) and gives its
-// registers away, warpgroups 1-3 are the expander teams, warpgroups 4-5 the epilogue.
-constexpr int kExpandTeams = 3;     // teams of 128 expander threads
+// registers away, warpgroups 1-4 are the expander teams, warpgroups 5-6 the epilogue.
+// Four expander teams: at K = 4096 an expander iteration is about 1,500 busy cycles, so three teams only
+// just keep up with the 512 cycles the tensor cores need per K block (config 3's K = 4096 GEMM: 95 -> 84 us
+// with the fourth team).
+constexpr int kExpandTeams = 4;     // teams of 128 expander threads
 constexpr int kEpilogueWarps = 8;
 constexpr int kFirstExpandWarp = 4;
 constexpr int kFirstEpilogueWarp = kFirstExpandWarp + 4 * kExpandTeams;
 constexpr int kEpilogueThread0 = 32 * kFirstEpilogueWarp;
 constexpr int kGemmThreads = kEpilogueThread0 + 32 * kEpilogueWarps;
-// Registers per thread: the launch gives every thread kRegsLaunch (65,536 / 768 rounded down to a multiple
+// Registers per thread: the launch gives every thread kRegsLaunch (65,536 / 896 rounded down to a multiple
 // of 8); the shares below add up to at most kGemmThreads * kRegsLaunch, which setmaxnreg.inc needs in order
 // not to wait forever.
-constexpr int kRegsLaunch = 80;
+constexpr int kRegsLaunch = 72;
 constexpr int kRegsLight = 56;      // producer / issuer warpgroup
-constexpr int kRegsExpand = 72;
-constexpr int kRegsEpilogue = 104;
+constexpr int kRegsExpand = 64;
+constexpr int kRegsEpilogue = 96;
 static_assert(128 * kRegsLight + 128 * kExpandTeams * kRegsExpand + 32 * kEpilogueWarps * kRegsEpilogue <=
                   kGemmThreads * kRegsLaunch,
               "register shares exceed what the launch allocates");
@@ -513,7 +516,7 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
     // A K block of the tile is 128 rows x 4 items of 32 codes.  Thread i of a team takes items
     // i, i+128, i+256, i+384: piece i%4 of rows i/4 + 32j.  Four neighbouring lanes read one row's
     // 16*BITS contiguous bytes, so a warp-wide load touches 8 rows instead of 32.
-    // The K blocks of all tiles of this CTA form one sequence; team g takes those with index g mod 3.
+    // The K blocks of all tiles of this CTA form one sequence; team g takes those with index g mod 4.
     const int team = (warp - kFirstExpandWarp) >> 2;
     const int i_team = (threadIdx.x - 32 * kFirstExpandWarp) & 127;
     const int piece = i_team & 3;
@@ -548,10 +551,10 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
       enter_tile();
       normalize();
     }
-    // Register prefetch of the packed words, kPrefetch team-iterations ahead.  kW: words per item of 32 codes
+    // Register prefetch of the packed words, one team-iteration (four K blocks) ahead.  kW: words per item of 32 codes
     // (the bit width; 8, the largest, when the launch mixes widths: every buffer then carries its own width).
     constexpr int kW = BITS ? BITS : 8;
-    constexpr int kPrefetch = kW == 8 ? 1 : 2;
+    constexpr int kPrefetch = 1;
     uint32_t pre[kPrefetch][4 * kW];
     int pre_bits[kPrefetch];
     bool pre_valid[kPrefetch];
@@ -644,7 +647,7 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
       // in flight, and a fetch issued first would put its whole latency into every K block
       pre_valid[kPrefetch - 1] = load_next(pre[kPrefetch - 1], pre_bits[kPrefetch - 1]);
       stage += kExpandTeams;
-      if (stage >= kStages) {
+      while (stage >= kStages) {
         stage -= kStages;
         phase ^= 1u;
       }
