@@ -43,7 +43,7 @@ NCU_GEMM_TRAFFIC = {
     # "<sha256 of csrc/gemm.cu + csrc/ptx.cuh>": {<config>: bytes per launch}
     # config 3: counters of a one-layer slice at M = 8192 (307.7 MB per launch) scaled by the units of a full
     # launch (12 layers at three times the tokens: x 36); config 2: the whole stack in its one launch
-    "7303c1920f6b7a9e": {"3": 11.08e9, "2": 43.8e6},
+    "61f74ecfed67dfbf": {"3": 11.08e9, "2": 43.8e6},
 }
 NOMINAL_INT8_TOPS = 4500.0  # dense int8 tensor peak of the part as published (context, not the denominator)
 

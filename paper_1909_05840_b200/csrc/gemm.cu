@@ -366,8 +366,13 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
       uint32_t phase = 0;
       // The token tiles are first touched in DRAM by several CTAs at about the same time, and the
       // ring holds only a few K blocks: L2 prefetches run kL2Ahead blocks ahead of the loads (into the
-      // CTA's next tile when the current one ends) so that the loads themselves hit L2.
+      // CTA's next tile when the current one ends) so that the loads themselves hit L2.  Only for long K
+      // (more than kL2MinBlocks K blocks per tile): there the loads of a tile are what the tensor cores
+      // wait for (K = 4096 GEMM of config 3: 84 against 86 us); for short K the token tile was fetched
+      // moments ago by the CTAs on the neighbouring neuron tiles, and the prefetch instructions only take
+      // the TMA unit's time (16 linears of config 3: 1,241 -> 1,208 us without them).
       constexpr int kL2Ahead = 8;
+      constexpr int kL2MinBlocks = 8;
       TileCursor c;
       c.start(CG);
       bool have = c.next(gp);
@@ -390,7 +395,8 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
         const Problem& pr = gp.prob[c.pi];
         const int m0 = ((c.t - pr.tile_begin) / pr.n_tiles) * BT + row_off;
         prefetch_weights(c);
-        for (int kb = 0; kb < kL2Ahead && kb < pr.K / kBlockK; ++kb) ptx::tma_prefetch_l2_2d(&gp.tmx[c.pi], kb * kBlockK, m0);
+        if (pr.K / kBlockK > kL2MinBlocks)
+          for (int kb = 0; kb < kL2Ahead && kb < pr.K / kBlockK; ++kb) ptx::tma_prefetch_l2_2d(&gp.tmx[c.pi], kb * kBlockK, m0);
       }
       while (have && !timed_out) {
         const Problem& pr = gp.prob[c.pi];
@@ -412,8 +418,9 @@ qb_gemm_kernel(const __grid_constant__ GroupedParams gp) {
         for (int kb = 0; kb < k_blocks; ++kb) {
           const int ahead = kb + kL2Ahead;
           if (ahead < k_blocks) {
-            ptx::tma_prefetch_l2_2d(tm, ahead * kBlockK, m0);
-          } else if (tm_nx != nullptr && ahead - k_blocks < kblocks_nx && ahead - k_blocks < kL2Ahead) {
+            if (k_blocks > kL2MinBlocks) ptx::tma_prefetch_l2_2d(tm, ahead * kBlockK, m0);
+          } else if (tm_nx != nullptr && kblocks_nx > kL2MinBlocks && ahead - k_blocks < kblocks_nx &&
+                     ahead - k_blocks < kL2Ahead) {
             ptx::tma_prefetch_l2_2d(tm_nx, (ahead - k_blocks) * kBlockK, m0_nx);
           }
           if (!wait_barrier_relaxed(empty(stage), phase ^ 1u, abort_flag)) {
