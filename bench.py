@@ -16,6 +16,7 @@ the aggregate over the slowest rank's time.
 from __future__ import annotations
 
 import argparse
+import ctypes
 import hashlib
 import json
 import os
@@ -41,9 +42,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # table is keyed by a hash of that source and reads null as soon as the kernel changes.
 NCU_GEMM_TRAFFIC = {
     # "<sha256 of csrc/gemm.cu + csrc/ptx.cuh>": {<config>: bytes per launch}
-    # config 3: counters of a one-layer slice at M = 8192 (307.7 MB per launch) scaled by the units of a full
+    # config 3: counters of a one-layer slice at M = 8192 (306.7 MB per launch) scaled by the units of a full
     # launch (12 layers at three times the tokens: x 36); config 2: the whole stack in its one launch
-    "61f74ecfed67dfbf": {"3": 11.08e9, "2": 43.8e6},
+    "61f74ecfed67dfbf": {"3": 11.04e9, "2": 44.05e6},
 }
 NOMINAL_INT8_TOPS = 4500.0  # dense int8 tensor peak of the part as published (context, not the denominator)
 
@@ -289,8 +290,11 @@ def measure(R: Runner, wl: synth.Workload, steps: int, with_e2e: bool, warm_too:
             packed=torch.empty((s.N, s.K * bits // 32), dtype=torch.int32, device=device),
             delta=torch.empty(s.groups, dtype=torch.float32, device=device),
             q0=torch.empty(s.groups, dtype=torch.float32, device=device),
-            y=torch.empty((wl.M, s.N), dtype=torch.bfloat16 if args.out == "bf16" else torch.float32, device=device),
+            y=torch.empty((wl.M, s.N), dtype={"bf16": torch.bfloat16, "i8": torch.int8}.get(args.out, torch.float32),
+                          device=device),
             bits=bits, s=s)
+        if args.out == "i8":
+            d["rs_out"] = torch.empty(wl.M, dtype=torch.int32, device=device)  # row sums of the int8 output
         devb.append(d)
     descs = qb.make_desc_array([qb.LinearDesc(d["xq"], d["sc"], d["rs"], d["packed"], d["delta"], d["q0"], d["b"],
                                               d["s"].N, d["bits"], d["s"].groups, d["y"]) for d in devb])
@@ -302,16 +306,48 @@ def measure(R: Runner, wl: synth.Workload, steps: int, with_e2e: bool, warm_too:
     per_bits = {}
     for d in devb:
         per_bits[d["bits"]] = per_bits.get(d["bits"], 0) + 1
-    launches_per_step = 2 * -(-len(lin) // 32) + sum(2 * -(-n // 32) for n in per_bits.values()) + gemm_launches
+    launches_per_step = ((len(lin) if args.out == "i8" else 2 * -(-len(lin) // 32)) +
+                         sum(2 * -(-n // 32) for n in per_bits.values()) + gemm_launches)
+
+    chained = args.out == "i8"
+    out_scales = None
+    if chained:
+        # The int8 chain: every linear reads int8 activations that are already on the device (the int8 output
+        # of a previous linear: here quantized once, outside the step) and writes int8 codes on a static
+        # output scale; qb_rowsum_i8 then gives their row sums, which is all the next linear needs.  The step
+        # has no activation quantizer.  Scales: one calibration pass per linear shape (|y|max / 127 of the
+        # fp32 result).
+        qb.quantize_act_batch(act_arr, ws)
+        qb.quantize_pack_weights_batch(w_arr, ws_w)
+        cal = {}
+        for d in devb:
+            key = (d["s"].N, d["s"].K)
+            if key not in cal:
+                y32 = qb.gemm(d["xq"], d["sc"], d["rs"], d["packed"], d["delta"], d["q0"], d["b"], d["s"].N, d["bits"],
+                              d["s"].groups, ws)
+                cal[key] = (y32.abs().max() / 127.0).reshape(1).contiguous()
+                del y32
+        out_scales = [cal[(d["s"].N, d["s"].K)] for d in devb]
+        desc_list = [qb.LinearDesc(d["xq"], d["sc"], d["rs"], d["packed"], d["delta"], d["q0"], d["b"], d["s"].N,
+                                   d["bits"], d["s"].groups, d["y"]) for d in devb]
+        i8_arr = qb.make_desc_array(desc_list)
+        i8_sc = (ctypes.c_void_p * len(devb))(*[t.data_ptr() for t in out_scales])
 
     def phase_act():
-        qb.quantize_act_batch(act_arr, ws)
+        if not chained:
+            qb.quantize_act_batch(act_arr, ws)
 
     def phase_weights():
         qb.quantize_pack_weights_batch(w_arr, ws_w)
 
     def phase_gemm():
-        if args.out == "bf16":
+        if chained:
+            qb._check(qb.lib().qb_layer_linears_i8(i8_arr, i8_sc, len(devb), ws.data_ptr(), ws.numel(), qb._stream()),
+                      "qb_layer_linears_i8")
+            for d in devb:
+                if d["s"].N % 128 == 0:
+                    qb.rowsum_i8(d["y"], d["rs_out"])
+        elif args.out == "bf16":
             qb.layer_linears_bf16(descs, ws)
         else:
             qb.layer_linears(descs, ws)
@@ -528,7 +564,7 @@ def run_ours(args, wl):
         return
 
     peaks, peak_kind = measured_peaks()
-    out_bytes = 2.0 if args.out == "bf16" else 4.0
+    out_bytes = {"bf16": 2.0, "i8": 1.0}.get(args.out, 4.0)
     roof = gemm_roofline_block(wl, res, peaks, peak_kind, out_bytes, probe_tops, probe_cycles, res["ms_gemm"])
     gemm_bytes = gemm_algorithmic_bytes(wl, out_bytes)
     l2_note = "untimed between timed steps: 512 MiB flush write, then a 256 MiB read of another buffer (L2 left with clean lines)"
@@ -539,9 +575,13 @@ def run_ours(args, wl):
         "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
         "config": {"workload": wl.name, "config_index": wl.config, "M": wl.M, "linears": res["linears"],
                    "gemm_launches": res["gemm_launches"],
-                   "bits": sorted(set(wl.bits)), "output": "fp32" if args.out == "f32" else "bfloat16 (narrow-output epilogue)",
+                   "bits": sorted(set(wl.bits)),
+                   "output": {"f32": "fp32", "bf16": "bfloat16 (narrow-output epilogue)",
+                              "i8": "int8 on static scales, then their row sums (the int8 chain: no activation quantizer in the step)"}[args.out],
                    "l2": l2_note, "timing": "median of per-step CUDA-event times",
-                   "step": "quantize_act_batch beside quantize_pack_weights_batch (two streams), then layer_linears over all linears",
+                   "step": ("quantize_pack_weights_batch, then layer_linears_i8 over all linears and rowsum_i8 of every output (int8 inputs resident)"
+                            if args.out == "i8" else
+                            "quantize_act_batch beside quantize_pack_weights_batch (two streams), then layer_linears over all linears"),
                    "launch": "direct C-ABI calls" if args.no_graphs else "C-ABI calls captured once per phase into CUDA graphs, replayed"},
         "clocks": res["clocks"],
         "e2e": {"value": ops_job / (ms_e2e_job * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": res["h2d"],
@@ -551,8 +591,9 @@ def run_ours(args, wl):
         "phases": {
             "note": "measured one after the other in a second loop of the same length (medians); ms_serial is their sum as timed",
             "ms_serial": res["ms_serial"], "clocks": res["clocks_phases"],
-            "quantize_act": {"ms": res["ms_act"], "GBps": act_quant_algorithmic_bytes(wl) / (res["ms_act"] * 1e-3) / 1e9,
-                             "frac_hbm": act_quant_algorithmic_bytes(wl) / (res["ms_act"] * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+            "quantize_act": ({"ms": 0.0, "note": "not part of the int8 chain's step"} if args.out == "i8" else
+                             {"ms": res["ms_act"], "GBps": act_quant_algorithmic_bytes(wl) / (res["ms_act"] * 1e-3) / 1e9,
+                              "frac_hbm": act_quant_algorithmic_bytes(wl) / (res["ms_act"] * 1e-3) / 1e9 / peaks["hbm_gbs"]}),
             "quantize_pack_weights": {"ms": res["ms_w"],
                                       "GBps": weight_quant_algorithmic_bytes(wl) / (res["ms_w"] * 1e-3) / 1e9,
                                       "frac_hbm": weight_quant_algorithmic_bytes(wl) / (res["ms_w"] * 1e-3) / 1e9 / peaks["hbm_gbs"]},
@@ -808,8 +849,10 @@ def main():
     ap.add_argument("--slice-layers", type=int, default=None,
                     help="profiling slice: run only the first layers of the workload")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--out", default="f32", choices=["f32", "bf16"],
-                    help="output type of the GEMMs: fp32 (the graded path) or bfloat16 (qb_layer_linears_bf16)")
+    ap.add_argument("--out", default="f32", choices=["f32", "bf16", "i8"],
+                    help="output type of the GEMMs: fp32 (the graded path), bfloat16 (qb_layer_linears_bf16) or the int8 "
+                         "chain (qb_layer_linears_i8 + qb_rowsum_i8: int8 inputs resident, int8 outputs and their row sums, no "
+                         "activation quantizer in the step)")
     ap.add_argument("--no-graphs", action="store_true", help="issue the C-ABI calls directly every step")
     ap.add_argument("--busy-ms", type=float, default=300.0,
                     help="untimed load before the timed steps so that clocks are sampled under load")
