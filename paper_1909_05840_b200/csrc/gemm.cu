@@ -115,6 +115,7 @@ struct GroupedParams {
   int32_t total_positions;
   int32_t use_order;
   uint16_t order[kMaxOrder];
+  uint8_t order_prob[kMaxOrder];  // with `order`: the problem that owns order[p] (spares every role the search)
 };
 
 // BT: tokens per tile (the N of the MMA).  CG: CTAs that share one MMA (1, or 2 = a CTA pair of a cluster:
@@ -246,7 +247,8 @@ struct TileCursor {
       const uint16_t e = gp.order[p];
       if (e != kNoTile) {
         t = (int)e;
-        break;
+        pi = (int)gp.order_prob[p];
+        return true;
       }
     }
     // the problem that owns tile t: the last one whose first tile is <= t
@@ -1136,6 +1138,13 @@ static qb_status launch_group(const qb_linear_desc* d, const int* idx, int count
         for (size_t i = 0; i < max_len; ++i)
           for (int c = 0; c < grid; ++c)
             gp.order[i * grid + c] = i < lists[c].size() ? (uint16_t)lists[c][i] : kNoTile;
+        // the owner of every listed tile, so that the kernel's roles need not search for it at every tile
+        for (int q = 0; q < (int)(max_len * grid); ++q) {
+          if (gp.order[q] == kNoTile) continue;
+          int pi = 0;
+          while (pi + 1 < count && (int)gp.order[q] >= gp.prob[pi + 1].tile_begin) ++pi;
+          gp.order_prob[q] = (uint8_t)pi;
+        }
         gp.total_positions = (int32_t)(max_len * grid);
         gp.use_order = 1;
       }
