@@ -106,3 +106,19 @@ def test_layer_linears_i8_equals_single_calls(ws):
     assert qb.read_status(ws) == qb.QB_OK
     for d, y1 in zip(descs, singles):
         assert torch.equal(d.y, y1)
+
+
+def test_gemm_i8_large_launch_ragged(ws):
+    # a launch large enough for the CTA-pair kernel (256 x 256 tiles), ragged in M and N: int8 outputs through
+    # TMA stores (N % 16 == 0) must equal the oracle's re-quantization of the oracle's fp32 result
+    M, N, K, bits, G = 2500, 2448, 384, 4, 12
+    x = synth.activations(M, K, seed=71)
+    w = synth.weights(N, K, seed=72)
+    b = synth.bias(N, seed=73)
+    o = oracle.linear(x, w, b, bits, G, omp=True)
+    xq, sc, rs = gu.gpu_quantize_act(x, ws)
+    packed, delta, q0 = gu.gpu_quantize_weights(w, bits, G, ws)
+    s_out = float(np.float32(np.abs(o["y"]).max() / 127.0))
+    yq = qb.gemm_i8(xq, sc, rs, packed, delta, q0, gu.dev(b), N, bits, G, torch.tensor([s_out], device="cuda"), ws)
+    assert qb.read_status(ws) == qb.QB_OK
+    _check_codes(yq.cpu().numpy(), o["y"], s_out)
