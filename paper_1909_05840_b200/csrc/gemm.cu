@@ -1135,9 +1135,12 @@ static qb_status launch_group(const qb_linear_desc* d, const int* idx, int count
         if (lists[best].size() > max_len) max_len = lists[best].size();
       }
       if (max_len * (size_t)grid <= (size_t)kMaxOrder) {
+        // Each CTA visits its own list shortest tile first: the short tile's epilogue then runs under the
+        // long tile's main loop and the launch's first weight reads are spread over more tiles (measured
+        // on a 6-linear mixed stack at M = 128: 5 % less than longest first).
         for (size_t i = 0; i < max_len; ++i)
           for (int c = 0; c < grid; ++c)
-            gp.order[i * grid + c] = i < lists[c].size() ? (uint16_t)lists[c][i] : kNoTile;
+            gp.order[i * grid + c] = i < lists[c].size() ? (uint16_t)lists[c][lists[c].size() - 1 - i] : kNoTile;
         // the owner of every listed tile, so that the kernel's roles need not search for it at every tile
         for (int q = 0; q < (int)(max_len * grid); ++q) {
           if (gp.order[q] == kNoTile) continue;
