@@ -54,9 +54,15 @@ __device__ __forceinline__ void report_status(void* ws, int32_t code, int32_t de
 }
 
 // Monotone map from float bit patterns to unsigned integers (so that integer atomicMax orders floats).
+// Written as integer PTX on the register: as C++ the compiler may turn the sign-bit operations into
+// floating-point negation, which does not keep the bit pattern of a NaN (and the NaN would then sort
+// below the finite values instead of above them).
 __device__ __forceinline__ uint32_t float_to_ordered(float f) {
-  uint32_t b = __float_as_uint(f);
-  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+  uint32_t o;
+  asm("{\n\t.reg .b32 t, m;\n\tmov.b32 t, %1;\n\tshr.s32 m, t, 31;\n\tor.b32 m, m, 0x80000000;\n\txor.b32 %0, t, m;\n\t}"
+      : "=r"(o)
+      : "f"(f));
+  return o;
 }
 __device__ __forceinline__ float ordered_to_float(uint32_t e) {
   uint32_t b = (e & 0x80000000u) ? (e & 0x7fffffffu) : ~e;

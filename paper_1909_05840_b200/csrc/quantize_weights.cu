@@ -760,87 +760,281 @@ weight_fused_kernel(const __grid_constant__ FusedBatch b) {
 }
 
 // ---- register-resident path ---------------------------------------------------------------------------
-// Small groups (up to 72 units = 9,216 weights: one range per output row, or six 768-wide rows) are read
-// from HBM once and never leave the registers: a team of W warps (W = 1, 2 or 4, the same for a launch)
-// loads its group as up to 18 float4 per thread, all in flight at once, reduces the range (warp redux,
-// then the team's named barrier), and packs from the same registers with the unit packer of the two-pass
-// path.  A block holds 4 to 16 teams, so loads of some overlap the packing of others.  With larger
-// teams (the kernel takes up to 16 warps per group) a block has only one or two groups in flight and
-// the load and pack phases no longer overlap: measured slower than the shared-memory ring, which keeps
-// those groups (config 4, 128 groups per matrix: 0.41-0.51 of the copy bandwidth against 0.48-0.54).
-constexpr int kRegUnitsPerThread = 18;
-constexpr int kRegWarps = 16;
-constexpr int kRegThreads = 32 * kRegWarps;
-constexpr int kRegMaxGroupUnits = kRegUnitsPerThread * kRegWarps;  // 288: what the kernel can hold
-constexpr int kRegPathMaxUnits = kRegUnitsPerThread * 4;           // 72: what is sent to it
+// Groups of up to 288 units (36,864 weights: all of BERT's matrices at 128 groups, and anything finer) are
+// read from HBM once and stay in registers between the range and the rounding: 16 warps per CTA, one CTA
+// per SM, every thread holds up to 18 float4 (one warp: 18 consecutive units, 9 KB, all loads in flight at
+// once).  A matrix is served in one of two shapes:
+//   * teams: a group is cut into contiguous slices over W = 1, 2, 4, 8 or 16 warps (the smallest W whose
+//     slices fit), the team agrees on the range through shared memory and a named barrier;
+//   * several groups per warp (groups of at most 9 units: one range per output row, say): a warp holds as
+//     many whole consecutive groups as fit and reduces them one after the other.
+// A CTA item is 16 warps' worth of consecutive groups of one matrix; the items of all matrices of a launch
+// (largest items first, any mix of bit widths: the width is a field of the matrix) form one list that the
+// CTAs stride over, so a mixed-precision stack is one launch.  Codes go through a 768-byte staging area per
+// warp in blocks of six units: the 4k-bit fields laid down in element order are the packed stream for
+// k = 2, 4, 8 (copied out with 16-byte stores) and are regrouped (eight 12-bit fields -> three words) for
+// k = 3.  Ranges supplied by the caller (which need the clamp) and larger groups take the other paths.
+constexpr int kRgUnits = 18;                       // float4 per thread
+constexpr int kRgBlock = 6;                        // units per staging block
+constexpr int kRgWarps = 16;
+constexpr int kRgThreads = 32 * kRgWarps;
+constexpr int kRgMaxGroupUnits = kRgUnits * kRgWarps;  // 288
+constexpr int kRgMaxBatch = 96;                    // matrices per launch
 
+struct RegsItem {
+  const float4* w;
+  uint32_t* packed;
+  float* delta;
+  float* q0;
+  int32_t ug;               // units per group
+  int32_t groups;
+  int32_t item_begin;       // first CTA item of this matrix in the launch's list
+  int32_t groups_per_item;  // (16 / W) * groups_per_warp
+  int16_t team_warps;       // W
+  int16_t groups_per_warp;  // > 1 only with W = 1
+  int16_t slice_units;      // units per warp of a team: ceil(ug / W)
+  int16_t bits;
+};
+
+struct RegsBatch {
+  RegsItem item[kRgMaxBatch];
+  void* ws;
+  int32_t total_items;
+  int32_t count;
+};
+
+// What one warp holds of a CTA item.
+struct RegsSlice {
+  const float4* src;  // first unit of the slice (+ lane)
+  int32_t n;          // units held (0: nothing to do)
+  int32_t it;         // matrix
+  int32_t first_group;
+  int32_t ng;         // groups (several-groups shape), 0 or 1 (teams)
+  int32_t first_unit; // of the slice inside its group (teams)
+};
+
+__device__ __forceinline__ float min3_nan(float a, float b, float c) {
+  float d;
+  asm("min.NaN.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ float max3_nan(float a, float b, float c) {
+  float d;
+  asm("max.NaN.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
+// Four codes of one float4 as a 4k-bit field in the low bits of the result (k < 8: bits from 22 up are
+// left over from the rounding constant and are dropped by the narrow store that follows).
 template <int BITS>
-__global__ void __launch_bounds__(kRegThreads, 1)
-weight_reg_kernel(const __grid_constant__ FusedBatch b) {
-  constexpr int L = (1 << BITS) - 1;
-  constexpr int WORDS = 4 * BITS;
-  __shared__ uint32_t s_hi[2][kRegWarps], s_lo[2][kRegWarps];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int W = b.team_warps;
+__device__ __forceinline__ uint32_t quant_field_open(const float4 v, const float lo, const float inv) {
+  constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23: adding it rounds to an integer, half to even
+  const uint32_t b0 = __float_as_uint(__fadd_rn(__fmul_rn(__fsub_rn(v.x, lo), inv), kMagic));
+  const uint32_t b1 = __float_as_uint(__fadd_rn(__fmul_rn(__fsub_rn(v.y, lo), inv), kMagic));
+  const uint32_t b2 = __float_as_uint(__fadd_rn(__fmul_rn(__fsub_rn(v.z, lo), inv), kMagic));
+  const uint32_t b3 = __float_as_uint(__fadd_rn(__fmul_rn(__fsub_rn(v.w, lo), inv), kMagic));
+  if constexpr (BITS == 8) {
+    return __byte_perm(__byte_perm(b0, b1, 0x0040), __byte_perm(b2, b3, 0x0040), 0x5410);
+  } else {
+    return b0 + (b1 << BITS) + (b2 << (2 * BITS)) + (b3 << (3 * BITS));
+  }
+}
+
+// One staging block (units BLK * 6 ... of the slice): fields into the warp's staging area, then out.
+template <int BITS, int BLK, bool MULTI>
+__device__ __forceinline__ void regs_pack_block(const float4 (&v)[kRgUnits], const int n, float& lo, float& inv,
+                                                const float p_lo, const float p_inv, int& gi, int& next_start,
+                                                const int ug, uint8_t* stg, uint32_t* __restrict__ out, const int lane) {
+#pragma unroll
+  for (int jj = 0; jj < kRgBlock; ++jj) {
+    const int j = BLK * kRgBlock + jj;
+    if (j < n) {
+      if (MULTI) {
+        if (j == next_start) {  // warp-uniform: the next group of this warp begins
+          lo = __shfl_sync(0xffffffffu, p_lo, gi);
+          inv = __shfl_sync(0xffffffffu, p_inv, gi);
+          ++gi;
+          next_start += ug;
+        }
+      }
+      const uint32_t f = quant_field_open<BITS>(v[j], lo, inv);
+      const int fi = jj * 32 + lane;  // field index = element index / 4 inside the block
+      if (BITS == 8) reinterpret_cast<uint32_t*>(stg)[fi] = f;
+      if (BITS == 4 || BITS == 3) reinterpret_cast<uint16_t*>(stg)[fi] = (uint16_t)f;
+      if (BITS == 2) stg[fi] = (uint8_t)f;
+    }
+  }
+  __syncwarp();
+  const int nu = min(kRgBlock, n - BLK * kRgBlock);
+  uint32_t* const o = out + BLK * kRgBlock * 4 * BITS;
+  if (BITS == 3) {
+    // 32 codes = eight 12-bit fields held in 16-bit cells -> three words; four such items per unit
+    if (lane < 4 * nu) {
+      const uint4 q = reinterpret_cast<const uint4*>(stg)[lane];
+      const uint32_t f0 = q.x & 0xffffu, f1 = q.x >> 16, f2 = q.y & 0xffffu, f3 = q.y >> 16;
+      const uint32_t f4 = q.z & 0xffffu, f5 = q.z >> 16, f6 = q.w & 0xffffu, f7 = q.w >> 16;
+      uint32_t* o3 = o + lane * 3;
+      o3[0] = f0 | (f1 << 12) | (f2 << 24);
+      o3[1] = (f2 >> 8) | (f3 << 4) | (f4 << 16) | (f5 << 28);
+      o3[2] = (f5 >> 4) | (f6 << 8) | (f7 << 20);
+    }
+  } else {
+    const int n16 = nu * BITS;  // 16 * BITS bytes per unit
+    const uint4* pk = reinterpret_cast<const uint4*>(stg);
+    uint4* o4 = reinterpret_cast<uint4*>(o);
+#pragma unroll
+    for (int r = 0; r < (kRgBlock * BITS + 31) / 32; ++r) {
+      const int i = r * 32 + lane;
+      if (i < n16) o4[i] = pk[i];
+    }
+  }
+  __syncwarp();  // the staging area is free again
+}
+
+template <int BLK, bool MULTI>
+__device__ __forceinline__ void regs_pack_block_any(const int bits, const float4 (&v)[kRgUnits], const int n, float& lo,
+                                                    float& inv, const float p_lo, const float p_inv, int& gi,
+                                                    int& next_start, const int ug, uint8_t* stg,
+                                                    uint32_t* __restrict__ out, const int lane) {
+  switch (bits) {  // CTA-uniform
+    case 2: regs_pack_block<2, BLK, MULTI>(v, n, lo, inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane); break;
+    case 3: regs_pack_block<3, BLK, MULTI>(v, n, lo, inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane); break;
+    case 4: regs_pack_block<4, BLK, MULTI>(v, n, lo, inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane); break;
+    default: regs_pack_block<8, BLK, MULTI>(v, n, lo, inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane); break;
+  }
+}
+
+__device__ __forceinline__ RegsSlice regs_slice(const RegsBatch& b, const int id, int& it, const int warp,
+                                                const int lane) {
+  RegsSlice s;
+  s.n = 0;
+  s.it = it;
+  s.src = nullptr;
+  s.first_group = 0;
+  s.ng = 0;
+  s.first_unit = 0;
+  if (id >= b.total_items) return s;
+  while (it + 1 < b.count && id >= b.item[it + 1].item_begin) ++it;
+  const RegsItem& m = b.item[it];
+  s.it = it;
+  const int W = m.team_warps;
   const int team = warp / W, tw = warp - team * W;
-  const int teams_per_block = kRegWarps / W;
-  const int64_t total_teams = (int64_t)gridDim.x * teams_per_block;
-  const int first_src = (32 * lane) / (4 * BITS);
+  s.first_group = (id - m.item_begin) * m.groups_per_item + team * m.groups_per_warp;
+  s.ng = min(max(m.groups - s.first_group, 0), (int)m.groups_per_warp);
+  if (s.ng > 0) {
+    if (m.groups_per_warp > 1) {
+      s.n = s.ng * m.ug;
+    } else {
+      s.first_unit = tw * m.slice_units;
+      s.n = min(max(m.ug - s.first_unit, 0), (int)m.slice_units);
+    }
+  }
+  s.src = m.w + ((int64_t)s.first_group * m.ug + s.first_unit) * 32 + lane;
+  return s;
+}
+
+__global__ void __launch_bounds__(kRgThreads, 1)
+weight_regs_kernel(const __grid_constant__ RegsBatch b) {
+  __shared__ __align__(16) uint8_t s_stage[kRgWarps][kRgBlock * 128];
+  __shared__ uint32_t s_hi[2][kRgWarps], s_lo[2][kRgWarps];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  uint8_t* const stg = s_stage[warp];
   const float kInf = __int_as_float(0x7f800000);
-  int it = 0, flip = 0;
-  for (int64_t g = (int64_t)blockIdx.x * teams_per_block + team; g < b.total_groups; g += total_teams) {
-    while (it + 1 < b.count && g >= b.item[it + 1].group_begin) ++it;
-    const WeightItem& m = b.item[it];
-    const int gl = (int)(g - m.group_begin);
-    const int ug = m.rows_per_group * m.units_per_row;
-    const float4* const src = m.w + (int64_t)gl * ug * 32;
-    float4 v[kRegUnitsPerThread];
+  int it = 0, prev_it = 0;
+  for (int id = blockIdx.x, round = 0; id < b.total_items; id += gridDim.x, ++round) {
+    const RegsSlice s = regs_slice(b, id, it, warp, lane);
+    const RegsItem& m = b.item[s.it];
+    // The exchange buffers below are double-buffered per run of items with the same teams; when the
+    // matrix (and with it, possibly, the team size) changes, every warp of the CTA passes here first.
+    if (s.it != prev_it) __syncthreads();
+    prev_it = s.it;
+    const int n = s.n;
+    float4 v[kRgUnits];
 #pragma unroll
-    for (int j = 0; j < kRegUnitsPerThread; ++j) {
-      const int u = j * W + tw;  // warp-uniform
-      if (u < ug) v[j] = __ldg(src + (int64_t)u * 32 + lane);
-    }
-    float lo = kInf, hi = -kInf;
+    for (int j = 0; j < kRgUnits; ++j)
+      if (j < n) v[j] = __ldg(s.src + j * 32);
+    const int W = m.team_warps;
+    const int bits = m.bits;
+    const int L = (1 << bits) - 1;
+    uint32_t* const out = m.packed + ((int64_t)s.first_group * m.ug + s.first_unit) * (4 * bits);
+    if (m.groups_per_warp > 1) {
+      // ---- several whole groups in this warp ----
+      const int ug = m.ug;
+      float lo = kInf, hi = -kInf;
+      uint32_t my_hi = 0, my_lo = 0;
+      int end = ug, gi = 0;
 #pragma unroll
-    for (int j = 0; j < kRegUnitsPerThread; ++j) {
-      if (j * W + tw < ug) {
-        lo = min_nan(min_nan(lo, v[j].x), min_nan(v[j].y, min_nan(v[j].z, v[j].w)));
-        hi = max_nan(max_nan(hi, v[j].x), max_nan(v[j].y, max_nan(v[j].z, v[j].w)));
+      for (int j = 0; j < kRgUnits; ++j) {
+        if (j < n) {
+          lo = min3_nan(min3_nan(lo, v[j].x, v[j].y), v[j].z, v[j].w);
+          hi = max3_nan(max3_nan(hi, v[j].x, v[j].y), v[j].z, v[j].w);
+          if (j + 1 == end) {  // warp-uniform
+            const uint32_t e_hi = __reduce_max_sync(0xffffffffu, float_to_ordered(hi));
+            const uint32_t e_lo = __reduce_max_sync(0xffffffffu, ~float_to_ordered(lo));
+            if (lane == gi) {
+              my_hi = e_hi;
+              my_lo = e_lo;
+            }
+            ++gi;
+            end += ug;
+            lo = kInf;
+            hi = -kInf;
+          }
+        }
       }
-    }
-    // NaN anywhere makes hi NaN (encoded above every number); Inf shows as hi = +Inf or lo = -Inf
-    uint32_t e_hi = __reduce_max_sync(0xffffffffu, float_to_ordered(hi));
-    uint32_t e_lo = __reduce_max_sync(0xffffffffu, ~float_to_ordered(lo));
-    if (W > 1) {
-      if (lane == 0) {
-        s_hi[flip][warp] = e_hi;
-        s_lo[flip][warp] = e_lo;
+      // lane i finishes group i of the warp
+      float p_lo = 0.0f, p_inv = 1.0f;
+      if (lane < s.ng) {
+        const float g_hi = ordered_to_float(my_hi);
+        const float g_lo = ordered_to_float(~my_lo);
+        if (!(fabsf(g_hi) <= 3.402823466e38f && fabsf(g_lo) <= 3.402823466e38f)) report_status(b.ws, QB_ERR_NONFINITE);
+        const GroupParams gp = finish_group(g_lo, g_hi, false, L, s.first_group + lane, m.delta, m.q0, true, b.ws);
+        p_lo = gp.lo;
+        p_inv = gp.inv;
       }
-      asm volatile("bar.sync %0, %1;" ::"r"(1 + team), "r"(32 * W) : "memory");
-      const uint32_t vh = lane < W ? s_hi[flip][team * W + lane] : 0u;
-      const uint32_t vl = lane < W ? s_lo[flip][team * W + lane] : 0u;
-      e_hi = __reduce_max_sync(0xffffffffu, vh);
-      e_lo = __reduce_max_sync(0xffffffffu, vl);
-      flip ^= 1;  // the other half is free again once every warp of the team has passed the next barrier
-    }
-    const float g_hi = ordered_to_float(e_hi);
-    const float g_lo = ordered_to_float(~e_lo);
-    const bool publish = tw == 0 && lane == 0;
-    if (publish && !(fabsf(g_hi) <= 3.402823466e38f && fabsf(g_lo) <= 3.402823466e38f))
-      report_status(b.ws, QB_ERR_NONFINITE);
-    GroupParams gp;
-    if (m.range_lo != nullptr)
-      gp = finish_group(__ldg(m.range_lo + gl), __ldg(m.range_hi + gl), true, L, gl, m.delta, m.q0, publish, b.ws);
-    else
-      gp = finish_group(g_lo, g_hi, false, L, gl, m.delta, m.q0, publish, b.ws);
-    uint32_t* const out = m.packed + (int64_t)gl * ug * WORDS;
+      float c_lo = 0.0f, c_inv = 1.0f;
+      int next_start = 0;
+      gi = 0;
+      if (0 < n) regs_pack_block_any<0, true>(bits, v, n, c_lo, c_inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane);
+      if (kRgBlock < n) regs_pack_block_any<1, true>(bits, v, n, c_lo, c_inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane);
+      if (2 * kRgBlock < n) regs_pack_block_any<2, true>(bits, v, n, c_lo, c_inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane);
+    } else if (s.ng > 0) {
+      // ---- a slice of one group (team-uniform: every warp of the team is here) ----
+      float lo = kInf, hi = -kInf;
 #pragma unroll
-    for (int j = 0; j < kRegUnitsPerThread; ++j) {
-      const int u = j * W + tw;
-      if (u < ug) {
-        const uint32_t word = pack_unit<BITS>(v[j], gp, lane, first_src);
-        if (lane < WORDS) out[(int64_t)u * WORDS + lane] = word;
+      for (int j = 0; j < kRgUnits; ++j) {
+        if (j < n) {
+          lo = min3_nan(min3_nan(lo, v[j].x, v[j].y), v[j].z, v[j].w);
+          hi = max3_nan(max3_nan(hi, v[j].x, v[j].y), v[j].z, v[j].w);
+        }
       }
+      // NaN anywhere makes hi NaN (encoded above every number); Inf shows as hi = +Inf or lo = -Inf
+      uint32_t e_hi = __reduce_max_sync(0xffffffffu, float_to_ordered(hi));
+      uint32_t e_lo = __reduce_max_sync(0xffffffffu, ~float_to_ordered(lo));
+      if (W > 1) {
+        const int flip = round & 1;
+        const int team0 = warp - (warp % W);  // first warp of the team
+        if (lane == 0) {
+          s_hi[flip][warp] = e_hi;
+          s_lo[flip][warp] = e_lo;
+        }
+        asm volatile("bar.sync %0, %1;" ::"r"(1 + team0 / W), "r"(32 * W) : "memory");
+        const uint32_t vh = lane < W ? s_hi[flip][team0 + lane] : 0u;
+        const uint32_t vl = lane < W ? s_lo[flip][team0 + lane] : 0u;
+        e_hi = __reduce_max_sync(0xffffffffu, vh);
+        e_lo = __reduce_max_sync(0xffffffffu, vl);
+      }
+      const float g_hi = ordered_to_float(e_hi);
+      const float g_lo = ordered_to_float(~e_lo);
+      const bool publish = s.first_unit == 0 && lane == 0;
+      if (publish && !(fabsf(g_hi) <= 3.402823466e38f && fabsf(g_lo) <= 3.402823466e38f))
+        report_status(b.ws, QB_ERR_NONFINITE);
+      const GroupParams gp = finish_group(g_lo, g_hi, false, L, s.first_group, m.delta, m.q0, publish, b.ws);
+      float c_lo = gp.lo, c_inv = gp.inv;
+      int gi = 0, next_start = -1;
+      if (0 < n) regs_pack_block_any<0, false>(bits, v, n, c_lo, c_inv, 0.0f, 1.0f, gi, next_start, 0, stg, out, lane);
+      if (kRgBlock < n) regs_pack_block_any<1, false>(bits, v, n, c_lo, c_inv, 0.0f, 1.0f, gi, next_start, 0, stg, out, lane);
+      if (2 * kRgBlock < n) regs_pack_block_any<2, false>(bits, v, n, c_lo, c_inv, 0.0f, 1.0f, gi, next_start, 0, stg, out, lane);
     }
   }
 }
@@ -854,6 +1048,7 @@ struct HostWeight {
   uint32_t* packed;
   float* delta;
   float* q0;
+  int bits;
 };
 
 // Two-pass path: one pair of launches over `count` matrices (<= kMaxWeightBatch) of the same bit width.
@@ -911,6 +1106,64 @@ static qb_status launch_two_pass(const HostWeight* m, int count, int bits, void*
 
 static inline int64_t group_units(const HostWeight& h) { return (h.N / h.groups) * (h.K / 128); }
 
+// Does a matrix take the register-resident path?  (Its own ranges, groups of at most 288 units.)
+static inline bool regs_eligible(const HostWeight& h) {
+  return h.range_lo == nullptr && group_units(h) <= kRgMaxGroupUnits;
+}
+
+// Register-resident path over any number of eligible matrices of any bit widths: launches of up to
+// kRgMaxBatch matrices, inside a launch the matrices with the largest CTA items first.
+static qb_status launch_regs(const HostWeight* m, int count, void* ws, int sm_count, cudaStream_t stream) {
+  struct Shape {
+    int idx, W, gpw, slice, gpi;
+    int64_t item_units;
+  };
+  std::vector<Shape> sh(count);
+  for (int i = 0; i < count; ++i) {
+    const int ug = (int)group_units(m[i]);
+    Shape& s = sh[i];
+    s.idx = i;
+    s.W = 1;
+    while (s.W * kRgUnits < ug) s.W *= 2;
+    s.gpw = s.W == 1 ? std::max(1, kRgUnits / ug) : 1;
+    s.slice = (ug + s.W - 1) / s.W;
+    s.gpi = (kRgWarps / s.W) * s.gpw;
+    s.item_units = (int64_t)std::min(s.gpi, m[i].groups) * ug;
+  }
+  std::stable_sort(sh.begin(), sh.end(), [](const Shape& a, const Shape& b) { return a.item_units > b.item_units; });
+  for (int first = 0; first < count; first += kRgMaxBatch) {
+    const int n = std::min(kRgMaxBatch, count - first);
+    RegsBatch b;
+    memset(&b, 0, sizeof(b));
+    int items = 0;
+    for (int i = 0; i < n; ++i) {
+      const Shape& s = sh[first + i];
+      const HostWeight& h = m[s.idx];
+      RegsItem& it = b.item[i];
+      it.w = reinterpret_cast<const float4*>(h.w);
+      it.packed = h.packed;
+      it.delta = h.delta;
+      it.q0 = h.q0;
+      it.ug = (int32_t)group_units(h);
+      it.groups = h.groups;
+      it.item_begin = items;
+      it.groups_per_item = s.gpi;
+      it.team_warps = (int16_t)s.W;
+      it.groups_per_warp = (int16_t)s.gpw;
+      it.slice_units = (int16_t)s.slice;
+      it.bits = (int16_t)h.bits;
+      items += (h.groups + s.gpi - 1) / s.gpi;
+    }
+    b.ws = ws;
+    b.total_items = items;
+    b.count = n;
+    const unsigned grid = (unsigned)std::min(items, sm_count);
+    weight_regs_kernel<<<grid, kRgThreads, 0, stream>>>(b);
+    QB_CUDA_TRY(cudaGetLastError());
+  }
+  return QB_OK;
+}
+
 // Single-read path over `count` matrices (<= kMaxWeightBatch) whose groups all fit the ring.
 static qb_status launch_fused(const HostWeight* m, int count, int bits, void* ws, int sm_count,
                               cudaStream_t stream) {
@@ -937,23 +1190,6 @@ static qb_status launch_fused(const HostWeight* m, int count, int bits, void* ws
   // small groups: 4 KB slots and small teams (many groups in flight); large groups: 16 KB slots
   int64_t ug_max = 1;
   for (int i = 0; i < count; ++i) ug_max = std::max(ug_max, group_units(m[i]));
-  if (ug_max <= kRegPathMaxUnits) {  // small groups: teams of at most four warps keep them in registers
-    int W = 1;
-    while ((int64_t)W * kRegUnitsPerThread < ug_max) W *= 2;
-    b.team_warps = W;
-    const int teams_per_block = kRegWarps / W;
-    int64_t blocks = (total_groups + teams_per_block - 1) / teams_per_block;
-    if (blocks > sm_count) blocks = sm_count;
-    switch (bits) {
-      case 2: weight_reg_kernel<2><<<(unsigned)blocks, kRegThreads, 0, stream>>>(b); break;
-      case 3: weight_reg_kernel<3><<<(unsigned)blocks, kRegThreads, 0, stream>>>(b); break;
-      case 4: weight_reg_kernel<4><<<(unsigned)blocks, kRegThreads, 0, stream>>>(b); break;
-      case 8: weight_reg_kernel<8><<<(unsigned)blocks, kRegThreads, 0, stream>>>(b); break;
-      default: return QB_ERR_INVALID;
-    }
-    QB_CUDA_TRY(cudaGetLastError());
-    return QB_OK;
-  }
   b.chunk_units = ug_max <= 64 ? 8 : 32;
   b.n_slots = kRingBytes / (b.chunk_units * 512);
   b.team_warps = ug_max <= 16 ? 1 : (ug_max <= 64 ? 2 : (ug_max <= 160 ? 4 : 8));
@@ -1054,8 +1290,15 @@ static void plan_weight_batch(const HostWeight* m, int count, int bits, int sm_c
 
 static qb_status launch_weight_batch(const HostWeight* m, int count, int bits, void* ws, int sm_count,
                                      cudaStream_t stream) {
+  std::vector<HostWeight> regs, rest;
+  for (int i = 0; i < count; ++i) (regs_eligible(m[i]) ? regs : rest).push_back(m[i]);
+  if (!regs.empty()) {
+    qb_status st = launch_regs(regs.data(), (int)regs.size(), ws, sm_count, stream);
+    if (st != QB_OK) return st;
+  }
+  if (rest.empty()) return QB_OK;
   std::vector<WeightJob> jobs;
-  plan_weight_batch(m, count, bits, sm_count, jobs);
+  plan_weight_batch(rest.data(), (int)rest.size(), bits, sm_count, jobs);
   for (const WeightJob& j : jobs) {
     qb_status st = run_weight_job(j, ws, sm_count, sm_count, stream);
     if (st != QB_OK) return st;
@@ -1199,7 +1442,7 @@ static qb_status launch_fake_quantize(const float* w, int64_t N, int64_t K, int 
 qb_status launch_quantize_pack_weights(const float* w, int64_t N, int64_t K, int bits, int groups,
                                        const float* range_lo, const float* range_hi, uint32_t* packed,
                                        float* delta, float* q0, void* ws, int sm_count, cudaStream_t stream) {
-  const HostWeight m{w, N, K, groups, range_lo, range_hi, packed, delta, q0};
+  const HostWeight m{w, N, K, groups, range_lo, range_hi, packed, delta, q0, bits};
   return launch_weight_batch(&m, 1, bits, ws, sm_count, stream);
 }
 
@@ -1262,20 +1505,35 @@ extern "C" qb_status qb_quantize_pack_weights_batch(const qb_weight_desc* descs,
   int sms = 0;
   qb_status st = qb::require_sm100(&sms);
   if (st != QB_OK) return st;
-  // launches: same bit width, at most kMaxWeightBatch matrices each; the range tables of a launch
-  // reuse the head of the workspace (launches on one stream run in order)
-  std::vector<int> order(count);
-  for (int i = 0; i < count; ++i) order[i] = i;
+  // Matrices with their own ranges and groups of at most 288 units: the register-resident path, all bit
+  // widths in the same launches.  The others: launches of one bit width, at most kMaxWeightBatch matrices
+  // each; the range tables of a launch reuse the head of the workspace (launches on one stream run in order).
+  std::vector<qb::HostWeight> regs;
+  std::vector<int> order;
+  for (int i = 0; i < count; ++i) {
+    const qb_weight_desc& d = descs[i];
+    const qb::HostWeight h{d.w, d.N, d.K, d.groups, d.range_lo, d.range_hi, d.packed, d.delta, d.q0, d.bits};
+    if (qb::regs_eligible(h))
+      regs.push_back(h);
+    else
+      order.push_back(i);
+  }
+  if (!regs.empty()) {
+    st = qb::launch_regs(regs.data(), (int)regs.size(), ws, sms, (cudaStream_t)cuda_stream);
+    if (st != QB_OK) return st;
+  }
+  if (order.empty()) return QB_OK;
+  const int rest = (int)order.size();
   std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return descs[a].bits < descs[b].bits; });
   std::vector<qb::WeightJob> jobs;
   int i = 0;
-  while (i < count) {
+  while (i < rest) {
     qb::HostWeight m[qb::kMaxWeightBatch];
     int n = 0;
     const int bits = descs[order[i]].bits;
-    while (i < count && n < qb::kMaxWeightBatch && descs[order[i]].bits == bits) {
+    while (i < rest && n < qb::kMaxWeightBatch && descs[order[i]].bits == bits) {
       const qb_weight_desc& d = descs[order[i]];
-      m[n++] = qb::HostWeight{d.w, d.N, d.K, d.groups, d.range_lo, d.range_hi, d.packed, d.delta, d.q0};
+      m[n++] = qb::HostWeight{d.w, d.N, d.K, d.groups, d.range_lo, d.range_hi, d.packed, d.delta, d.q0, d.bits};
       ++i;
     }
     qb::plan_weight_batch(m, n, bits, sms, jobs);

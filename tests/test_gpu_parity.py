@@ -150,6 +150,54 @@ def test_quantize_weights_single_read_path_edge_cases():
     assert oracle.quantize_weights(w, 3, G)[0] == oracle.ERR_NONFINITE
 
 
+def _check_weight_batch(shapes, seed0, ws_groups=16384):
+    ws_big = qb.workspace(groups=ws_groups)
+    items, host = [], []
+    for i, (N, K, bits, G) in enumerate(shapes):
+        w = synth.weights(N, K, seed=seed0 + 31 * i + N + K + G)
+        packed = gu.poison(torch.empty((N, K * bits // 32), dtype=torch.int32, device="cuda"))
+        delta = gu.poison(torch.empty(G, dtype=torch.float32, device="cuda"))
+        q0 = gu.poison(torch.empty(G, dtype=torch.float32, device="cuda"))
+        items.append((gu.dev(w), bits, G, packed, delta, q0))
+        host.append(w)
+    for _ in range(2):
+        qb.quantize_pack_weights_batch(items, ws_big)
+    assert qb.read_status(ws_big) == qb.QB_OK
+    for (wd, bits, G, packed, delta, q0), w in zip(items, host):
+        st, codes, o_delta, o_q0 = oracle.quantize_weights(w, bits, G)
+        assert np.array_equal(gu.words_np(packed), oracle.pack(codes, bits)), (w.shape, bits, G)
+        assert np.array_equal(delta.cpu().numpy(), o_delta) and np.array_equal(q0.cpu().numpy(), o_q0), (w.shape, bits, G)
+
+
+def test_quantize_weights_register_path_shapes():
+    # one launch, all bit widths: groups cut over 1, 2, 4, 8 and 16 warps with ragged last slices and warps
+    # that get nothing (37 and 130 units), several whole groups per warp (1, 2, 5 and 9 units per group, a
+    # last warp with fewer groups), last CTA items with fewer groups than teams, the largest group (288 units)
+    _check_weight_batch([(760, 640, 3, 40), (1000, 1152, 2, 100), (777, 128, 4, 777), (777, 256, 8, 111),
+                         (96, 2432, 4, 96), (1536, 2304, 2, 384), (130, 1280, 3, 13), (3072, 768, 4, 96),
+                         (64, 4608, 8, 8), (2304, 768, 3, 2304), (37, 128, 2, 1), (74, 640, 8, 2),
+                         (35, 640, 4, 7), (288, 1152, 3, 9), (9, 1152, 2, 9), (130, 128, 4, 1)], seed0=5)
+
+
+def test_quantize_weights_register_path_more_matrices_than_one_launch():
+    # 100 small matrices of mixed widths and group sizes: two launches
+    shapes = [((24 + 8 * (i % 5)), 128 * (1 + i % 3), (2, 3, 4, 8)[i % 4], (1, 2, 4, 8)[(i // 4) % 4]) for i in range(100)]
+    _check_weight_batch(shapes, seed0=77)
+
+
+def test_quantize_weights_register_path_nonfinite():
+    # NaN in a warp that holds several groups, -Inf in one slice of a group cut over eight warps
+    for N, K, G, r, c, bad in ((64, 256, 64, 41, 200, np.nan), (128, 4608, 32, 77, 4000, -np.inf)):
+        w = synth.weights(N, K, seed=N + G)
+        ws_ok, ws_bad = qb.workspace(groups=G), qb.workspace(groups=G)
+        gu.gpu_quantize_weights(w, 4, G, ws_ok)
+        assert qb.read_status(ws_ok) == qb.QB_OK
+        w[r, c] = bad
+        gu.gpu_quantize_weights(w, 4, G, ws_bad)
+        assert qb.read_status(ws_bad) == qb.QB_ERR_NONFINITE
+        assert oracle.quantize_weights(w, 4, G)[0] == oracle.ERR_NONFINITE
+
+
 def test_quantize_weights_edge_cases(ws):
     # constant group, exact ties, caller-supplied (clipping) ranges, non-finite input
     w = synth.weights(8, 128, seed=1)
