@@ -829,10 +829,19 @@ __device__ __forceinline__ float max3_nan(float a, float b, float c) {
 template <int BITS>
 __device__ __forceinline__ uint32_t quant_field_open(const float4 v, const float lo, const float inv) {
   constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23: adding it rounds to an integer, half to even
-  const uint32_t b0 = __float_as_uint(__fadd_rn(__fmul_rn(__fsub_rn(v.x, lo), inv), kMagic));
-  const uint32_t b1 = __float_as_uint(__fadd_rn(__fmul_rn(__fsub_rn(v.y, lo), inv), kMagic));
-  const uint32_t b2 = __float_as_uint(__fadd_rn(__fmul_rn(__fsub_rn(v.z, lo), inv), kMagic));
-  const uint32_t b3 = __float_as_uint(__fadd_rn(__fmul_rn(__fsub_rn(v.w, lo), inv), kMagic));
+  // Two lanes of fp32 per instruction (sub, mul, then the rounding add).  The add is written as a fused
+  // multiply-add with 1.0: a packed mul followed by a packed add gets contracted into one fused operation,
+  // which rounds the exact product instead of the rounded one and lands on the other side of a tie.
+  uint32_t b0, b1, b2, b3;
+  asm("{\n\t.reg .b64 p0, p1, l2, i2, m2, o2;\n\t"
+      "mov.b64 p0, {%4, %5};\n\tmov.b64 p1, {%6, %7};\n\t"
+      "mov.b64 l2, {%8, %8};\n\tmov.b64 i2, {%9, %9};\n\tmov.b64 m2, {%10, %10};\n\tmov.b64 o2, {%11, %11};\n\t"
+      "sub.rn.f32x2 p0, p0, l2;\n\tsub.rn.f32x2 p1, p1, l2;\n\t"
+      "mul.rn.f32x2 p0, p0, i2;\n\tmul.rn.f32x2 p1, p1, i2;\n\t"
+      "fma.rn.f32x2 p0, p0, o2, m2;\n\tfma.rn.f32x2 p1, p1, o2, m2;\n\t"
+      "mov.b64 {%0, %1}, p0;\n\tmov.b64 {%2, %3}, p1;\n\t}"
+      : "=r"(b0), "=r"(b1), "=r"(b2), "=r"(b3)
+      : "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "f"(lo), "f"(inv), "f"(kMagic), "f"(1.0f));
   if constexpr (BITS == 8) {
     return __byte_perm(__byte_perm(b0, b1, 0x0040), __byte_perm(b2, b3, 0x0040), 0x5410);
   } else {
@@ -842,9 +851,10 @@ __device__ __forceinline__ uint32_t quant_field_open(const float4 v, const float
 
 // One staging block (units BLK * 6 ... of the slice): fields into the warp's staging area, then out.
 template <int BITS, int BLK, bool MULTI>
-__device__ __forceinline__ void regs_pack_block(const float4 (&v)[kRgUnits], const int n, float& lo, float& inv,
+__device__ __forceinline__ void regs_pack_block(float4 (&v)[kRgUnits], const int n, float& lo, float& inv,
                                                 const float p_lo, const float p_inv, int& gi, int& next_start,
-                                                const int ug, uint8_t* stg, uint32_t* __restrict__ out, const int lane) {
+                                                const int ug, uint8_t* stg, uint32_t* __restrict__ out, const int lane,
+                                                const float4* __restrict__ next_src, const int next_n) {
 #pragma unroll
   for (int jj = 0; jj < kRgBlock; ++jj) {
     const int j = BLK * kRgBlock + jj;
@@ -863,6 +873,12 @@ __device__ __forceinline__ void regs_pack_block(const float4 (&v)[kRgUnits], con
       if (BITS == 4 || BITS == 3) reinterpret_cast<uint16_t*>(stg)[fi] = (uint16_t)f;
       if (BITS == 2) stg[fi] = (uint8_t)f;
     }
+  }
+  // the registers of this block are free: the same units of the warp's next slice start their way here
+#pragma unroll
+  for (int jj = 0; jj < kRgBlock; ++jj) {
+    const int j = BLK * kRgBlock + jj;
+    if (j < next_n) v[j] = __ldg(next_src + j * 32);
   }
   __syncwarp();
   const int nu = min(kRgBlock, n - BLK * kRgBlock);
@@ -892,15 +908,24 @@ __device__ __forceinline__ void regs_pack_block(const float4 (&v)[kRgUnits], con
 }
 
 template <int BLK, bool MULTI>
-__device__ __forceinline__ void regs_pack_block_any(const int bits, const float4 (&v)[kRgUnits], const int n, float& lo,
+__device__ __forceinline__ void regs_pack_block_any(const int bits, float4 (&v)[kRgUnits], const int n, float& lo,
                                                     float& inv, const float p_lo, const float p_inv, int& gi,
                                                     int& next_start, const int ug, uint8_t* stg,
-                                                    uint32_t* __restrict__ out, const int lane) {
+                                                    uint32_t* __restrict__ out, const int lane,
+                                                    const float4* __restrict__ next_src, const int next_n) {
+  if (BLK * kRgBlock >= n) {  // nothing of this slice here: only the next slice's loads
+#pragma unroll
+    for (int jj = 0; jj < kRgBlock; ++jj) {
+      const int j = BLK * kRgBlock + jj;
+      if (j < next_n) v[j] = __ldg(next_src + j * 32);
+    }
+    return;
+  }
   switch (bits) {  // CTA-uniform
-    case 2: regs_pack_block<2, BLK, MULTI>(v, n, lo, inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane); break;
-    case 3: regs_pack_block<3, BLK, MULTI>(v, n, lo, inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane); break;
-    case 4: regs_pack_block<4, BLK, MULTI>(v, n, lo, inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane); break;
-    default: regs_pack_block<8, BLK, MULTI>(v, n, lo, inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane); break;
+    case 2: regs_pack_block<2, BLK, MULTI>(v, n, lo, inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane, next_src, next_n); break;
+    case 3: regs_pack_block<3, BLK, MULTI>(v, n, lo, inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane, next_src, next_n); break;
+    case 4: regs_pack_block<4, BLK, MULTI>(v, n, lo, inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane, next_src, next_n); break;
+    default: regs_pack_block<8, BLK, MULTI>(v, n, lo, inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane, next_src, next_n); break;
   }
 }
 
@@ -941,18 +966,20 @@ weight_regs_kernel(const __grid_constant__ RegsBatch b) {
   uint8_t* const stg = s_stage[warp];
   const float kInf = __int_as_float(0x7f800000);
   int it = 0, prev_it = 0;
+  float4 v[kRgUnits];
+  RegsSlice s = regs_slice(b, blockIdx.x, it, warp, lane);
+#pragma unroll
+  for (int j = 0; j < kRgUnits; ++j)
+    if (j < s.n) v[j] = __ldg(s.src + j * 32);
   for (int id = blockIdx.x, round = 0; id < b.total_items; id += gridDim.x, ++round) {
-    const RegsSlice s = regs_slice(b, id, it, warp, lane);
     const RegsItem& m = b.item[s.it];
     // The exchange buffers below are double-buffered per run of items with the same teams; when the
     // matrix (and with it, possibly, the team size) changes, every warp of the CTA passes here first.
     if (s.it != prev_it) __syncthreads();
     prev_it = s.it;
     const int n = s.n;
-    float4 v[kRgUnits];
-#pragma unroll
-    for (int j = 0; j < kRgUnits; ++j)
-      if (j < n) v[j] = __ldg(s.src + j * 32);
+    // the warp's slice of the CTA's next item: its loads are issued as the registers come free below
+    const RegsSlice nx = regs_slice(b, id + gridDim.x, it, warp, lane);
     const int W = m.team_warps;
     const int bits = m.bits;
     const int L = (1 << bits) - 1;
@@ -995,9 +1022,9 @@ weight_regs_kernel(const __grid_constant__ RegsBatch b) {
       float c_lo = 0.0f, c_inv = 1.0f;
       int next_start = 0;
       gi = 0;
-      if (0 < n) regs_pack_block_any<0, true>(bits, v, n, c_lo, c_inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane);
-      if (kRgBlock < n) regs_pack_block_any<1, true>(bits, v, n, c_lo, c_inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane);
-      if (2 * kRgBlock < n) regs_pack_block_any<2, true>(bits, v, n, c_lo, c_inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane);
+      regs_pack_block_any<0, true>(bits, v, n, c_lo, c_inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane, nx.src, nx.n);
+      regs_pack_block_any<1, true>(bits, v, n, c_lo, c_inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane, nx.src, nx.n);
+      regs_pack_block_any<2, true>(bits, v, n, c_lo, c_inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane, nx.src, nx.n);
     } else if (s.ng > 0) {
       // ---- a slice of one group (team-uniform: every warp of the team is here) ----
       float lo = kInf, hi = -kInf;
@@ -1032,10 +1059,16 @@ weight_regs_kernel(const __grid_constant__ RegsBatch b) {
       const GroupParams gp = finish_group(g_lo, g_hi, false, L, s.first_group, m.delta, m.q0, publish, b.ws);
       float c_lo = gp.lo, c_inv = gp.inv;
       int gi = 0, next_start = -1;
-      if (0 < n) regs_pack_block_any<0, false>(bits, v, n, c_lo, c_inv, 0.0f, 1.0f, gi, next_start, 0, stg, out, lane);
-      if (kRgBlock < n) regs_pack_block_any<1, false>(bits, v, n, c_lo, c_inv, 0.0f, 1.0f, gi, next_start, 0, stg, out, lane);
-      if (2 * kRgBlock < n) regs_pack_block_any<2, false>(bits, v, n, c_lo, c_inv, 0.0f, 1.0f, gi, next_start, 0, stg, out, lane);
+      regs_pack_block_any<0, false>(bits, v, n, c_lo, c_inv, 0.0f, 1.0f, gi, next_start, 0, stg, out, lane, nx.src, nx.n);
+      regs_pack_block_any<1, false>(bits, v, n, c_lo, c_inv, 0.0f, 1.0f, gi, next_start, 0, stg, out, lane, nx.src, nx.n);
+      regs_pack_block_any<2, false>(bits, v, n, c_lo, c_inv, 0.0f, 1.0f, gi, next_start, 0, stg, out, lane, nx.src, nx.n);
+    } else {
+      // nothing of this item here (a last item with fewer groups than teams): only the next slice's loads
+#pragma unroll
+      for (int j = 0; j < kRgUnits; ++j)
+        if (j < nx.n) v[j] = __ldg(nx.src + j * 32);
     }
+    s = nx;
   }
 }
 

@@ -185,6 +185,35 @@ def test_quantize_weights_register_path_more_matrices_than_one_launch():
     _check_weight_batch(shapes, seed0=77)
 
 
+@pytest.mark.parametrize("bits", BITS)
+def test_quantize_weights_products_that_round_onto_ties(bits):
+    # Every weight sits within a few ulp of the midpoint between two grid points, so that thousands of
+    # products (w - q0) * (1/Delta) round to k + 0.5 exactly while the exact product does not: a fused
+    # multiply-add in the rounding step, or a rounding other than half-to-even, shows here.
+    N, K, G = 96, 1152, 12
+    rng = np.random.default_rng(100 + bits)
+    L = (1 << bits) - 1
+    w = np.empty((N, K), np.float32)
+    R = N // G
+    for g in range(G):
+        lo = np.float32(-0.05 - 0.02 * rng.random())
+        hi = np.float32(0.04 + 0.03 * rng.random())
+        d = np.float32((hi - lo) / np.float32(L))
+        m = rng.integers(0, L, size=(R, K)).astype(np.float32)
+        x = (lo + (m + np.float32(0.5)) * d).astype(np.float32)
+        x = (x.view(np.int32) + rng.integers(-4, 5, size=x.shape).astype(np.int32)).view(np.float32)
+        x[0, 0], x[0, 1] = lo, hi
+        w[g * R:(g + 1) * R] = np.clip(x, lo, hi)
+    ws1 = qb.workspace(groups=G)
+    packed, delta, q0 = gu.gpu_quantize_weights(w, bits, G, ws1)
+    assert qb.read_status(ws1) == qb.QB_OK
+    st, codes, o_delta, o_q0 = oracle.quantize_weights(w, bits, G)
+    prod = (w.reshape(G, -1) - o_q0[:, None]) * (np.float32(1.0) / o_delta)[:, None]
+    assert np.count_nonzero(prod - np.floor(prod) == 0.5) > 1000
+    assert np.array_equal(delta.cpu().numpy(), o_delta) and np.array_equal(q0.cpu().numpy(), o_q0)
+    assert np.array_equal(gu.words_np(packed), oracle.pack(codes, bits))
+
+
 def test_quantize_weights_register_path_nonfinite():
     # NaN in a warp that holds several groups, -Inf in one slice of a group cut over eight warps
     for N, K, G, r, c, bad in ((64, 256, 64, 41, 200, np.nan), (128, 4608, 32, 77, 4000, -np.inf)):
