@@ -42,9 +42,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # table is keyed by a hash of that source and reads null as soon as the kernel changes.
 NCU_GEMM_TRAFFIC = {
     # "<sha256 of csrc/gemm.cu + csrc/ptx.cuh>": {<config>: bytes per launch}
-    # config 3: counters of a one-layer slice at M = 8192 (306.7 MB per launch) scaled by the units of a full
+    # config 3: counters of a one-layer slice at M = 8192 (315.0 MB per launch) scaled by the units of a full
     # launch (12 layers at three times the tokens: x 36); config 2: the whole stack in its one launch
-    "524fcd17e5ed7905": {"3": 11.04e9, "2": 43.85e6},
+    "96b38d2a74063ce3": {"3": 11.34e9, "2": 44.34e6},
 }
 NOMINAL_INT8_TOPS = 4500.0  # dense int8 tensor peak of the part as published (context, not the denominator)
 
@@ -303,11 +303,8 @@ def measure(R: Runner, wl: synth.Workload, steps: int, with_e2e: bool, warm_too:
                                        for d in devb])
     # kernels launched per step, counted from the library's own launch plan for these descriptors
     gemm_launches = qb.layer_linears_launch_count(descs)
-    per_bits = {}
-    for d in devb:
-        per_bits[d["bits"]] = per_bits.get(d["bits"], 0) + 1
-    launches_per_step = ((len(lin) if args.out == "i8" else 2 * -(-len(lin) // 32)) +
-                         sum(2 * -(-n // 32) for n in per_bits.values()) + gemm_launches)
+    weight_launches = qb.quantize_pack_weights_launch_count(w_arr)
+    launches_per_step = ((len(lin) if args.out == "i8" else 2 * -(-len(lin) // 32)) + weight_launches + gemm_launches)
 
     chained = args.out == "i8"
     out_scales = None

@@ -103,7 +103,10 @@ qb_status qb_quantize_act(const float* x, int64_t M, int64_t K, int8_t* xq, floa
  *   range_lo, range_hi: dev fp32 [G] or both NULL.  When given they replace the group's min and
  *            max (Appendix A: the range "can be a subinterval of [min, max]"); values outside are
  *            clamped.  They must be finite with range_lo <= range_hi.
- * Two kernels: per-group min/max reduction into the workspace, then round/clamp/pack.
+ * One kernel (the weights are read once and stay in registers between the range and the rounding)
+ * when the groups have at most 36,864 weights each and the range is the group's own; otherwise two
+ * kernels (per-group min/max reduction into the workspace, then round/clamp/pack), or one that stages
+ * the group in shared memory (caller-supplied ranges, groups of up to 49,152 weights).
  */
 qb_status qb_quantize_pack_weights(const float* w, int64_t N, int64_t K, int bits, int groups,
                                    const float* range_lo, const float* range_hi, uint32_t* packed,
@@ -137,12 +140,14 @@ typedef struct {
  * tensor: BERT's matrices are a few MB each, so single launches are bound by launch latency, not by
  * memory bandwidth.  `descs` is a HOST array; every element is validated before anything is launched;
  * each result equals the single call on the same arguments bit for bit.  Each activation tensor keeps
- * its own scale (per-tensor quantization).  Weight matrices of different bit widths may be mixed;
- * each bit width gets its own launches, and when these are several small single-read launches (a
- * mixed-precision stack) they run side by side on streams the library creates once per device
- * (host objects only), forking from and joining `cuda_stream` inside the call (after the fork every
- * side stream is joined, also when a launch in between fails; the fork / launch / join sequence is
- * serialised per device, so concurrent calls from several host threads are safe).
+ * its own scale (per-tensor quantization).  Weight matrices of different bit widths may be mixed:
+ * all matrices whose groups have at most 36,864 weights and take their own [min, max] go into one
+ * launch per 96 matrices, whatever their widths (a mixed-precision stack is one launch).  The others
+ * get launches per bit width; when these are several small single-read launches they run side by
+ * side on streams the library creates once per device (host objects only), forking from and joining
+ * `cuda_stream` inside the call (after the fork every side stream is joined, also when a launch in
+ * between fails; the fork / launch / join sequence is serialised per device, so concurrent calls
+ * from several host threads are safe).
  * Workspace: qb_workspace_bytes(0, 0, 0, 0, G) bytes with G = max(32, sum of `groups` over the batch).
  */
 qb_status qb_quantize_act_batch(const qb_act_desc* descs /*host*/, int32_t count, void* ws, size_t ws_bytes,
@@ -228,6 +233,14 @@ typedef struct {
  */
 qb_status qb_layer_linears(const qb_linear_desc* descs /*host*/, int32_t count, void* ws,
                            size_t ws_bytes, void* cuda_stream);
+
+/*
+ * How many kernel launches qb_quantize_pack_weights_batch issues for these matrices: host arithmetic on
+ * the descriptors only (shapes, groups, bit widths, whether ranges are supplied), no GPU work.  (No
+ * counterpart in the paper; for callers that count or budget launches.)  The plan is the one of a
+ * 148-SM device.  Returns 0 for a null or empty batch or a descriptor with impossible shapes.
+ */
+int32_t qb_quantize_pack_weights_launch_count(const qb_weight_desc* descs /*host*/, int32_t count);
 
 /*
  * How many GEMM kernel launches qb_layer_linears (and its narrow-output forms) issue for this stack: host

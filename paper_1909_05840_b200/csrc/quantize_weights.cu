@@ -1516,6 +1516,41 @@ extern "C" qb_status qb_quantize_pack_weights(const float* w, int64_t N, int64_t
                                           (cudaStream_t)cuda_stream);
 }
 
+namespace qb {
+
+// The launch plan of a batch: the matrices of the register-resident path, and the jobs of the others.
+static void plan_batch(const qb_weight_desc* descs, int count, int sms, std::vector<HostWeight>& regs,
+                       std::vector<WeightJob>& jobs) {
+  // Matrices with their own ranges and groups of at most 288 units: the register-resident path, all bit
+  // widths in the same launches.  The others: launches of one bit width, at most kMaxWeightBatch matrices
+  // each; the range tables of a launch reuse the head of the workspace (launches on one stream run in order).
+  std::vector<int> order;
+  for (int i = 0; i < count; ++i) {
+    const qb_weight_desc& d = descs[i];
+    const HostWeight h{d.w, d.N, d.K, d.groups, d.range_lo, d.range_hi, d.packed, d.delta, d.q0, d.bits};
+    if (regs_eligible(h))
+      regs.push_back(h);
+    else
+      order.push_back(i);
+  }
+  const int rest = (int)order.size();
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return descs[a].bits < descs[b].bits; });
+  int i = 0;
+  while (i < rest) {
+    HostWeight m[kMaxWeightBatch];
+    int n = 0;
+    const int bits = descs[order[i]].bits;
+    while (i < rest && n < kMaxWeightBatch && descs[order[i]].bits == bits) {
+      const qb_weight_desc& d = descs[order[i]];
+      m[n++] = HostWeight{d.w, d.N, d.K, d.groups, d.range_lo, d.range_hi, d.packed, d.delta, d.q0, d.bits};
+      ++i;
+    }
+    plan_weight_batch(m, n, bits, sms, jobs);
+  }
+}
+
+}  // namespace qb
+
 extern "C" qb_status qb_quantize_pack_weights_batch(const qb_weight_desc* descs, int32_t count, void* ws,
                                                     size_t ws_bytes, void* cuda_stream) {
   if (!descs || count <= 0) {
@@ -1538,40 +1573,29 @@ extern "C" qb_status qb_quantize_pack_weights_batch(const qb_weight_desc* descs,
   int sms = 0;
   qb_status st = qb::require_sm100(&sms);
   if (st != QB_OK) return st;
-  // Matrices with their own ranges and groups of at most 288 units: the register-resident path, all bit
-  // widths in the same launches.  The others: launches of one bit width, at most kMaxWeightBatch matrices
-  // each; the range tables of a launch reuse the head of the workspace (launches on one stream run in order).
   std::vector<qb::HostWeight> regs;
-  std::vector<int> order;
-  for (int i = 0; i < count; ++i) {
-    const qb_weight_desc& d = descs[i];
-    const qb::HostWeight h{d.w, d.N, d.K, d.groups, d.range_lo, d.range_hi, d.packed, d.delta, d.q0, d.bits};
-    if (qb::regs_eligible(h))
-      regs.push_back(h);
-    else
-      order.push_back(i);
-  }
+  std::vector<qb::WeightJob> jobs;
+  qb::plan_batch(descs, count, sms, regs, jobs);
   if (!regs.empty()) {
     st = qb::launch_regs(regs.data(), (int)regs.size(), ws, sms, (cudaStream_t)cuda_stream);
     if (st != QB_OK) return st;
   }
-  if (order.empty()) return QB_OK;
-  const int rest = (int)order.size();
-  std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return descs[a].bits < descs[b].bits; });
-  std::vector<qb::WeightJob> jobs;
-  int i = 0;
-  while (i < rest) {
-    qb::HostWeight m[qb::kMaxWeightBatch];
-    int n = 0;
-    const int bits = descs[order[i]].bits;
-    while (i < rest && n < qb::kMaxWeightBatch && descs[order[i]].bits == bits) {
-      const qb_weight_desc& d = descs[order[i]];
-      m[n++] = qb::HostWeight{d.w, d.N, d.K, d.groups, d.range_lo, d.range_hi, d.packed, d.delta, d.q0, d.bits};
-      ++i;
-    }
-    qb::plan_weight_batch(m, n, bits, sms, jobs);
-  }
+  if (jobs.empty()) return QB_OK;
   return qb::run_weight_jobs(jobs, ws, sms, (cudaStream_t)cuda_stream);
+}
+
+extern "C" int32_t qb_quantize_pack_weights_launch_count(const qb_weight_desc* descs, int32_t count) {
+  if (!descs || count <= 0) return 0;
+  for (int i = 0; i < count; ++i) {
+    const qb_weight_desc& d = descs[i];
+    if (d.N <= 0 || d.K <= 0 || d.groups < 1 || d.N % d.groups != 0 || d.K % 128 != 0) return 0;
+  }
+  std::vector<qb::HostWeight> regs;
+  std::vector<qb::WeightJob> jobs;
+  qb::plan_batch(descs, count, 148, regs, jobs);
+  int32_t n = (int32_t)((regs.size() + qb::kRgMaxBatch - 1) / qb::kRgMaxBatch);
+  for (const qb::WeightJob& j : jobs) n += j.single_read ? 1 : 2;
+  return n;
 }
 
 extern "C" qb_status qb_fake_quantize_weights(const float* w, int64_t N, int64_t K, int bits, int groups,

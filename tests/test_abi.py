@@ -118,3 +118,22 @@ def test_no_cpu_fallback_without_a_device(lib):
     A = 0x1000
     st = lib.qb_quantize_act(A, 4, 128, A, A, A, A, qb.workspace_bytes(), None)
     assert st == qb.QB_ERR_CUDA  # valid arguments, but no sm_100 device: an error, never a CPU path
+
+
+def test_weight_launch_count_is_host_arithmetic(lib):
+    """qb_quantize_pack_weights_launch_count plans on the host: no device, no pointer is touched."""
+    def arr_of(shapes):
+        arr = (qb.WeightDescC * len(shapes))()
+        for i, (N, K, bits, G, ranged) in enumerate(shapes):
+            r = 0x1000 if ranged else None
+            arr[i] = qb.WeightDescC(0x1000, N, K, bits, G, r, r, 0x1000, 0x1000, 0x1000)
+        return arr
+    base = [(2304, 768, 384), (768, 768, 128), (3072, 768, 128), (768, 3072, 128)]
+    mixed = [(N, K, (2, 3, 4, 8)[l % 4], G, False) for l in range(12) for (N, K, G) in base]
+    assert lib.qb_quantize_pack_weights_launch_count(arr_of(mixed), len(mixed)) == 1      # a mixed-precision stack: one launch
+    assert lib.qb_quantize_pack_weights_launch_count(arr_of(mixed * 3), 3 * len(mixed)) == 2  # 144 matrices: 96 + 48
+    assert lib.qb_quantize_pack_weights_launch_count(arr_of([(768, 768, 4, 1, False)]), 1) == 2  # one range per tensor: two passes
+    both = [(768, 768, 4, 128, False), (768, 768, 4, 1, False)]
+    assert lib.qb_quantize_pack_weights_launch_count(arr_of(both), 2) == 3
+    assert lib.qb_quantize_pack_weights_launch_count(None, 0) == 0
+    assert lib.qb_quantize_pack_weights_launch_count(arr_of([(768, 700, 4, 128, False)]), 1) == 0
