@@ -1,10 +1,16 @@
 // qb_quantize_pack_weights(_batch): group-wise uniform quantizer Q (Section 3.3, Appendix A) and dense
-// k-bit packing (Table 1 counts exactly k bits per weight), for one matrix or a batch of matrices of
-// the same bit width in one pair of launches.
+// k-bit packing (Table 1 counts exactly k bits per weight), for one matrix or a batch of matrices.
 //
-// The matrices of a launch are walked as one sequence of "units" of 128 consecutive elements of one
-// row (one float4 per lane, fully coalesced; K % 128 == 0 so a unit never crosses a row).  Each warp
-// owns a contiguous run of units, so it crosses few group (and matrix) boundaries.
+// Three paths, chosen per matrix on the host:
+//   weight_regs_kernel   groups of up to 288 units with their own [min, max]: one read of W, the group
+//                        stays in registers between the range and the rounding; any bit widths in one launch.
+//   weight_fused_kernel  groups of up to 384 units, also with caller-supplied ranges: one read of W through
+//                        a shared-memory ring.
+//   two passes           everything else (a range per tensor, say), below.
+//
+// Two-pass path: the matrices of a launch are walked as one sequence of "units" of 128 consecutive
+// elements of one row (one float4 per lane, fully coalesced; K % 128 == 0 so a unit never crosses a row).
+// Each warp owns a contiguous run of units, so it crosses few group (and matrix) boundaries.
 //
 // Kernel 1  weight_range_kernel  running min/max per lane, warp reduction when the group changes,
 //                                atomicMax on order-preserving integer encodings in the workspace
@@ -13,6 +19,7 @@
 //                                codes per lane, and assembles the unit's 4k output words with warp
 //                                shuffles so that the stores are contiguous 16k-byte runs.
 #include <algorithm>
+#include <atomic>
 #include <cstring>
 #include <mutex>
 #include <vector>
@@ -929,8 +936,9 @@ __device__ __forceinline__ void regs_pack_block_any(const int bits, float4 (&v)[
   }
 }
 
+template <bool CLUSTER>
 __device__ __forceinline__ RegsSlice regs_slice(const RegsBatch& b, const int id, int& it, const int warp,
-                                                const int lane) {
+                                                const int lane, const int crank) {
   RegsSlice s;
   s.n = 0;
   s.it = it;
@@ -942,49 +950,76 @@ __device__ __forceinline__ RegsSlice regs_slice(const RegsBatch& b, const int id
   while (it + 1 < b.count && id >= b.item[it + 1].item_begin) ++it;
   const RegsItem& m = b.item[it];
   s.it = it;
-  const int W = m.team_warps;
-  const int team = warp / W, tw = warp - team * W;
-  s.first_group = (id - m.item_begin) * m.groups_per_item + team * m.groups_per_warp;
-  s.ng = min(max(m.groups - s.first_group, 0), (int)m.groups_per_warp);
-  if (s.ng > 0) {
-    if (m.groups_per_warp > 1) {
-      s.n = s.ng * m.ug;
-    } else {
-      s.first_unit = tw * m.slice_units;
-      s.n = min(max(m.ug - s.first_unit, 0), (int)m.slice_units);
+  if (CLUSTER) {
+    // one group per cluster item, cut into slices over the 16 warps of each of the cluster's CTAs
+    s.first_group = id - m.item_begin;
+    s.ng = 1;
+    s.first_unit = (crank * kRgWarps + warp) * m.slice_units;
+    s.n = min(max(m.ug - s.first_unit, 0), (int)m.slice_units);
+  } else {
+    const int W = m.team_warps;
+    const int team = warp / W, tw = warp - team * W;
+    s.first_group = (id - m.item_begin) * m.groups_per_item + team * m.groups_per_warp;
+    s.ng = min(max(m.groups - s.first_group, 0), (int)m.groups_per_warp);
+    if (s.ng > 0) {
+      if (m.groups_per_warp > 1) {
+        s.n = s.ng * m.ug;
+      } else {
+        s.first_unit = tw * m.slice_units;
+        s.n = min(max(m.ug - s.first_unit, 0), (int)m.slice_units);
+      }
     }
   }
   s.src = m.w + ((int64_t)s.first_group * m.ug + s.first_unit) * 32 + lane;
   return s;
 }
 
+__device__ __forceinline__ uint32_t cluster_size() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v) {
+  asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
+}
+
+// CLUSTER = false: the kernel described above.  CLUSTER = true: groups of 289 to 2,304 units; a thread-block
+// cluster of 2 to 8 CTAs (the launch's cluster size) holds one group, every CTA reduces its 16 slices,
+// writes its range into every CTA's shared memory and the cluster's barrier publishes them.  Every CTA of a
+// cluster runs the same number of items, so the barriers pair up; the last one also keeps a CTA's shared
+// memory alive until no peer writes to it any more.
+template <bool CLUSTER>
 __global__ void __launch_bounds__(kRgThreads, 1)
 weight_regs_kernel(const __grid_constant__ RegsBatch b) {
   __shared__ __align__(16) uint8_t s_stage[kRgWarps][kRgBlock * 128];
   __shared__ uint32_t s_hi[2][kRgWarps], s_lo[2][kRgWarps];
+  __shared__ uint32_t x_hi[2][8], x_lo[2][8];  // CLUSTER: the ranges of the cluster's CTAs
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   uint8_t* const stg = s_stage[warp];
   const float kInf = __int_as_float(0x7f800000);
+  const int csize = CLUSTER ? (int)cluster_size() : 1;
+  const int crank = CLUSTER ? (int)ptx::cluster_ctarank() : 0;
+  const int id0 = (int)blockIdx.x / csize, stride = (int)gridDim.x / csize;  // items go to clusters
   int it = 0, prev_it = 0;
   float4 v[kRgUnits];
-  RegsSlice s = regs_slice(b, blockIdx.x, it, warp, lane);
+  RegsSlice s = regs_slice<CLUSTER>(b, id0, it, warp, lane, crank);
 #pragma unroll
   for (int j = 0; j < kRgUnits; ++j)
     if (j < s.n) v[j] = __ldg(s.src + j * 32);
-  for (int id = blockIdx.x, round = 0; id < b.total_items; id += gridDim.x, ++round) {
+  for (int id = id0, round = 0; id < b.total_items; id += stride, ++round) {
     const RegsItem& m = b.item[s.it];
     // The exchange buffers below are double-buffered per run of items with the same teams; when the
     // matrix (and with it, possibly, the team size) changes, every warp of the CTA passes here first.
-    if (s.it != prev_it) __syncthreads();
+    if (!CLUSTER && s.it != prev_it) __syncthreads();
     prev_it = s.it;
     const int n = s.n;
     // the warp's slice of the CTA's next item: its loads are issued as the registers come free below
-    const RegsSlice nx = regs_slice(b, id + gridDim.x, it, warp, lane);
+    const RegsSlice nx = regs_slice<CLUSTER>(b, id + stride, it, warp, lane, crank);
     const int W = m.team_warps;
     const int bits = m.bits;
     const int L = (1 << bits) - 1;
     uint32_t* const out = m.packed + ((int64_t)s.first_group * m.ug + s.first_unit) * (4 * bits);
-    if (m.groups_per_warp > 1) {
+    if (!CLUSTER && m.groups_per_warp > 1) {
       // ---- several whole groups in this warp ----
       const int ug = m.ug;
       float lo = kInf, hi = -kInf;
@@ -1038,7 +1073,23 @@ weight_regs_kernel(const __grid_constant__ RegsBatch b) {
       // NaN anywhere makes hi NaN (encoded above every number); Inf shows as hi = +Inf or lo = -Inf
       uint32_t e_hi = __reduce_max_sync(0xffffffffu, float_to_ordered(hi));
       uint32_t e_lo = __reduce_max_sync(0xffffffffu, ~float_to_ordered(lo));
-      if (W > 1) {
+      if (CLUSTER) {
+        const int flip = round & 1;
+        if (lane == 0) {
+          s_hi[flip][warp] = e_hi;
+          s_lo[flip][warp] = e_lo;
+        }
+        __syncthreads();
+        e_hi = __reduce_max_sync(0xffffffffu, lane < kRgWarps ? s_hi[flip][lane] : 0u);
+        e_lo = __reduce_max_sync(0xffffffffu, lane < kRgWarps ? s_lo[flip][lane] : 0u);
+        if (warp == 0 && lane < csize) {  // this CTA's range into slot `crank` of CTA `lane`
+          st_cluster_u32(ptx::map_to_cta(ptx::smem_u32(&x_hi[flip][crank]), (uint32_t)lane), e_hi);
+          st_cluster_u32(ptx::map_to_cta(ptx::smem_u32(&x_lo[flip][crank]), (uint32_t)lane), e_lo);
+        }
+        ptx::cluster_sync_all();
+        e_hi = __reduce_max_sync(0xffffffffu, lane < csize ? x_hi[flip][lane] : 0u);
+        e_lo = __reduce_max_sync(0xffffffffu, lane < csize ? x_lo[flip][lane] : 0u);
+      } else if (W > 1) {
         const int flip = round & 1;
         const int team0 = warp - (warp % W);  // first warp of the team
         if (lane == 0) {
@@ -1070,6 +1121,7 @@ weight_regs_kernel(const __grid_constant__ RegsBatch b) {
     }
     s = nx;
   }
+  if (CLUSTER) ptx::cluster_sync_all();
 }
 
 struct HostWeight {
@@ -1139,14 +1191,113 @@ static qb_status launch_two_pass(const HostWeight* m, int count, int bits, void*
 
 static inline int64_t group_units(const HostWeight& h) { return (h.N / h.groups) * (h.K / 128); }
 
-// Does a matrix take the register-resident path?  (Its own ranges, groups of at most 288 units.)
+// Does a matrix take the register-resident path?  (Its own ranges; groups of at most 288 units in one
+// CTA, up to 2,304 in a cluster of up to 8 CTAs.)
+constexpr int kRgMaxCluster = 8;
+static inline int regs_cluster_size(const HostWeight& h) {
+  return (int)((group_units(h) + kRgMaxGroupUnits - 1) / kRgMaxGroupUnits);
+}
 static inline bool regs_eligible(const HostWeight& h) {
-  return h.range_lo == nullptr && group_units(h) <= kRgMaxGroupUnits;
+  return h.range_lo == nullptr && group_units(h) <= (int64_t)kRgMaxGroupUnits * kRgMaxCluster;
+}
+
+// Clusters of `cl` CTAs that can be resident at once (asked once per device and cluster size).
+static qb_status regs_max_clusters(int cl, int* out) {
+  static std::atomic<int> cached[64][kRgMaxCluster + 1] = {};
+  int dev = 0;
+  QB_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) {
+    set_last_error("device ordinal %d out of range", dev);
+    return QB_ERR_CUDA;
+  }
+  int n = cached[dev][cl].load(std::memory_order_acquire);
+  if (n == 0) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)cl * 64u);
+    cfg.blockDim = dim3(kRgThreads);
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = (unsigned)cl;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    QB_CUDA_TRY(cudaOccupancyMaxActiveClusters(&n, weight_regs_kernel<true>, &cfg));
+    if (n < 1) {
+      set_last_error("no cluster of %d CTAs fits the device", cl);
+      return QB_ERR_CUDA;
+    }
+    cached[dev][cl].store(n, std::memory_order_release);
+  }
+  *out = n;
+  return QB_OK;
+}
+
+// Matrices whose groups need a cluster of `cl` CTAs (289 to 2,304 units per group), any bit widths: one
+// group per cluster item.
+static qb_status launch_regs_cluster(const HostWeight* m, int count, int cl, void* ws, cudaStream_t stream) {
+  int max_clusters = 0;
+  qb_status st = regs_max_clusters(cl, &max_clusters);
+  if (st != QB_OK) return st;
+  for (int first = 0; first < count; first += kRgMaxBatch) {
+    const int n = std::min(kRgMaxBatch, count - first);
+    RegsBatch b;
+    memset(&b, 0, sizeof(b));
+    int items = 0;
+    for (int i = 0; i < n; ++i) {
+      const HostWeight& h = m[first + i];
+      RegsItem& it = b.item[i];
+      const int ug = (int)group_units(h);
+      it.w = reinterpret_cast<const float4*>(h.w);
+      it.packed = h.packed;
+      it.delta = h.delta;
+      it.q0 = h.q0;
+      it.ug = ug;
+      it.groups = h.groups;
+      it.item_begin = items;
+      it.groups_per_item = 1;
+      it.team_warps = (int16_t)kRgWarps;
+      it.groups_per_warp = 1;
+      it.slice_units = (int16_t)((ug + kRgWarps * cl - 1) / (kRgWarps * cl));
+      it.bits = (int16_t)h.bits;
+      items += h.groups;
+    }
+    b.ws = ws;
+    b.total_items = items;
+    b.count = n;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(std::min(items, max_clusters) * cl));
+    cfg.blockDim = dim3(kRgThreads);
+    cfg.stream = stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = (unsigned)cl;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    QB_CUDA_TRY(cudaLaunchKernelEx(&cfg, weight_regs_kernel<true>, b));
+  }
+  return QB_OK;
 }
 
 // Register-resident path over any number of eligible matrices of any bit widths: launches of up to
-// kRgMaxBatch matrices, inside a launch the matrices with the largest CTA items first.
-static qb_status launch_regs(const HostWeight* m, int count, void* ws, int sm_count, cudaStream_t stream) {
+// kRgMaxBatch matrices, inside a launch the matrices with the largest CTA items first.  Matrices whose
+// groups need a cluster go to launches of their cluster size.
+static qb_status launch_regs(const HostWeight* m_all, int count_all, void* ws, int sm_count, cudaStream_t stream) {
+  std::vector<HostWeight> single, clustered[kRgMaxCluster + 1];
+  for (int i = 0; i < count_all; ++i) {
+    const int cl = regs_cluster_size(m_all[i]);
+    (cl <= 1 ? single : clustered[cl]).push_back(m_all[i]);
+  }
+  for (int cl = 2; cl <= kRgMaxCluster; ++cl) {
+    if (clustered[cl].empty()) continue;
+    qb_status st = launch_regs_cluster(clustered[cl].data(), (int)clustered[cl].size(), cl, ws, stream);
+    if (st != QB_OK) return st;
+  }
+  if (single.empty()) return QB_OK;
+  const HostWeight* m = single.data();
+  const int count = (int)single.size();
   struct Shape {
     int idx, W, gpw, slice, gpi;
     int64_t item_units;
@@ -1191,7 +1342,7 @@ static qb_status launch_regs(const HostWeight* m, int count, void* ws, int sm_co
     b.total_items = items;
     b.count = n;
     const unsigned grid = (unsigned)std::min(items, sm_count);
-    weight_regs_kernel<<<grid, kRgThreads, 0, stream>>>(b);
+    weight_regs_kernel<false><<<grid, kRgThreads, 0, stream>>>(b);
     QB_CUDA_TRY(cudaGetLastError());
   }
   return QB_OK;
@@ -1593,7 +1744,10 @@ extern "C" int32_t qb_quantize_pack_weights_launch_count(const qb_weight_desc* d
   std::vector<qb::HostWeight> regs;
   std::vector<qb::WeightJob> jobs;
   qb::plan_batch(descs, count, 148, regs, jobs);
-  int32_t n = (int32_t)((regs.size() + qb::kRgMaxBatch - 1) / qb::kRgMaxBatch);
+  int per_cluster[qb::kRgMaxCluster + 1] = {};
+  for (const qb::HostWeight& h : regs) ++per_cluster[std::max(1, qb::regs_cluster_size(h))];
+  int32_t n = 0;
+  for (int cl = 1; cl <= qb::kRgMaxCluster; ++cl) n += (per_cluster[cl] + qb::kRgMaxBatch - 1) / qb::kRgMaxBatch;
   for (const qb::WeightJob& j : jobs) n += j.single_read ? 1 : 2;
   return n;
 }

@@ -135,5 +135,7 @@ def test_weight_launch_count_is_host_arithmetic(lib):
     assert lib.qb_quantize_pack_weights_launch_count(arr_of([(768, 768, 4, 1, False)]), 1) == 2  # one range per tensor: two passes
     both = [(768, 768, 4, 128, False), (768, 768, 4, 1, False)]
     assert lib.qb_quantize_pack_weights_launch_count(arr_of(both), 2) == 3
+    clustered = [(768, 768, 4, 12, False), (3072, 768, 2, 12, False), (768, 768, 3, 128, False)]  # clusters of 2 and 6, and single CTAs
+    assert lib.qb_quantize_pack_weights_launch_count(arr_of(clustered), 3) == 3
     assert lib.qb_quantize_pack_weights_launch_count(None, 0) == 0
     assert lib.qb_quantize_pack_weights_launch_count(arr_of([(768, 700, 4, 128, False)]), 1) == 0

@@ -179,6 +179,31 @@ def test_quantize_weights_register_path_shapes():
                          (35, 640, 4, 7), (288, 1152, 3, 9), (9, 1152, 2, 9), (130, 128, 4, 1)], seed0=5)
 
 
+def test_quantize_weights_cluster_path_shapes():
+    # groups of 289 to 2,304 units are held by a thread-block cluster of 2 to 8 CTAs: every cluster size, slices
+    # with ragged ends and warps that get nothing, more groups than resident clusters (several items per
+    # cluster), all bit widths; 2,368 units is past the largest cluster and takes the two passes
+    _check_weight_batch([(34, 2176, 4, 2), (36, 4096, 2, 2), (40, 3712, 3, 2), (12, 30720, 8, 2), (72, 8192, 4, 2),
+                         (74, 8192, 3, 2), (2560, 1536, 2, 80), (2048, 9600, 4, 512), (2640, 1536, 8, 80),
+                         (1000, 2560, 3, 50), (1400, 1408, 2, 40), (96, 16384, 4, 8), (36, 4096, 3, 1), (63, 4096, 4, 1)], seed0=9)
+
+
+def test_quantize_weights_cluster_path_nonfinite():
+    # an Inf in the slice of the last CTA of a cluster of five must reach the group's published range check
+    N, K, G = 12, 30720, 2
+    w = synth.weights(N, K, seed=3)
+    ws_ok, ws_bad = qb.workspace(groups=G), qb.workspace(groups=G)
+    gu.gpu_quantize_weights(w, 3, G, ws_ok)
+    assert qb.read_status(ws_ok) == qb.QB_OK
+    w[11, 30000] = np.inf
+    gu.gpu_quantize_weights(w, 3, G, ws_bad)
+    assert qb.read_status(ws_bad) == qb.QB_ERR_NONFINITE
+    w[11, 30000] = np.nan
+    ws_bad2 = qb.workspace(groups=G)
+    gu.gpu_quantize_weights(w, 3, G, ws_bad2)
+    assert qb.read_status(ws_bad2) == qb.QB_ERR_NONFINITE
+
+
 def test_quantize_weights_register_path_more_matrices_than_one_launch():
     # 100 small matrices of mixed widths and group sizes: two launches
     shapes = [((24 + 8 * (i % 5)), 128 * (1 + i % 3), (2, 3, 4, 8)[i % 4], (1, 2, 4, 8)[(i // 4) % 4]) for i in range(100)]
