@@ -104,9 +104,10 @@ qb_status qb_quantize_act(const float* x, int64_t M, int64_t K, int8_t* xq, floa
  *            max (Appendix A: the range "can be a subinterval of [min, max]"); values outside are
  *            clamped.  They must be finite with range_lo <= range_hi.
  * One kernel (the weights are read once and stay in registers between the range and the rounding)
- * when the groups have at most 36,864 weights each and the range is the group's own; otherwise two
- * kernels (per-group min/max reduction into the workspace, then round/clamp/pack), or one that stages
- * the group in shared memory (caller-supplied ranges, groups of up to 49,152 weights).
+ * when the groups have at most 294,912 weights each and the range is the group's own (groups above
+ * 36,864 weights are held by a thread-block cluster); otherwise two kernels (per-group min/max
+ * reduction into the workspace, then round/clamp/pack), or one that stages the group in shared
+ * memory (caller-supplied ranges, groups of up to 49,152 weights).
  */
 qb_status qb_quantize_pack_weights(const float* w, int64_t N, int64_t K, int bits, int groups,
                                    const float* range_lo, const float* range_hi, uint32_t* packed,
@@ -142,7 +143,8 @@ typedef struct {
  * each result equals the single call on the same arguments bit for bit.  Each activation tensor keeps
  * its own scale (per-tensor quantization).  Weight matrices of different bit widths may be mixed:
  * all matrices whose groups have at most 36,864 weights and take their own [min, max] go into one
- * launch per 96 matrices, whatever their widths (a mixed-precision stack is one launch).  The others
+ * launch per 96 matrices, whatever their widths (a mixed-precision stack is one launch); groups of up
+ * to 294,912 weights likewise, one launch per cluster size.  The others
  * get launches per bit width; when these are several small single-read launches they run side by
  * side on streams the library creates once per device (host objects only), forking from and joining
  * `cuda_stream` inside the call (after the fork every side stream is joined, also when a launch in
