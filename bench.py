@@ -304,7 +304,7 @@ def measure(R: Runner, wl: synth.Workload, steps: int, with_e2e: bool, warm_too:
     # kernels launched per step, counted from the library's own launch plan for these descriptors
     gemm_launches = qb.layer_linears_launch_count(descs)
     weight_launches = qb.quantize_pack_weights_launch_count(w_arr)
-    launches_per_step = ((len(lin) if args.out == "i8" else 2 * -(-len(lin) // 32)) + weight_launches + gemm_launches)
+    launches_per_step = ((len(lin) if args.out == "i8" else qb.quantize_act_launch_count(len(lin))) + weight_launches + gemm_launches)
 
     chained = args.out == "i8"
     out_scales = None
@@ -712,7 +712,7 @@ def run_quantizer_sweep(args):
             assert qb.read_status(ws) == qb.QB_OK
             gbs = params * (4.0 + bits / 8.0) / (ms * 1e-3) / 1e9
             table[f"k{bits}_g{groups}"] = {"ms": ms, "GBps": gbs, "frac_hbm": gbs / peaks["hbm_gbs"]}
-            launches += 2 * -(-len(shapes) // 32) * (3 + steps)
+            launches += qb.quantize_pack_weights_launch_count(arr) * (3 + steps)
             del items, arr
     M, K = synth.QUANTIZER_SWEEP_ACT
     x = torch.from_numpy(synth.activations(M, K, synth.seed_for(4))).to(dev)

@@ -237,6 +237,12 @@ qb_status qb_layer_linears(const qb_linear_desc* descs /*host*/, int32_t count, 
                            size_t ws_bytes, void* cuda_stream);
 
 /*
+ * How many kernel launches qb_quantize_act_batch issues for `count` tensors (two per 64 tensors); host
+ * arithmetic, no GPU work.  (No counterpart in the paper; for callers that count or budget launches.)
+ */
+int32_t qb_quantize_act_launch_count(int32_t count);
+
+/*
  * How many kernel launches qb_quantize_pack_weights_batch issues for these matrices: host arithmetic on
  * the descriptors only (shapes, groups, bit widths, whether ranges are supplied), no GPU work.  (No
  * counterpart in the paper; for callers that count or budget launches.)  The plan is the one of a

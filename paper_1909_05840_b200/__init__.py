@@ -32,7 +32,7 @@ EXPORTS = (
     "qb_layer_linears", "qb_quantize_pack_weights_noalloc", "qb_probe_i8_mma", "qb_quantize_act_batch",
     "qb_quantize_pack_weights_batch", "qb_gemm_bf16", "qb_layer_linears_bf16",
     "qb_fake_quantize_weights", "qb_ste_backward", "qb_quantize_embedding", "qb_embedding_lookup",
-    "qb_gemm_i8", "qb_rowsum_i8", "qb_layer_linears_i8", "qb_sensitivity_bits", "qb_probe_wait_limit", "qb_layer_linears_launch_count", "qb_quantize_pack_weights_launch_count",
+    "qb_gemm_i8", "qb_rowsum_i8", "qb_layer_linears_i8", "qb_sensitivity_bits", "qb_probe_wait_limit", "qb_layer_linears_launch_count", "qb_quantize_pack_weights_launch_count", "qb_quantize_act_launch_count",
 )
 NOALLOC_MAX_GROUPS = 4096
 
@@ -105,6 +105,8 @@ def lib() -> ctypes.CDLL:
     L.qb_layer_linears_launch_count.restype = i32
     L.qb_quantize_pack_weights_launch_count.argtypes = [ctypes.POINTER(WeightDescC), i32]
     L.qb_quantize_pack_weights_launch_count.restype = i32
+    L.qb_quantize_act_launch_count.argtypes = [i32]
+    L.qb_quantize_act_launch_count.restype = i32
     L.qb_probe_wait_limit.argtypes = [vp, sz, i64, vp, vp]
     L.qb_probe_wait_limit.restype = i32
     L.qb_sensitivity_bits.argtypes = [vp, i32, i32, vp, i32, vp, vp, vp]
@@ -429,6 +431,11 @@ def layer_linears(descs, ws: torch.Tensor) -> None:
     """``qb_layer_linears`` over a list of ``LinearDesc`` (or an array from ``make_desc_array``)."""
     arr = descs if isinstance(descs, ctypes.Array) else make_desc_array(descs)
     _check(lib().qb_layer_linears(arr, len(arr), ws.data_ptr(), ws.numel(), _stream()), "qb_layer_linears")
+
+
+def quantize_act_launch_count(count: int) -> int:
+    """``qb_quantize_act_launch_count``: kernel launches ``quantize_act_batch`` issues for ``count`` tensors."""
+    return int(lib().qb_quantize_act_launch_count(int(count)))
 
 
 def quantize_pack_weights_launch_count(items) -> int:

@@ -18,7 +18,7 @@
 namespace qb {
 
 constexpr int kActThreads = 256;
-constexpr int kMaxActBatch = 32;  // tensors per launch (descriptors travel as kernel parameters)
+constexpr int kMaxActBatch = 64;  // tensors per launch (descriptors travel as kernel parameters, 4 KB)
 
 struct ActItem {
   const float* x;
@@ -251,4 +251,9 @@ extern "C" qb_status qb_quantize_act_batch(const qb_act_desc* descs, int32_t cou
     if (st != QB_OK) return st;
   }
   return QB_OK;
+}
+
+extern "C" int32_t qb_quantize_act_launch_count(int32_t count) {
+  if (count <= 0) return 0;
+  return 2 * ((count + qb::kMaxActBatch - 1) / qb::kMaxActBatch);
 }
