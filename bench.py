@@ -738,7 +738,7 @@ def run_quantizer_sweep(args):
         fq[f"{n}x{k}"] = {
             "fake_quantize_k4_g128": {"ms": ms_f, "GBps": 8.0 * n * k / (ms_f * 1e-3) / 1e9,
                                       "frac_hbm": 8.0 * n * k / (ms_f * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                                      "bytes": "8 B per weight (one DRAM read, one write; the second read hits L2)"},
+                                      "bytes": "8 B per weight (one read, one write)"},
             "ste_backward": {"ms": ms_b, "GBps": 12.0 * n * k / (ms_b * 1e-3) / 1e9,
                              "frac_hbm": 12.0 * n * k / (ms_b * 1e-3) / 1e9 / peaks["hbm_gbs"],
                              "bytes": "12 B per weight (gradient and weight read, gradient written)"}}

@@ -314,7 +314,9 @@ qb_status qb_layer_linears_i8(const qb_linear_desc* descs /*host*/, const float*
  *   wq       dev fp32 [N][K], 16-byte aligned                     (written)
  *   delta,q0 dev fp32 [G]                                         (written)
  *   range_lo, range_hi: dev fp32 [G] or both NULL, as for qb_quantize_pack_weights.
- * Two kernels: per-group min/max reduction into the workspace, then round/clamp/dequantize.
+ * One kernel (W read once, as in qb_quantize_pack_weights) for the group's own range and groups of
+ * at most 294,912 weights; otherwise two: per-group min/max reduction into the workspace, then
+ * round/clamp/dequantize.
  *
  * Backward: grad_w = grad_wq where Clamp passes the weight through (range_lo[g] <= w <= range_hi[g],
  * both ends included), 0 where Clamp holds it at an end of the range; the rounding is treated as the

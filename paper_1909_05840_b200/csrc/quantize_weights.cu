@@ -227,6 +227,12 @@ __device__ __forceinline__ GroupParams finish_group(float lo, float hi, bool fro
   return p;
 }
 
+// Delta of a finished group as finish_group publishes it (a constant group comes back with hi == lo: Delta = 1).
+__device__ __forceinline__ float group_step(const GroupParams& gp, int bits_levels) {
+  const float d = __fdiv_rn(__fsub_rn(gp.hi, gp.lo), (float)bits_levels);
+  return d > 0.0f ? d : 1.0f;
+}
+
 // Group g of a matrix: range from the caller's tables or from the reduced encodings in the workspace.
 __device__ __forceinline__ GroupParams load_group(int g, int bits_levels, const uint32_t* __restrict__ hi_enc,
                                                   const uint32_t* __restrict__ lo_inv,
@@ -856,25 +862,33 @@ __device__ __forceinline__ uint32_t quant_field_open(const float4 v, const float
   }
 }
 
+// Parameters of the group a warp is rounding: q0, 1/Delta, and Delta (fake quantization only).
+struct RgGroup {
+  float lo, inv, d;
+};
+// Several groups per warp: lane gi holds the parameters of the warp's group gi.
+__device__ __forceinline__ void rg_next_group(RgGroup& cur, const RgGroup& mine, int& gi, int& next_start, const int ug) {
+  cur.lo = __shfl_sync(0xffffffffu, mine.lo, gi);
+  cur.inv = __shfl_sync(0xffffffffu, mine.inv, gi);
+  cur.d = __shfl_sync(0xffffffffu, mine.d, gi);
+  ++gi;
+  next_start += ug;
+}
+
 // One staging block (units BLK * 6 ... of the slice): fields into the warp's staging area, then out.
 template <int BITS, int BLK, bool MULTI>
-__device__ __forceinline__ void regs_pack_block(float4 (&v)[kRgUnits], const int n, float& lo, float& inv,
-                                                const float p_lo, const float p_inv, int& gi, int& next_start,
-                                                const int ug, uint8_t* stg, uint32_t* __restrict__ out, const int lane,
+__device__ __forceinline__ void regs_pack_block(float4 (&v)[kRgUnits], const int n, RgGroup& cur, const RgGroup& mine,
+                                                int& gi, int& next_start, const int ug, uint8_t* stg,
+                                                uint32_t* __restrict__ out, const int lane,
                                                 const float4* __restrict__ next_src, const int next_n) {
 #pragma unroll
   for (int jj = 0; jj < kRgBlock; ++jj) {
     const int j = BLK * kRgBlock + jj;
     if (j < n) {
       if (MULTI) {
-        if (j == next_start) {  // warp-uniform: the next group of this warp begins
-          lo = __shfl_sync(0xffffffffu, p_lo, gi);
-          inv = __shfl_sync(0xffffffffu, p_inv, gi);
-          ++gi;
-          next_start += ug;
-        }
+        if (j == next_start) rg_next_group(cur, mine, gi, next_start, ug);  // warp-uniform: the warp's next group begins
       }
-      const uint32_t f = quant_field_open<BITS>(v[j], lo, inv);
+      const uint32_t f = quant_field_open<BITS>(v[j], cur.lo, cur.inv);
       const int fi = jj * 32 + lane;  // field index = element index / 4 inside the block
       if (BITS == 8) reinterpret_cast<uint32_t*>(stg)[fi] = f;
       if (BITS == 4 || BITS == 3) reinterpret_cast<uint16_t*>(stg)[fi] = (uint16_t)f;
@@ -914,11 +928,48 @@ __device__ __forceinline__ void regs_pack_block(float4 (&v)[kRgUnits], const int
   __syncwarp();  // the staging area is free again
 }
 
+// Fake quantization (Appendix A, forward of the fine-tuning step): Q(w) = Delta * code + q0 as fp32, written
+// where the packed words would go.  code = (t + 1.5 * 2^23) - 1.5 * 2^23 is the rounded product as a float
+// (exact), then one fused multiply-add; packed two lanes wide like the rounding itself.
+__device__ __forceinline__ float4 fake_quant4(const float4 v, const RgGroup& g) {
+  constexpr float kMagic = 12582912.0f;
+  float4 q;
+  asm("{\n\t.reg .b64 p0, p1, l2, i2, m2, o2, d2;\n\t"
+      "mov.b64 p0, {%4, %5};\n\tmov.b64 p1, {%6, %7};\n\t"
+      "mov.b64 l2, {%8, %8};\n\tmov.b64 i2, {%9, %9};\n\tmov.b64 m2, {%10, %10};\n\tmov.b64 o2, {%11, %11};\n\t"
+      "mov.b64 d2, {%12, %12};\n\t"
+      "sub.rn.f32x2 p0, p0, l2;\n\tsub.rn.f32x2 p1, p1, l2;\n\t"
+      "mul.rn.f32x2 p0, p0, i2;\n\tmul.rn.f32x2 p1, p1, i2;\n\t"
+      "fma.rn.f32x2 p0, p0, o2, m2;\n\tfma.rn.f32x2 p1, p1, o2, m2;\n\t"
+      "sub.rn.f32x2 p0, p0, m2;\n\tsub.rn.f32x2 p1, p1, m2;\n\t"
+      "fma.rn.f32x2 p0, d2, p0, l2;\n\tfma.rn.f32x2 p1, d2, p1, l2;\n\t"
+      "mov.b64 {%0, %1}, p0;\n\tmov.b64 {%2, %3}, p1;\n\t}"
+      : "=f"(q.x), "=f"(q.y), "=f"(q.z), "=f"(q.w)
+      : "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "f"(g.lo), "f"(g.inv), "f"(kMagic), "f"(1.0f), "f"(g.d));
+  return q;
+}
+
 template <int BLK, bool MULTI>
-__device__ __forceinline__ void regs_pack_block_any(const int bits, float4 (&v)[kRgUnits], const int n, float& lo,
-                                                    float& inv, const float p_lo, const float p_inv, int& gi,
-                                                    int& next_start, const int ug, uint8_t* stg,
-                                                    uint32_t* __restrict__ out, const int lane,
+__device__ __forceinline__ void regs_fake_block(float4 (&v)[kRgUnits], const int n, RgGroup& cur, const RgGroup& mine,
+                                                int& gi, int& next_start, const int ug, float4* __restrict__ out,
+                                                const float4* __restrict__ next_src, const int next_n) {
+#pragma unroll
+  for (int jj = 0; jj < kRgBlock; ++jj) {
+    const int j = BLK * kRgBlock + jj;
+    if (j < n) {
+      if (MULTI) {
+        if (j == next_start) rg_next_group(cur, mine, gi, next_start, ug);
+      }
+      out[j * 32] = fake_quant4(v[j], cur);
+    }
+    if (j < next_n) v[j] = __ldg(next_src + j * 32);
+  }
+}
+
+template <int BLK, bool MULTI, bool FAKE>
+__device__ __forceinline__ void regs_pack_block_any(const int bits, float4 (&v)[kRgUnits], const int n, RgGroup& cur,
+                                                    const RgGroup& mine, int& gi, int& next_start, const int ug,
+                                                    uint8_t* stg, uint32_t* __restrict__ out, const int lane,
                                                     const float4* __restrict__ next_src, const int next_n) {
   if (BLK * kRgBlock >= n) {  // nothing of this slice here: only the next slice's loads
 #pragma unroll
@@ -928,11 +979,15 @@ __device__ __forceinline__ void regs_pack_block_any(const int bits, float4 (&v)[
     }
     return;
   }
+  if (FAKE) {
+    regs_fake_block<BLK, MULTI>(v, n, cur, mine, gi, next_start, ug, reinterpret_cast<float4*>(out) + lane, next_src, next_n);
+    return;
+  }
   switch (bits) {  // CTA-uniform
-    case 2: regs_pack_block<2, BLK, MULTI>(v, n, lo, inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane, next_src, next_n); break;
-    case 3: regs_pack_block<3, BLK, MULTI>(v, n, lo, inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane, next_src, next_n); break;
-    case 4: regs_pack_block<4, BLK, MULTI>(v, n, lo, inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane, next_src, next_n); break;
-    default: regs_pack_block<8, BLK, MULTI>(v, n, lo, inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane, next_src, next_n); break;
+    case 2: regs_pack_block<2, BLK, MULTI>(v, n, cur, mine, gi, next_start, ug, stg, out, lane, next_src, next_n); break;
+    case 3: regs_pack_block<3, BLK, MULTI>(v, n, cur, mine, gi, next_start, ug, stg, out, lane, next_src, next_n); break;
+    case 4: regs_pack_block<4, BLK, MULTI>(v, n, cur, mine, gi, next_start, ug, stg, out, lane, next_src, next_n); break;
+    default: regs_pack_block<8, BLK, MULTI>(v, n, cur, mine, gi, next_start, ug, stg, out, lane, next_src, next_n); break;
   }
 }
 
@@ -988,7 +1043,8 @@ __device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v
 // writes its range into every CTA's shared memory and the cluster's barrier publishes them.  Every CTA of a
 // cluster runs the same number of items, so the barriers pair up; the last one also keeps a CTA's shared
 // memory alive until no peer writes to it any more.
-template <bool CLUSTER>
+// FAKE: the fp32 fake-quantized matrix is written instead of packed words (`packed` of the item points to it).
+template <bool CLUSTER, bool FAKE>
 __global__ void __launch_bounds__(kRgThreads, 1)
 weight_regs_kernel(const __grid_constant__ RegsBatch b) {
   __shared__ __align__(16) uint8_t s_stage[kRgWarps][kRgBlock * 128];
@@ -1018,7 +1074,8 @@ weight_regs_kernel(const __grid_constant__ RegsBatch b) {
     const int W = m.team_warps;
     const int bits = m.bits;
     const int L = (1 << bits) - 1;
-    uint32_t* const out = m.packed + ((int64_t)s.first_group * m.ug + s.first_unit) * (4 * bits);
+    // first output word of the slice: 4k packed words per unit, or the unit's 128 floats
+    uint32_t* const out = m.packed + ((int64_t)s.first_group * m.ug + s.first_unit) * (FAKE ? 128 : 4 * bits);
     if (!CLUSTER && m.groups_per_warp > 1) {
       // ---- several whole groups in this warp ----
       const int ug = m.ug;
@@ -1045,21 +1102,22 @@ weight_regs_kernel(const __grid_constant__ RegsBatch b) {
         }
       }
       // lane i finishes group i of the warp
-      float p_lo = 0.0f, p_inv = 1.0f;
+      RgGroup mine{0.0f, 1.0f, 1.0f};
       if (lane < s.ng) {
         const float g_hi = ordered_to_float(my_hi);
         const float g_lo = ordered_to_float(~my_lo);
         if (!(fabsf(g_hi) <= 3.402823466e38f && fabsf(g_lo) <= 3.402823466e38f)) report_status(b.ws, QB_ERR_NONFINITE);
         const GroupParams gp = finish_group(g_lo, g_hi, false, L, s.first_group + lane, m.delta, m.q0, true, b.ws);
-        p_lo = gp.lo;
-        p_inv = gp.inv;
+        mine.lo = gp.lo;
+        mine.inv = gp.inv;
+        mine.d = group_step(gp, L);
       }
-      float c_lo = 0.0f, c_inv = 1.0f;
+      RgGroup cur{0.0f, 1.0f, 1.0f};
       int next_start = 0;
       gi = 0;
-      regs_pack_block_any<0, true>(bits, v, n, c_lo, c_inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane, nx.src, nx.n);
-      regs_pack_block_any<1, true>(bits, v, n, c_lo, c_inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane, nx.src, nx.n);
-      regs_pack_block_any<2, true>(bits, v, n, c_lo, c_inv, p_lo, p_inv, gi, next_start, ug, stg, out, lane, nx.src, nx.n);
+      regs_pack_block_any<0, true, FAKE>(bits, v, n, cur, mine, gi, next_start, ug, stg, out, lane, nx.src, nx.n);
+      regs_pack_block_any<1, true, FAKE>(bits, v, n, cur, mine, gi, next_start, ug, stg, out, lane, nx.src, nx.n);
+      regs_pack_block_any<2, true, FAKE>(bits, v, n, cur, mine, gi, next_start, ug, stg, out, lane, nx.src, nx.n);
     } else if (s.ng > 0) {
       // ---- a slice of one group (team-uniform: every warp of the team is here) ----
       float lo = kInf, hi = -kInf;
@@ -1108,11 +1166,12 @@ weight_regs_kernel(const __grid_constant__ RegsBatch b) {
       if (publish && !(fabsf(g_hi) <= 3.402823466e38f && fabsf(g_lo) <= 3.402823466e38f))
         report_status(b.ws, QB_ERR_NONFINITE);
       const GroupParams gp = finish_group(g_lo, g_hi, false, L, s.first_group, m.delta, m.q0, publish, b.ws);
-      float c_lo = gp.lo, c_inv = gp.inv;
+      RgGroup cur{gp.lo, gp.inv, group_step(gp, L)};
+      const RgGroup mine{0.0f, 1.0f, 1.0f};
       int gi = 0, next_start = -1;
-      regs_pack_block_any<0, false>(bits, v, n, c_lo, c_inv, 0.0f, 1.0f, gi, next_start, 0, stg, out, lane, nx.src, nx.n);
-      regs_pack_block_any<1, false>(bits, v, n, c_lo, c_inv, 0.0f, 1.0f, gi, next_start, 0, stg, out, lane, nx.src, nx.n);
-      regs_pack_block_any<2, false>(bits, v, n, c_lo, c_inv, 0.0f, 1.0f, gi, next_start, 0, stg, out, lane, nx.src, nx.n);
+      regs_pack_block_any<0, false, FAKE>(bits, v, n, cur, mine, gi, next_start, 0, stg, out, lane, nx.src, nx.n);
+      regs_pack_block_any<1, false, FAKE>(bits, v, n, cur, mine, gi, next_start, 0, stg, out, lane, nx.src, nx.n);
+      regs_pack_block_any<2, false, FAKE>(bits, v, n, cur, mine, gi, next_start, 0, stg, out, lane, nx.src, nx.n);
     } else {
       // nothing of this item here (a last item with fewer groups than teams): only the next slice's loads
 #pragma unroll
@@ -1222,7 +1281,7 @@ static qb_status regs_max_clusters(int cl, int* out) {
     at[0].val.clusterDim.z = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    QB_CUDA_TRY(cudaOccupancyMaxActiveClusters(&n, weight_regs_kernel<true>, &cfg));
+    QB_CUDA_TRY(cudaOccupancyMaxActiveClusters(&n, weight_regs_kernel<true, false>, &cfg));
     if (n < 1) {
       set_last_error("no cluster of %d CTAs fits the device", cl);
       return QB_ERR_CUDA;
@@ -1235,7 +1294,7 @@ static qb_status regs_max_clusters(int cl, int* out) {
 
 // Matrices whose groups need a cluster of `cl` CTAs (289 to 2,304 units per group), any bit widths: one
 // group per cluster item.
-static qb_status launch_regs_cluster(const HostWeight* m, int count, int cl, void* ws, cudaStream_t stream) {
+static qb_status launch_regs_cluster(const HostWeight* m, int count, int cl, void* ws, cudaStream_t stream, bool fake) {
   int max_clusters = 0;
   qb_status st = regs_max_clusters(cl, &max_clusters);
   if (st != QB_OK) return st;
@@ -1276,7 +1335,10 @@ static qb_status launch_regs_cluster(const HostWeight* m, int count, int cl, voi
     at[0].val.clusterDim.z = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    QB_CUDA_TRY(cudaLaunchKernelEx(&cfg, weight_regs_kernel<true>, b));
+    if (fake)
+      QB_CUDA_TRY(cudaLaunchKernelEx(&cfg, weight_regs_kernel<true, true>, b));
+    else
+      QB_CUDA_TRY(cudaLaunchKernelEx(&cfg, weight_regs_kernel<true, false>, b));
   }
   return QB_OK;
 }
@@ -1284,7 +1346,8 @@ static qb_status launch_regs_cluster(const HostWeight* m, int count, int cl, voi
 // Register-resident path over any number of eligible matrices of any bit widths: launches of up to
 // kRgMaxBatch matrices, inside a launch the matrices with the largest CTA items first.  Matrices whose
 // groups need a cluster go to launches of their cluster size.
-static qb_status launch_regs(const HostWeight* m_all, int count_all, void* ws, int sm_count, cudaStream_t stream) {
+static qb_status launch_regs(const HostWeight* m_all, int count_all, void* ws, int sm_count, cudaStream_t stream,
+                             bool fake = false) {
   std::vector<HostWeight> single, clustered[kRgMaxCluster + 1];
   for (int i = 0; i < count_all; ++i) {
     const int cl = regs_cluster_size(m_all[i]);
@@ -1292,7 +1355,7 @@ static qb_status launch_regs(const HostWeight* m_all, int count_all, void* ws, i
   }
   for (int cl = 2; cl <= kRgMaxCluster; ++cl) {
     if (clustered[cl].empty()) continue;
-    qb_status st = launch_regs_cluster(clustered[cl].data(), (int)clustered[cl].size(), cl, ws, stream);
+    qb_status st = launch_regs_cluster(clustered[cl].data(), (int)clustered[cl].size(), cl, ws, stream, fake);
     if (st != QB_OK) return st;
   }
   if (single.empty()) return QB_OK;
@@ -1342,7 +1405,10 @@ static qb_status launch_regs(const HostWeight* m_all, int count_all, void* ws, i
     b.total_items = items;
     b.count = n;
     const unsigned grid = (unsigned)std::min(items, sm_count);
-    weight_regs_kernel<false><<<grid, kRgThreads, 0, stream>>>(b);
+    if (fake)
+      weight_regs_kernel<false, true><<<grid, kRgThreads, 0, stream>>>(b);
+    else
+      weight_regs_kernel<false, false><<<grid, kRgThreads, 0, stream>>>(b);
     QB_CUDA_TRY(cudaGetLastError());
   }
   return QB_OK;
@@ -1585,10 +1651,16 @@ static qb_status run_weight_jobs(const std::vector<WeightJob>& jobs, void* ws, i
   return first_error;
 }
 
-// Fake quantization of one matrix: the range kernel of the two-pass path, then weight_fake_kernel.
+// Fake quantization of one matrix: the register-resident kernel where the groups fit it, else the range
+// kernel of the two-pass path, then weight_fake_kernel.
 static qb_status launch_fake_quantize(const float* w, int64_t N, int64_t K, int bits, int groups,
                                       const float* range_lo, const float* range_hi, float* wq, float* delta,
                                       float* q0, void* ws, int sm_count, cudaStream_t stream) {
+  {
+    // groups that fit the registers of a CTA or of a cluster, with their own ranges: one read of W
+    const HostWeight h{w, N, K, groups, range_lo, range_hi, reinterpret_cast<uint32_t*>(wq), delta, q0, bits};
+    if (regs_eligible(h)) return launch_regs(&h, 1, ws, sm_count, stream, true);
+  }
   WeightBatch b;
   memset(&b, 0, sizeof(b));
   WeightItem& it = b.item[0];

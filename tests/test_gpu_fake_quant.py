@@ -20,7 +20,10 @@ def ws():
 
 
 @pytest.mark.parametrize("bits", (2, 3, 4, 8))
-@pytest.mark.parametrize("N,K,groups", [(768, 768, 12), (264, 384, 11), (96, 3072, 96), (128, 128, 1), (3072, 768, 128)])
+@pytest.mark.parametrize("N,K,groups", [(768, 768, 12), (264, 384, 11), (96, 3072, 96), (128, 128, 1), (3072, 768, 128),
+                                        (70, 256, 70),     # two units per group: nine groups per warp, a last warp with fewer
+                                        (12, 30720, 2),    # 1,440 units per group: a cluster of five CTAs
+                                        (74, 8192, 2)])    # 2,368 units per group: the two-pass path
 def test_fake_quantize_matches_oracle(ws, bits, N, K, groups):
     w = synth.weights(N, K, seed=3 * N + K + groups + bits)
     wq = gu.poison(torch.empty((N, K), dtype=torch.float32, device="cuda"))
@@ -57,6 +60,28 @@ def test_fake_quantize_clipped_ranges_constant_group_and_nonfinite(ws):
     ws2 = qb.workspace(groups=64)
     qb.fake_quantize_weights(gu.dev(bad), 4, G, ws2)
     assert qb.read_status(ws2) == qb.QB_ERR_NONFINITE
+
+
+def test_fake_quantize_products_that_round_onto_ties(ws):
+    # weights within a few ulp of the midpoints between grid points (see the packer's test of the same name)
+    N, K, G, bits = 96, 1152, 12, 4
+    rng = np.random.default_rng(5)
+    L = (1 << bits) - 1
+    w = np.empty((N, K), np.float32)
+    R = N // G
+    for g in range(G):
+        lo = np.float32(-0.05 - 0.02 * rng.random())
+        hi = np.float32(0.04 + 0.03 * rng.random())
+        d = np.float32((hi - lo) / np.float32(L))
+        m = rng.integers(0, L, size=(R, K)).astype(np.float32)
+        x = (lo + (m + np.float32(0.5)) * d).astype(np.float32)
+        x = (x.view(np.int32) + rng.integers(-4, 5, size=x.shape).astype(np.int32)).view(np.float32)
+        x[0, 0], x[0, 1] = lo, hi
+        w[g * R:(g + 1) * R] = np.clip(x, lo, hi)
+    wq, delta, q0 = qb.fake_quantize_weights(gu.dev(w), bits, G, ws)
+    st, o_q, o_delta, o_q0 = oracle.fake_quantize_weights(w, bits, G)
+    assert st == oracle.OK and qb.read_status(ws) == qb.QB_OK
+    assert np.array_equal(wq.cpu().numpy().view(np.uint32), o_q.view(np.uint32))
 
 
 @pytest.mark.parametrize("N,K,groups", [(768, 768, 12), (264, 384, 11), (3072, 768, 128), (8, 128, 1)])
