@@ -807,6 +807,10 @@ struct RegsItem {
   int16_t groups_per_warp;  // > 1 only with W = 1
   int16_t slice_units;      // units per warp of a team: ceil(ug / W)
   int16_t bits;
+  const float* range_lo;    // caller-supplied ranges (the kernel that clamps), else null
+  const float* range_hi;
+  int32_t chunks;           // caller-supplied ranges only: a group of more than 288 units is cut into this many items
+  int32_t pad;
 };
 
 struct RegsBatch {
@@ -839,9 +843,15 @@ __device__ __forceinline__ float max3_nan(float a, float b, float c) {
 
 // Four codes of one float4 as a 4k-bit field in the low bits of the result (k < 8: bits from 22 up are
 // left over from the rounding constant and are dropped by the narrow store that follows).
-template <int BITS>
-__device__ __forceinline__ uint32_t quant_field_open(const float4 v, const float lo, const float inv) {
+template <int BITS, bool CLAMP>
+__device__ __forceinline__ uint32_t quant_field_open(float4 v, const float lo, const float inv, const float hi) {
   constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23: adding it rounds to an integer, half to even
+  if (CLAMP) {  // Clamp(X, q0, qmax): a caller's range may leave weights outside
+    v.x = fminf(fmaxf(v.x, lo), hi);
+    v.y = fminf(fmaxf(v.y, lo), hi);
+    v.z = fminf(fmaxf(v.z, lo), hi);
+    v.w = fminf(fmaxf(v.w, lo), hi);
+  }
   // Two lanes of fp32 per instruction (sub, mul, then the rounding add).  The add is written as a fused
   // multiply-add with 1.0: a packed mul followed by a packed add gets contracted into one fused operation,
   // which rounds the exact product instead of the rounded one and lands on the other side of a tie.
@@ -864,19 +874,20 @@ __device__ __forceinline__ uint32_t quant_field_open(const float4 v, const float
 
 // Parameters of the group a warp is rounding: q0, 1/Delta, and Delta (fake quantization only).
 struct RgGroup {
-  float lo, inv, d;
+  float lo, inv, d, hi;  // hi: the kernel that clamps only
 };
 // Several groups per warp: lane gi holds the parameters of the warp's group gi.
 __device__ __forceinline__ void rg_next_group(RgGroup& cur, const RgGroup& mine, int& gi, int& next_start, const int ug) {
   cur.lo = __shfl_sync(0xffffffffu, mine.lo, gi);
   cur.inv = __shfl_sync(0xffffffffu, mine.inv, gi);
   cur.d = __shfl_sync(0xffffffffu, mine.d, gi);
+  cur.hi = __shfl_sync(0xffffffffu, mine.hi, gi);
   ++gi;
   next_start += ug;
 }
 
 // One staging block (units BLK * 6 ... of the slice): fields into the warp's staging area, then out.
-template <int BITS, int BLK, bool MULTI>
+template <int BITS, int BLK, bool MULTI, bool CLAMP>
 __device__ __forceinline__ void regs_pack_block(float4 (&v)[kRgUnits], const int n, RgGroup& cur, const RgGroup& mine,
                                                 int& gi, int& next_start, const int ug, uint8_t* stg,
                                                 uint32_t* __restrict__ out, const int lane,
@@ -888,7 +899,7 @@ __device__ __forceinline__ void regs_pack_block(float4 (&v)[kRgUnits], const int
       if (MULTI) {
         if (j == next_start) rg_next_group(cur, mine, gi, next_start, ug);  // warp-uniform: the warp's next group begins
       }
-      const uint32_t f = quant_field_open<BITS>(v[j], cur.lo, cur.inv);
+      const uint32_t f = quant_field_open<BITS, CLAMP>(v[j], cur.lo, cur.inv, cur.hi);
       const int fi = jj * 32 + lane;  // field index = element index / 4 inside the block
       if (BITS == 8) reinterpret_cast<uint32_t*>(stg)[fi] = f;
       if (BITS == 4 || BITS == 3) reinterpret_cast<uint16_t*>(stg)[fi] = (uint16_t)f;
@@ -931,9 +942,16 @@ __device__ __forceinline__ void regs_pack_block(float4 (&v)[kRgUnits], const int
 // Fake quantization (Appendix A, forward of the fine-tuning step): Q(w) = Delta * code + q0 as fp32, written
 // where the packed words would go.  code = (t + 1.5 * 2^23) - 1.5 * 2^23 is the rounded product as a float
 // (exact), then one fused multiply-add; packed two lanes wide like the rounding itself.
-__device__ __forceinline__ float4 fake_quant4(const float4 v, const RgGroup& g) {
+template <bool CLAMP>
+__device__ __forceinline__ float4 fake_quant4(float4 v, const RgGroup& g) {
   constexpr float kMagic = 12582912.0f;
   float4 q;
+  if (CLAMP) {
+    v.x = fminf(fmaxf(v.x, g.lo), g.hi);
+    v.y = fminf(fmaxf(v.y, g.lo), g.hi);
+    v.z = fminf(fmaxf(v.z, g.lo), g.hi);
+    v.w = fminf(fmaxf(v.w, g.lo), g.hi);
+  }
   asm("{\n\t.reg .b64 p0, p1, l2, i2, m2, o2, d2;\n\t"
       "mov.b64 p0, {%4, %5};\n\tmov.b64 p1, {%6, %7};\n\t"
       "mov.b64 l2, {%8, %8};\n\tmov.b64 i2, {%9, %9};\n\tmov.b64 m2, {%10, %10};\n\tmov.b64 o2, {%11, %11};\n\t"
@@ -949,7 +967,7 @@ __device__ __forceinline__ float4 fake_quant4(const float4 v, const RgGroup& g) 
   return q;
 }
 
-template <int BLK, bool MULTI>
+template <int BLK, bool MULTI, bool CLAMP>
 __device__ __forceinline__ void regs_fake_block(float4 (&v)[kRgUnits], const int n, RgGroup& cur, const RgGroup& mine,
                                                 int& gi, int& next_start, const int ug, float4* __restrict__ out,
                                                 const float4* __restrict__ next_src, const int next_n) {
@@ -960,13 +978,13 @@ __device__ __forceinline__ void regs_fake_block(float4 (&v)[kRgUnits], const int
       if (MULTI) {
         if (j == next_start) rg_next_group(cur, mine, gi, next_start, ug);
       }
-      out[j * 32] = fake_quant4(v[j], cur);
+      out[j * 32] = fake_quant4<CLAMP>(v[j], cur);
     }
     if (j < next_n) v[j] = __ldg(next_src + j * 32);
   }
 }
 
-template <int BLK, bool MULTI, bool FAKE>
+template <int BLK, bool MULTI, bool FAKE, bool CLAMP>
 __device__ __forceinline__ void regs_pack_block_any(const int bits, float4 (&v)[kRgUnits], const int n, RgGroup& cur,
                                                     const RgGroup& mine, int& gi, int& next_start, const int ug,
                                                     uint8_t* stg, uint32_t* __restrict__ out, const int lane,
@@ -980,14 +998,14 @@ __device__ __forceinline__ void regs_pack_block_any(const int bits, float4 (&v)[
     return;
   }
   if (FAKE) {
-    regs_fake_block<BLK, MULTI>(v, n, cur, mine, gi, next_start, ug, reinterpret_cast<float4*>(out) + lane, next_src, next_n);
+    regs_fake_block<BLK, MULTI, CLAMP>(v, n, cur, mine, gi, next_start, ug, reinterpret_cast<float4*>(out) + lane, next_src, next_n);
     return;
   }
   switch (bits) {  // CTA-uniform
-    case 2: regs_pack_block<2, BLK, MULTI>(v, n, cur, mine, gi, next_start, ug, stg, out, lane, next_src, next_n); break;
-    case 3: regs_pack_block<3, BLK, MULTI>(v, n, cur, mine, gi, next_start, ug, stg, out, lane, next_src, next_n); break;
-    case 4: regs_pack_block<4, BLK, MULTI>(v, n, cur, mine, gi, next_start, ug, stg, out, lane, next_src, next_n); break;
-    default: regs_pack_block<8, BLK, MULTI>(v, n, cur, mine, gi, next_start, ug, stg, out, lane, next_src, next_n); break;
+    case 2: regs_pack_block<2, BLK, MULTI, CLAMP>(v, n, cur, mine, gi, next_start, ug, stg, out, lane, next_src, next_n); break;
+    case 3: regs_pack_block<3, BLK, MULTI, CLAMP>(v, n, cur, mine, gi, next_start, ug, stg, out, lane, next_src, next_n); break;
+    case 4: regs_pack_block<4, BLK, MULTI, CLAMP>(v, n, cur, mine, gi, next_start, ug, stg, out, lane, next_src, next_n); break;
+    default: regs_pack_block<8, BLK, MULTI, CLAMP>(v, n, cur, mine, gi, next_start, ug, stg, out, lane, next_src, next_n); break;
   }
 }
 
@@ -1014,6 +1032,17 @@ __device__ __forceinline__ RegsSlice regs_slice(const RegsBatch& b, const int id
   } else {
     const int W = m.team_warps;
     const int team = warp / W, tw = warp - team * W;
+    if (m.chunks > 1) {
+      // caller-supplied ranges, a group larger than a CTA's registers: no reduction ties the group together,
+      // so it is cut into items of 288 units
+      const int local = id - m.item_begin;
+      s.first_group = local / m.chunks;
+      s.ng = 1;
+      s.first_unit = (local - s.first_group * m.chunks) * kRgMaxGroupUnits + warp * kRgUnits;
+      s.n = min(max(m.ug - s.first_unit, 0), kRgUnits);
+      s.src = m.w + ((int64_t)s.first_group * m.ug + s.first_unit) * 32 + lane;
+      return s;
+    }
     s.first_group = (id - m.item_begin) * m.groups_per_item + team * m.groups_per_warp;
     s.ng = min(max(m.groups - s.first_group, 0), (int)m.groups_per_warp);
     if (s.ng > 0) {
@@ -1044,7 +1073,9 @@ __device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v
 // cluster runs the same number of items, so the barriers pair up; the last one also keeps a CTA's shared
 // memory alive until no peer writes to it any more.
 // FAKE: the fp32 fake-quantized matrix is written instead of packed words (`packed` of the item points to it).
-template <bool CLUSTER, bool FAKE>
+// CLAMP: the ranges are the caller's (`range_lo`, `range_hi` of the item): no reduction and no exchange, the
+// weights are clamped into the range, and the pass over the registers only looks for NaN and Inf.
+template <bool CLUSTER, bool FAKE, bool CLAMP>
 __global__ void __launch_bounds__(kRgThreads, 1)
 weight_regs_kernel(const __grid_constant__ RegsBatch b) {
   __shared__ __align__(16) uint8_t s_stage[kRgWarps][kRgBlock * 128];
@@ -1087,7 +1118,7 @@ weight_regs_kernel(const __grid_constant__ RegsBatch b) {
         if (j < n) {
           lo = min3_nan(min3_nan(lo, v[j].x, v[j].y), v[j].z, v[j].w);
           hi = max3_nan(max3_nan(hi, v[j].x, v[j].y), v[j].z, v[j].w);
-          if (j + 1 == end) {  // warp-uniform
+          if (!CLAMP && j + 1 == end) {  // warp-uniform
             const uint32_t e_hi = __reduce_max_sync(0xffffffffu, float_to_ordered(hi));
             const uint32_t e_lo = __reduce_max_sync(0xffffffffu, ~float_to_ordered(lo));
             if (lane == gi) {
@@ -1102,22 +1133,34 @@ weight_regs_kernel(const __grid_constant__ RegsBatch b) {
         }
       }
       // lane i finishes group i of the warp
-      RgGroup mine{0.0f, 1.0f, 1.0f};
+      RgGroup mine{0.0f, 1.0f, 1.0f, 0.0f};
+      if (CLAMP) {
+        // hi / lo hold this lane's running extremes over all of the warp's groups: NaN or Inf anywhere shows
+        if (__any_sync(0xffffffffu, !(fabsf(hi) <= 3.402823466e38f && fabsf(lo) <= 3.402823466e38f)) && lane == 0 && n > 0)
+          report_status(b.ws, QB_ERR_NONFINITE);
+      }
       if (lane < s.ng) {
-        const float g_hi = ordered_to_float(my_hi);
-        const float g_lo = ordered_to_float(~my_lo);
-        if (!(fabsf(g_hi) <= 3.402823466e38f && fabsf(g_lo) <= 3.402823466e38f)) report_status(b.ws, QB_ERR_NONFINITE);
-        const GroupParams gp = finish_group(g_lo, g_hi, false, L, s.first_group + lane, m.delta, m.q0, true, b.ws);
+        GroupParams gp;
+        if (CLAMP) {
+          const int g = s.first_group + lane;
+          gp = finish_group(__ldg(m.range_lo + g), __ldg(m.range_hi + g), true, L, g, m.delta, m.q0, true, b.ws);
+        } else {
+          const float g_hi = ordered_to_float(my_hi);
+          const float g_lo = ordered_to_float(~my_lo);
+          if (!(fabsf(g_hi) <= 3.402823466e38f && fabsf(g_lo) <= 3.402823466e38f)) report_status(b.ws, QB_ERR_NONFINITE);
+          gp = finish_group(g_lo, g_hi, false, L, s.first_group + lane, m.delta, m.q0, true, b.ws);
+        }
         mine.lo = gp.lo;
         mine.inv = gp.inv;
         mine.d = group_step(gp, L);
+        mine.hi = gp.hi;
       }
-      RgGroup cur{0.0f, 1.0f, 1.0f};
+      RgGroup cur{0.0f, 1.0f, 1.0f, 0.0f};
       int next_start = 0;
       gi = 0;
-      regs_pack_block_any<0, true, FAKE>(bits, v, n, cur, mine, gi, next_start, ug, stg, out, lane, nx.src, nx.n);
-      regs_pack_block_any<1, true, FAKE>(bits, v, n, cur, mine, gi, next_start, ug, stg, out, lane, nx.src, nx.n);
-      regs_pack_block_any<2, true, FAKE>(bits, v, n, cur, mine, gi, next_start, ug, stg, out, lane, nx.src, nx.n);
+      regs_pack_block_any<0, true, FAKE, CLAMP>(bits, v, n, cur, mine, gi, next_start, ug, stg, out, lane, nx.src, nx.n);
+      regs_pack_block_any<1, true, FAKE, CLAMP>(bits, v, n, cur, mine, gi, next_start, ug, stg, out, lane, nx.src, nx.n);
+      regs_pack_block_any<2, true, FAKE, CLAMP>(bits, v, n, cur, mine, gi, next_start, ug, stg, out, lane, nx.src, nx.n);
     } else if (s.ng > 0) {
       // ---- a slice of one group (team-uniform: every warp of the team is here) ----
       float lo = kInf, hi = -kInf;
@@ -1129,9 +1172,15 @@ weight_regs_kernel(const __grid_constant__ RegsBatch b) {
         }
       }
       // NaN anywhere makes hi NaN (encoded above every number); Inf shows as hi = +Inf or lo = -Inf
-      uint32_t e_hi = __reduce_max_sync(0xffffffffu, float_to_ordered(hi));
-      uint32_t e_lo = __reduce_max_sync(0xffffffffu, ~float_to_ordered(lo));
-      if (CLUSTER) {
+      uint32_t e_hi = 0, e_lo = 0;
+      if (!CLAMP) {
+        e_hi = __reduce_max_sync(0xffffffffu, float_to_ordered(hi));
+        e_lo = __reduce_max_sync(0xffffffffu, ~float_to_ordered(lo));
+      }
+      if (CLAMP) {
+        if (__any_sync(0xffffffffu, !(fabsf(hi) <= 3.402823466e38f && fabsf(lo) <= 3.402823466e38f)) && lane == 0 && n > 0)
+          report_status(b.ws, QB_ERR_NONFINITE);
+      } else if (CLUSTER) {
         const int flip = round & 1;
         if (lane == 0) {
           s_hi[flip][warp] = e_hi;
@@ -1160,18 +1209,24 @@ weight_regs_kernel(const __grid_constant__ RegsBatch b) {
         e_hi = __reduce_max_sync(0xffffffffu, vh);
         e_lo = __reduce_max_sync(0xffffffffu, vl);
       }
-      const float g_hi = ordered_to_float(e_hi);
-      const float g_lo = ordered_to_float(~e_lo);
       const bool publish = s.first_unit == 0 && lane == 0;
-      if (publish && !(fabsf(g_hi) <= 3.402823466e38f && fabsf(g_lo) <= 3.402823466e38f))
-        report_status(b.ws, QB_ERR_NONFINITE);
-      const GroupParams gp = finish_group(g_lo, g_hi, false, L, s.first_group, m.delta, m.q0, publish, b.ws);
-      RgGroup cur{gp.lo, gp.inv, group_step(gp, L)};
-      const RgGroup mine{0.0f, 1.0f, 1.0f};
+      GroupParams gp;
+      if (CLAMP) {
+        gp = finish_group(__ldg(m.range_lo + s.first_group), __ldg(m.range_hi + s.first_group), true, L, s.first_group,
+                          m.delta, m.q0, publish, b.ws);
+      } else {
+        const float g_hi = ordered_to_float(e_hi);
+        const float g_lo = ordered_to_float(~e_lo);
+        if (publish && !(fabsf(g_hi) <= 3.402823466e38f && fabsf(g_lo) <= 3.402823466e38f))
+          report_status(b.ws, QB_ERR_NONFINITE);
+        gp = finish_group(g_lo, g_hi, false, L, s.first_group, m.delta, m.q0, publish, b.ws);
+      }
+      RgGroup cur{gp.lo, gp.inv, group_step(gp, L), gp.hi};
+      const RgGroup mine{0.0f, 1.0f, 1.0f, 0.0f};
       int gi = 0, next_start = -1;
-      regs_pack_block_any<0, false, FAKE>(bits, v, n, cur, mine, gi, next_start, 0, stg, out, lane, nx.src, nx.n);
-      regs_pack_block_any<1, false, FAKE>(bits, v, n, cur, mine, gi, next_start, 0, stg, out, lane, nx.src, nx.n);
-      regs_pack_block_any<2, false, FAKE>(bits, v, n, cur, mine, gi, next_start, 0, stg, out, lane, nx.src, nx.n);
+      regs_pack_block_any<0, false, FAKE, CLAMP>(bits, v, n, cur, mine, gi, next_start, 0, stg, out, lane, nx.src, nx.n);
+      regs_pack_block_any<1, false, FAKE, CLAMP>(bits, v, n, cur, mine, gi, next_start, 0, stg, out, lane, nx.src, nx.n);
+      regs_pack_block_any<2, false, FAKE, CLAMP>(bits, v, n, cur, mine, gi, next_start, 0, stg, out, lane, nx.src, nx.n);
     } else {
       // nothing of this item here (a last item with fewer groups than teams): only the next slice's loads
 #pragma unroll
@@ -1250,14 +1305,15 @@ static qb_status launch_two_pass(const HostWeight* m, int count, int bits, void*
 
 static inline int64_t group_units(const HostWeight& h) { return (h.N / h.groups) * (h.K / 128); }
 
-// Does a matrix take the register-resident path?  (Its own ranges; groups of at most 288 units in one
-// CTA, up to 2,304 in a cluster of up to 8 CTAs.)
+// Does a matrix take the register-resident path?  With its own ranges: groups of at most 288 units in one
+// CTA, up to 2,304 in a cluster of up to 8 CTAs.  With the caller's ranges: always (nothing to reduce).
 constexpr int kRgMaxCluster = 8;
 static inline int regs_cluster_size(const HostWeight& h) {
+  if (h.range_lo != nullptr) return 1;
   return (int)((group_units(h) + kRgMaxGroupUnits - 1) / kRgMaxGroupUnits);
 }
 static inline bool regs_eligible(const HostWeight& h) {
-  return h.range_lo == nullptr && group_units(h) <= (int64_t)kRgMaxGroupUnits * kRgMaxCluster;
+  return h.range_lo != nullptr || group_units(h) <= (int64_t)kRgMaxGroupUnits * kRgMaxCluster;
 }
 
 // Clusters of `cl` CTAs that can be resident at once (asked once per device and cluster size).
@@ -1281,7 +1337,7 @@ static qb_status regs_max_clusters(int cl, int* out) {
     at[0].val.clusterDim.z = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    QB_CUDA_TRY(cudaOccupancyMaxActiveClusters(&n, weight_regs_kernel<true, false>, &cfg));
+    QB_CUDA_TRY(cudaOccupancyMaxActiveClusters(&n, weight_regs_kernel<true, false, false>, &cfg));
     if (n < 1) {
       set_last_error("no cluster of %d CTAs fits the device", cl);
       return QB_ERR_CUDA;
@@ -1336,44 +1392,41 @@ static qb_status launch_regs_cluster(const HostWeight* m, int count, int cl, voi
     cfg.attrs = at;
     cfg.numAttrs = 1;
     if (fake)
-      QB_CUDA_TRY(cudaLaunchKernelEx(&cfg, weight_regs_kernel<true, true>, b));
+      QB_CUDA_TRY(cudaLaunchKernelEx(&cfg, weight_regs_kernel<true, true, false>, b));
     else
-      QB_CUDA_TRY(cudaLaunchKernelEx(&cfg, weight_regs_kernel<true, false>, b));
+      QB_CUDA_TRY(cudaLaunchKernelEx(&cfg, weight_regs_kernel<true, false, false>, b));
   }
   return QB_OK;
 }
 
-// Register-resident path over any number of eligible matrices of any bit widths: launches of up to
-// kRgMaxBatch matrices, inside a launch the matrices with the largest CTA items first.  Matrices whose
-// groups need a cluster go to launches of their cluster size.
-static qb_status launch_regs(const HostWeight* m_all, int count_all, void* ws, int sm_count, cudaStream_t stream,
-                             bool fake = false) {
-  std::vector<HostWeight> single, clustered[kRgMaxCluster + 1];
-  for (int i = 0; i < count_all; ++i) {
-    const int cl = regs_cluster_size(m_all[i]);
-    (cl <= 1 ? single : clustered[cl]).push_back(m_all[i]);
-  }
-  for (int cl = 2; cl <= kRgMaxCluster; ++cl) {
-    if (clustered[cl].empty()) continue;
-    qb_status st = launch_regs_cluster(clustered[cl].data(), (int)clustered[cl].size(), cl, ws, stream, fake);
-    if (st != QB_OK) return st;
-  }
-  if (single.empty()) return QB_OK;
-  const HostWeight* m = single.data();
-  const int count = (int)single.size();
+// Matrices served by single CTAs (own ranges with groups of at most 288 units, or the caller's ranges with
+// groups of any size: `ranged`), any bit widths: launches of up to kRgMaxBatch matrices, inside a launch
+// the matrices with the largest CTA items first.
+static qb_status launch_regs_single(const HostWeight* m, int count, bool ranged, void* ws, int sm_count,
+                                    cudaStream_t stream, bool fake) {
   struct Shape {
-    int idx, W, gpw, slice, gpi;
+    int idx, W, gpw, slice, gpi, chunks;
     int64_t item_units;
   };
   std::vector<Shape> sh(count);
   for (int i = 0; i < count; ++i) {
-    const int ug = (int)group_units(m[i]);
+    const int64_t ug = group_units(m[i]);
     Shape& s = sh[i];
     s.idx = i;
+    s.chunks = 1;
+    if (ug > kRgMaxGroupUnits) {  // `ranged` only: the group is cut into items of 288 units
+      s.W = kRgWarps;
+      s.gpw = 1;
+      s.slice = kRgUnits;
+      s.gpi = 1;
+      s.chunks = (int)((ug + kRgMaxGroupUnits - 1) / kRgMaxGroupUnits);
+      s.item_units = kRgMaxGroupUnits;
+      continue;
+    }
     s.W = 1;
     while (s.W * kRgUnits < ug) s.W *= 2;
-    s.gpw = s.W == 1 ? std::max(1, kRgUnits / ug) : 1;
-    s.slice = (ug + s.W - 1) / s.W;
+    s.gpw = s.W == 1 ? std::max(1, kRgUnits / (int)ug) : 1;
+    s.slice = ((int)ug + s.W - 1) / s.W;
     s.gpi = (kRgWarps / s.W) * s.gpw;
     s.item_units = (int64_t)std::min(s.gpi, m[i].groups) * ug;
   }
@@ -1382,7 +1435,7 @@ static qb_status launch_regs(const HostWeight* m_all, int count_all, void* ws, i
     const int n = std::min(kRgMaxBatch, count - first);
     RegsBatch b;
     memset(&b, 0, sizeof(b));
-    int items = 0;
+    int64_t items = 0;
     for (int i = 0; i < n; ++i) {
       const Shape& s = sh[first + i];
       const HostWeight& h = m[s.idx];
@@ -1393,25 +1446,66 @@ static qb_status launch_regs(const HostWeight* m_all, int count_all, void* ws, i
       it.q0 = h.q0;
       it.ug = (int32_t)group_units(h);
       it.groups = h.groups;
-      it.item_begin = items;
+      it.item_begin = (int32_t)items;
       it.groups_per_item = s.gpi;
       it.team_warps = (int16_t)s.W;
       it.groups_per_warp = (int16_t)s.gpw;
       it.slice_units = (int16_t)s.slice;
       it.bits = (int16_t)h.bits;
-      items += (h.groups + s.gpi - 1) / s.gpi;
+      it.range_lo = h.range_lo;
+      it.range_hi = h.range_hi;
+      it.chunks = s.chunks;
+      items += s.chunks > 1 ? (int64_t)h.groups * s.chunks : (h.groups + s.gpi - 1) / s.gpi;
+    }
+    if (items > 0x7fffffff) {
+      set_last_error("weight batch too large for one launch (%lld items)", (long long)items);
+      return QB_ERR_INVALID;
     }
     b.ws = ws;
-    b.total_items = items;
+    b.total_items = (int32_t)items;
     b.count = n;
-    const unsigned grid = (unsigned)std::min(items, sm_count);
-    if (fake)
-      weight_regs_kernel<false, true><<<grid, kRgThreads, 0, stream>>>(b);
-    else
-      weight_regs_kernel<false, false><<<grid, kRgThreads, 0, stream>>>(b);
+    const unsigned grid = (unsigned)std::min<int64_t>(items, sm_count);
+    if (ranged) {
+      if (fake)
+        weight_regs_kernel<false, true, true><<<grid, kRgThreads, 0, stream>>>(b);
+      else
+        weight_regs_kernel<false, false, true><<<grid, kRgThreads, 0, stream>>>(b);
+    } else {
+      if (fake)
+        weight_regs_kernel<false, true, false><<<grid, kRgThreads, 0, stream>>>(b);
+      else
+        weight_regs_kernel<false, false, false><<<grid, kRgThreads, 0, stream>>>(b);
+    }
     QB_CUDA_TRY(cudaGetLastError());
   }
   return QB_OK;
+}
+
+// Register-resident path over any number of eligible matrices of any bit widths.  Matrices whose groups
+// need a cluster go to launches of their cluster size, matrices with caller-supplied ranges to launches of
+// the kernel that clamps.
+static qb_status launch_regs(const HostWeight* m_all, int count_all, void* ws, int sm_count, cudaStream_t stream,
+                             bool fake = false) {
+  std::vector<HostWeight> single, ranged, clustered[kRgMaxCluster + 1];
+  for (int i = 0; i < count_all; ++i) {
+    if (m_all[i].range_lo != nullptr) {
+      ranged.push_back(m_all[i]);
+      continue;
+    }
+    const int cl = regs_cluster_size(m_all[i]);
+    (cl <= 1 ? single : clustered[cl]).push_back(m_all[i]);
+  }
+  for (int cl = 2; cl <= kRgMaxCluster; ++cl) {
+    if (clustered[cl].empty()) continue;
+    qb_status st = launch_regs_cluster(clustered[cl].data(), (int)clustered[cl].size(), cl, ws, stream, fake);
+    if (st != QB_OK) return st;
+  }
+  if (!ranged.empty()) {
+    qb_status st = launch_regs_single(ranged.data(), (int)ranged.size(), true, ws, sm_count, stream, fake);
+    if (st != QB_OK) return st;
+  }
+  if (single.empty()) return QB_OK;
+  return launch_regs_single(single.data(), (int)single.size(), false, ws, sm_count, stream, fake);
 }
 
 // Single-read path over `count` matrices (<= kMaxWeightBatch) whose groups all fit the ring.
@@ -1817,8 +1911,14 @@ extern "C" int32_t qb_quantize_pack_weights_launch_count(const qb_weight_desc* d
   std::vector<qb::WeightJob> jobs;
   qb::plan_batch(descs, count, 148, regs, jobs);
   int per_cluster[qb::kRgMaxCluster + 1] = {};
-  for (const qb::HostWeight& h : regs) ++per_cluster[std::max(1, qb::regs_cluster_size(h))];
-  int32_t n = 0;
+  int ranged = 0;
+  for (const qb::HostWeight& h : regs) {
+    if (h.range_lo != nullptr)
+      ++ranged;
+    else
+      ++per_cluster[std::max(1, qb::regs_cluster_size(h))];
+  }
+  int32_t n = (ranged + qb::kRgMaxBatch - 1) / qb::kRgMaxBatch;
   for (int cl = 1; cl <= qb::kRgMaxCluster; ++cl) n += (per_cluster[cl] + qb::kRgMaxBatch - 1) / qb::kRgMaxBatch;
   for (const qb::WeightJob& j : jobs) n += j.single_read ? 1 : 2;
   return n;

@@ -204,6 +204,42 @@ def test_quantize_weights_cluster_path_nonfinite():
     assert qb.read_status(ws_bad2) == qb.QB_ERR_NONFINITE
 
 
+@pytest.mark.parametrize("N,K,G", [(74, 8192, 2),      # 2,368 units per group: nine items per group
+                                   (768, 768, 1),      # one range for the tensor: 4,608 units, sixteen items
+                                   (3072, 768, 128),   # 144 units: teams of eight warps
+                                   (70, 256, 70),      # two units per group: several groups per warp
+                                   (40, 3712, 2)])     # 580 units: three items per group, the last one ragged
+def test_quantize_weights_caller_ranges_any_group_size(N, K, G):
+    # ranges that clip about 4 % of the weights (Appendix A: the range "can be a subinterval of [min, max]");
+    # with ranges supplied nothing is reduced, so a group of any size stays on the single-read path
+    w = synth.weights(N, K, seed=N + K + G)
+    lo = np.quantile(w.reshape(G, -1), 0.02, axis=1).astype(np.float32)
+    hi = np.quantile(w.reshape(G, -1), 0.98, axis=1).astype(np.float32)
+    ws1 = qb.workspace(groups=max(32, G))
+    for bits in BITS:
+        packed, delta, q0 = gu.gpu_quantize_weights(w, bits, G, ws1, lo, hi)
+        st, codes, o_delta, o_q0 = oracle.quantize_weights(w, bits, G, lo, hi)
+        assert st == oracle.OK
+        assert np.array_equal(gu.words_np(packed), oracle.pack(codes, bits)), bits
+        assert np.array_equal(delta.cpu().numpy(), o_delta) and np.array_equal(q0.cpu().numpy(), o_q0)
+        wq, d2, z2 = qb.fake_quantize_weights(gu.dev(w), bits, G, ws1, gu.dev(lo), gu.dev(hi))
+        st, o_q, _, _ = oracle.fake_quantize_weights(w, bits, G, lo, hi)
+        assert np.array_equal(wq.cpu().numpy().view(np.uint32), o_q.view(np.uint32)), bits
+    assert qb.read_status(ws1) == qb.QB_OK
+    # a NaN among the weights is still reported, and so is a range that is not ordered
+    ws2, ws3 = qb.workspace(groups=max(32, G)), qb.workspace(groups=max(32, G))
+    bad = w.copy()
+    bad[N - 1, K - 3] = np.nan
+    gu.gpu_quantize_weights(bad, 4, G, ws2, lo, hi)
+    assert qb.read_status(ws2) == qb.QB_ERR_NONFINITE
+    assert oracle.quantize_weights(bad, 4, G, lo, hi)[0] == oracle.ERR_NONFINITE
+    lo_bad = lo.copy()
+    lo_bad[G - 1] = hi[G - 1] + 1.0
+    gu.gpu_quantize_weights(w, 4, G, ws3, lo_bad, hi)
+    assert qb.read_status(ws3) == qb.QB_ERR_NONFINITE
+    assert oracle.quantize_weights(w, 4, G, lo_bad, hi)[0] == oracle.ERR_NONFINITE
+
+
 def test_quantize_weights_register_path_more_matrices_than_one_launch():
     # 100 small matrices of mixed widths and group sizes: two launches
     shapes = [((24 + 8 * (i % 5)), 128 * (1 + i % 3), (2, 3, 4, 8)[i % 4], (1, 2, 4, 8)[(i // 4) % 4]) for i in range(100)]
