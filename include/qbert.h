@@ -104,10 +104,10 @@ qb_status qb_quantize_act(const float* x, int64_t M, int64_t K, int8_t* xq, floa
  *            max (Appendix A: the range "can be a subinterval of [min, max]"); values outside are
  *            clamped.  They must be finite with range_lo <= range_hi.
  * One kernel (the weights are read once and stay in registers between the range and the rounding)
- * when the groups have at most 294,912 weights each and the range is the group's own (groups above
- * 36,864 weights are held by a thread-block cluster); otherwise two kernels (per-group min/max
- * reduction into the workspace, then round/clamp/pack), or one that stages the group in shared
- * memory (caller-supplied ranges, groups of up to 49,152 weights).
+ * when the range is the group's own and the groups have at most 294,912 weights each (groups above
+ * 36,864 weights are held by a thread-block cluster), and always with caller-supplied ranges
+ * (nothing is reduced then); otherwise two kernels: per-group min/max reduction into the workspace,
+ * then round/clamp/pack.
  */
 qb_status qb_quantize_pack_weights(const float* w, int64_t N, int64_t K, int bits, int groups,
                                    const float* range_lo, const float* range_hi, uint32_t* packed,
@@ -142,14 +142,11 @@ typedef struct {
  * memory bandwidth.  `descs` is a HOST array; every element is validated before anything is launched;
  * each result equals the single call on the same arguments bit for bit.  Each activation tensor keeps
  * its own scale (per-tensor quantization).  Weight matrices of different bit widths may be mixed:
- * all matrices whose groups have at most 36,864 weights and take their own [min, max] go into one
- * launch per 96 matrices, whatever their widths (a mixed-precision stack is one launch); groups of up
- * to 294,912 weights likewise, one launch per cluster size.  The others
- * get launches per bit width; when these are several small single-read launches they run side by
- * side on streams the library creates once per device (host objects only), forking from and joining
- * `cuda_stream` inside the call (after the fork every side stream is joined, also when a launch in
- * between fails; the fork / launch / join sequence is serialised per device, so concurrent calls
- * from several host threads are safe).
+ * all matrices that take the single-kernel path of qb_quantize_pack_weights go into one launch per 96
+ * matrices, whatever their widths (a mixed-precision stack is one launch), separately for groups that
+ * fit one thread block, for each cluster size, and for caller-supplied ranges.  The others get a pair
+ * of launches per bit width and 32 matrices.  Everything is enqueued on `cuda_stream`; the call
+ * creates no host or device object.
  * Workspace: qb_workspace_bytes(0, 0, 0, 0, G) bytes with G = max(32, sum of `groups` over the batch).
  */
 qb_status qb_quantize_act_batch(const qb_act_desc* descs /*host*/, int32_t count, void* ws, size_t ws_bytes,
@@ -245,8 +242,8 @@ int32_t qb_quantize_act_launch_count(int32_t count);
 /*
  * How many kernel launches qb_quantize_pack_weights_batch issues for these matrices: host arithmetic on
  * the descriptors only (shapes, groups, bit widths, whether ranges are supplied), no GPU work.  (No
- * counterpart in the paper; for callers that count or budget launches.)  The plan is the one of a
- * 148-SM device.  Returns 0 for a null or empty batch or a descriptor with impossible shapes.
+ * counterpart in the paper; for callers that count or budget launches.)  Returns 0 for a null or
+ * empty batch or a descriptor with impossible shapes.
  */
 int32_t qb_quantize_pack_weights_launch_count(const qb_weight_desc* descs /*host*/, int32_t count);
 
@@ -314,9 +311,8 @@ qb_status qb_layer_linears_i8(const qb_linear_desc* descs /*host*/, const float*
  *   wq       dev fp32 [N][K], 16-byte aligned                     (written)
  *   delta,q0 dev fp32 [G]                                         (written)
  *   range_lo, range_hi: dev fp32 [G] or both NULL, as for qb_quantize_pack_weights.
- * One kernel (W read once, as in qb_quantize_pack_weights) for the group's own range and groups of
- * at most 294,912 weights; otherwise two: per-group min/max reduction into the workspace, then
- * round/clamp/dequantize.
+ * One kernel (W read once) in the cases where qb_quantize_pack_weights takes one; otherwise two:
+ * per-group min/max reduction into the workspace, then round/clamp/dequantize.
  *
  * Backward: grad_w = grad_wq where Clamp passes the weight through (range_lo[g] <= w <= range_hi[g],
  * both ends included), 0 where Clamp holds it at an end of the range; the rounding is treated as the

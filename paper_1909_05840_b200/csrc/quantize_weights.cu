@@ -1,12 +1,12 @@
 // qb_quantize_pack_weights(_batch): group-wise uniform quantizer Q (Section 3.3, Appendix A) and dense
 // k-bit packing (Table 1 counts exactly k bits per weight), for one matrix or a batch of matrices.
 //
-// Three paths, chosen per matrix on the host:
-//   weight_regs_kernel   groups of up to 288 units with their own [min, max]: one read of W, the group
-//                        stays in registers between the range and the rounding; any bit widths in one launch.
-//   weight_fused_kernel  groups of up to 384 units, also with caller-supplied ranges: one read of W through
-//                        a shared-memory ring.
-//   two passes           everything else (a range per tensor, say), below.
+// Two paths, chosen per matrix on the host:
+//   weight_regs_kernel   one read of W; any bit widths in one launch.  With the group's own [min, max]: groups
+//                        of up to 288 units stay in the registers of one CTA between the range and the
+//                        rounding, groups of up to 2,304 units in those of a thread-block cluster.  With
+//                        caller-supplied ranges: groups of any size (nothing to reduce).
+//   two passes           own ranges of larger groups (a range per tensor, say), below.
 //
 // Two-pass path: the matrices of a launch are walked as one sequence of "units" of 128 consecutive
 // elements of one row (one float4 per lane, fully coalesced; K % 128 == 0 so a unit never crosses a row).
@@ -21,16 +21,10 @@
 #include <algorithm>
 #include <atomic>
 #include <cstring>
-#include <mutex>
 #include <vector>
 
 #include "common.cuh"
 #include "ptx.cuh"
-
-#ifndef FUSED_WARPS
-#define FUSED_WARPS 16
-#define FUSED_RING_KB 192
-#endif
 
 namespace qb {
 
@@ -404,371 +398,6 @@ ste_backward_kernel(const float4* __restrict__ grad_q, const float4* __restrict_
     gq.z = (x.z >= l && x.z <= h) ? gq.z : 0.0f;
     gq.w = (x.w >= l && x.w <= h) ? gq.w : 0.0f;
     grad_w[i] = gq;
-  }
-}
-
-// ---- single-read path ------------------------------------------------------------------------------
-// When a whole group fits in shared memory the matrix is read from HBM once.  A persistent CTA per SM
-// takes groups round-robin.  Four producer lanes (in warps of their own) stream the CTA's groups as bulk
-// copies into a ring of shared-memory slots, running ahead into the next groups.  The sixteen consumer warps form teams of
-// 1, 2, 4, 8 or 16 warps (small groups: many small teams); the CTA's groups go to the teams in turn, so
-// one team reduces a range while another packs.  A team takes the range of its group from shared
-// memory as the chunks land, agrees on it through its named barrier, then quantizes the group from
-// shared memory in blocks of 8 units: the 4k-bit fields of a block are laid down in element order in
-// the warp's staging area, which for k = 2, 4, 8 is already the packed stream (copied out with 16-byte
-// stores) and for k = 3 is regrouped (eight 12-bit fields -> three words) on the way out.
-constexpr int kFusedConsumerWarps = FUSED_WARPS;
-constexpr int kFusedProducers = 4;                              // producer warps (one lane each issues copies)
-constexpr int kFusedThreads = 32 * (kFusedConsumerWarps + kFusedProducers);
-constexpr int kRingBytes = FUSED_RING_KB * 1024;
-constexpr int kMaxRingSlots = kRingBytes / 4096;               // 4 KB slots, or a quarter as many of 16 KB
-constexpr int kFusedMaxGroupUnits = kRingBytes / 512;           // 384 units = 49,152 weights per group
-constexpr int kStagingBytes = kFusedConsumerWarps * 1024;       // per consumer warp: fields of one block
-constexpr int kTailBarriers = 0;                                // full[kMaxRingSlots], empty[kMaxRingSlots]
-constexpr int kTailScratch = 16 * kMaxRingSlots;                // s_hi, s_lo: [2][kFusedConsumerWarps] each
-constexpr int kTailFlags = kTailScratch + 16 * kFusedConsumerWarps;  // abort flag, then issued[kMaxRingSlots]
-constexpr int kFusedTailBytes = (kTailFlags + 8 + 4 * kMaxRingSlots + 127) / 128 * 128;
-constexpr int kFusedSmemBytes = kRingBytes + kStagingBytes + kFusedTailBytes;
-constexpr long long kFusedWaitLimit = 4000000000ll;             // SM cycles, about 2 s
-
-struct FusedBatch {
-  WeightItem item[kMaxWeightBatch];
-  void* ws;
-  int32_t total_groups;
-  int32_t count;
-  int32_t team_warps;   // 1, 2, 4, 8 or 16
-  int32_t chunk_units;  // units of 128 weights per ring slot: 8 or 32
-  int32_t n_slots;      // kRingBytes / (chunk_units * 512)
-};
-
-// Bounded wait on an mbarrier phase; false when it expired (or, if asked, when another role gave up).
-__device__ __forceinline__ bool fused_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  if (ptx::mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  for (uint32_t spin = 1;; ++spin) {
-    if (ptx::mbar_try_wait(bar, parity)) return true;
-    if ((spin & 1023u) == 0u) {
-      if (abort_flag != nullptr && *abort_flag) return false;
-      if (clock64() - t0 > kFusedWaitLimit) return false;
-    }
-  }
-}
-
-// Bounded wait until a slot has been issued more than `index` times (`issued` is the slot's counter).
-__device__ __forceinline__ bool wait_issued(volatile int* issued, int index, volatile int* abort_flag) {
-  if (*issued > index) {
-    __threadfence_block();
-    return true;
-  }
-  const long long t0 = clock64();
-  for (uint32_t spin = 1;; ++spin) {
-    if (*issued > index) {
-      __threadfence_block();
-      return true;
-    }
-    if ((spin & 1023u) == 0u && (*abort_flag || clock64() - t0 > kFusedWaitLimit)) return false;
-  }
-}
-
-// Barrier over the threads of a team that also ORs a predicate over them: every thread gets the same
-// answer, so all of them leave the group loop together.  A one-warp team needs no named barrier.
-__device__ __forceinline__ bool team_sync_or(bool pred, int team_warps, int bar_id) {
-  if (team_warps == 1) return __any_sync(0xffffffffu, pred) != 0;
-  uint32_t res;
-  asm volatile(
-      "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.or.pred p, %2, %3, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(res)
-      : "r"((uint32_t)pred), "r"(bar_id), "r"(32 * team_warps)
-      : "memory");
-  return res != 0;
-}
-
-// min / max that return NaN when an input is NaN, so a single NaN survives to the group's range
-__device__ __forceinline__ float min_nan(float a, float b) {
-  float d;
-  asm("min.NaN.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
-  return d;
-}
-__device__ __forceinline__ float max_nan(float a, float b) {
-  float d;
-  asm("max.NaN.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
-  return d;
-}
-
-// Four codes of one float4 as a 4k-bit field (code i at bits [k*i, k*i + k)).  Adding 1.5 * 2^23 rounds
-// (X' - q0) * (1/Delta) to an integer, half to even, and leaves it in the low mantissa bits; the four bit
-// patterns are combined with integer multiply-adds and the constant they carry is taken off once.
-// With a range that covers the data no clamp is needed: 0 <= t <= L (1 + 3 * 2^-24) rounds into [0, L].
-template <int BITS, bool kClamp>
-__device__ __forceinline__ uint32_t quant_field(const float4 v, const GroupParams& gp) {
-  constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23, bit pattern 0x4B400000
-  constexpr uint32_t kCarry = 0x4B400000u * (1u + (1u << BITS) + (1u << (2 * BITS)) + (1u << (3 * BITS)));
-  const float e[4] = {v.x, v.y, v.z, v.w};
-  uint32_t bits[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    float x = e[i];
-    if (kClamp) x = fminf(fmaxf(x, gp.lo), gp.hi);                    // Clamp(X, q0, qmax)
-    const float t = __fmul_rn(__fsub_rn(x, gp.lo), gp.inv);          // (X' - q0) * (1/Delta)
-    bits[i] = __float_as_uint(__fadd_rn(t, kMagic));                  // round half to even
-  }
-  uint32_t f = bits[0] + (bits[1] << BITS) + (bits[2] << (2 * BITS)) + (bits[3] << (3 * BITS)) - kCarry;
-  if constexpr (BITS < 8) f &= (1u << (4 * BITS)) - 1u;
-  return f;
-}
-
-// A block of `nu` <= 8 units (1024 weights) that starts at `blk` in shared memory: quantize it and
-// write its packed words to `out` (the words of the block's first unit).  One warp; `stg` is the
-// warp's own 1 KB staging area, where the 4k-bit fields are laid down in element order.
-template <int BITS, bool kClamp>
-__device__ __forceinline__ void pack_block(const uint8_t* blk, uint8_t* stg, int nu, const GroupParams& gp,
-                                           uint32_t* __restrict__ out, int lane) {
-  const float4* src = reinterpret_cast<const float4*>(blk);
-#pragma unroll
-  for (int h = 0; h < 2; ++h) {
-    float4 v[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j)
-      if (4 * h + j < nu) v[j] = src[(4 * h + j) * 32 + lane];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      if (4 * h + j < nu) {
-        const uint32_t f = quant_field<BITS, kClamp>(v[j], gp);
-        const int fi = (4 * h + j) * 32 + lane;  // field index = element index / 4
-        if (BITS == 8) reinterpret_cast<uint32_t*>(stg)[fi] = f;
-        if (BITS == 4 || BITS == 3) reinterpret_cast<uint16_t*>(stg)[fi] = (uint16_t)f;
-        if (BITS == 2) stg[fi] = (uint8_t)f;
-      }
-    }
-  }
-  __syncwarp();
-  if (BITS == 3) {
-    // item = 32 codes = eight 12-bit fields held in 16-bit cells -> three words
-    if (lane < 4 * nu) {
-      const uint4 q = reinterpret_cast<const uint4*>(stg)[lane];
-      const uint32_t f0 = q.x & 0xffffu, f1 = q.x >> 16, f2 = q.y & 0xffffu, f3 = q.y >> 16;
-      const uint32_t f4 = q.z & 0xffffu, f5 = q.z >> 16, f6 = q.w & 0xffffu, f7 = q.w >> 16;
-      uint32_t* o = out + lane * 3;
-      o[0] = f0 | (f1 << 12) | (f2 << 24);
-      o[1] = (f2 >> 8) | (f3 << 4) | (f4 << 16) | (f5 << 28);
-      o[2] = (f5 >> 4) | (f6 << 8) | (f7 << 20);
-    }
-  } else {
-    const int n16 = nu * BITS;  // 16 * BITS bytes per unit
-    const uint4* pk = reinterpret_cast<const uint4*>(stg);
-    uint4* o = reinterpret_cast<uint4*>(out);
-    for (int i = lane; i < n16; i += 32) o[i] = pk[i];
-  }
-  __syncwarp();  // the staging area is free again
-}
-
-template <int BITS>
-__global__ void __launch_bounds__(kFusedThreads, 1)
-weight_fused_kernel(const __grid_constant__ FusedBatch b) {
-  constexpr int L = (1 << BITS) - 1;
-  constexpr int WORDS = 4 * BITS;
-  extern __shared__ __align__(1024) uint8_t fused_smem[];
-  const uint32_t ring = ptx::smem_u32(fused_smem);
-  uint8_t* const staging = fused_smem + kRingBytes + (threadIdx.x >> 5) * 1024;  // consumer warps only
-  uint8_t* tail = fused_smem + kRingBytes + kStagingBytes;
-  const uint32_t bar0 = ring + kRingBytes + kStagingBytes;
-  auto full = [&](int s) { return bar0 + 8u * (uint32_t)s; };
-  auto empty = [&](int s) { return bar0 + 8u * (uint32_t)(kMaxRingSlots + s); };
-  uint32_t* s_hi = reinterpret_cast<uint32_t*>(tail + kTailScratch);  // [2][kFusedConsumerWarps]
-  uint32_t* s_lo = s_hi + 2 * kFusedConsumerWarps;
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + kTailFlags);
-  volatile int* issued = reinterpret_cast<volatile int*>(tail + kTailFlags + 8);  // [kMaxRingSlots] copies issued into each slot
-  const int warp = threadIdx.x >> 5;
-  const int lane = threadIdx.x & 31;
-  const int W = b.team_warps;
-  const int chunk_units = b.chunk_units;
-  const int chunk_bytes = chunk_units * 512;
-  const int n_slots = b.n_slots;
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < n_slots; ++s) {
-      ptx::mbar_init(full(s), 1);
-      ptx::mbar_init(empty(s), (uint32_t)W);
-    }
-    *abort_flag = 0;
-    for (int s = 0; s < kMaxRingSlots; ++s) issued[s] = 0;
-    ptx::fence_mbar_init();
-  }
-  __syncthreads();
-
-  if (warp >= kFusedConsumerWarps) {
-    // ---------------- producers ---------------------------------------------------------------------
-    // One lane issues a copy every few hundred cycles, too slow for small chunks: several producer
-    // warps share the CTA's chunk sequence, producer p taking the chunks whose index is p modulo the
-    // number of producers.
-    if (lane == 0) {
-      const int me = warp - kFusedConsumerWarps;
-      int slot = 0, it = 0, use = 0, turn = 0;  // use: how often `slot` has been filled so far
-      bool ok = true;
-      for (int g = blockIdx.x; ok && g < b.total_groups; g += gridDim.x) {
-        while (it + 1 < b.count && g >= b.item[it + 1].group_begin) ++it;
-        const WeightItem& m = b.item[it];
-        const int ug = m.rows_per_group * m.units_per_row;
-        const char* src = reinterpret_cast<const char*>(m.w) + (int64_t)(g - m.group_begin) * ug * 512;
-        for (int u0 = 0; u0 < ug; u0 += chunk_units) {
-          if (turn == me) {
-            // the slot's previous copy may be another producer's: it must have been issued before the
-            // parity of its release can be waited for
-            if (!((use == 0 || wait_issued(issued + slot, use - 1, abort_flag)) &&
-                  fused_wait(empty(slot), (uint32_t)(use & 1) ^ 1u, abort_flag))) {
-              ok = false;
-              break;
-            }
-            const uint32_t bytes = (uint32_t)min(chunk_units, ug - u0) * 512u;
-            ptx::mbar_arrive_expect_tx(full(slot), bytes);
-            ptx::bulk_load_1d(ring + (uint32_t)(slot * chunk_bytes), src + (int64_t)u0 * 512, bytes, full(slot));
-            __threadfence_block();
-            issued[slot] = use + 1;  // consumers wait on a slot's barrier only once its copy has been issued
-          }
-          if (++turn == kFusedProducers) turn = 0;
-          if (++slot == n_slots) {
-            slot = 0;
-            ++use;
-          }
-        }
-      }
-      if (!ok) {
-        *abort_flag = 1;
-        report_status(b.ws, QB_ERR_TIMEOUT, 0x40000);
-      }
-    }
-  } else {
-    // ---------------- consumer teams ----------------------------------------------------------------
-    const float kInf = __int_as_float(0x7f800000);
-    const int n_teams = kFusedConsumerWarps / W;
-    const int team = warp / W;
-    const int tw = warp - team * W;     // warp inside the team
-    const int tthread = tw * 32 + lane;  // thread inside the team
-    const int tthreads = 32 * W;
-    int slot = 0, it = 0, flip = 0, turn = 0;
-    int use = 0;  // how often `slot` has been filled before the current chunk
-    uint32_t phase = 0;
-    bool ok = true;
-    for (int g = blockIdx.x; g < b.total_groups; g += gridDim.x) {
-      while (it + 1 < b.count && g >= b.item[it + 1].group_begin) ++it;
-      const WeightItem& m = b.item[it];
-      const int gl = g - m.group_begin;
-      const int ug = m.rows_per_group * m.units_per_row;
-      const int n_chunks = (ug + chunk_units - 1) / chunk_units;
-      const bool mine = turn == team;
-      if (++turn == n_teams) turn = 0;
-      if (!mine) {  // another team's group: step over its slots
-        slot += n_chunks;
-        if (slot >= n_slots) {
-          slot -= n_slots;
-          phase ^= 1u;
-          ++use;
-        }
-        continue;
-      }
-      // pass 1: range of the group as the chunks arrive (NaN propagates; Inf shows in the range)
-      float lo = kInf, hi = -kInf;
-      {
-        int s = slot, us = use;
-        uint32_t ph = phase;
-        for (int c = 0; c < n_chunks; ++c) {
-          // A team does not see the phases of the slots it steps over, and a parity wait cannot tell
-          // phase n from phase n - 2: wait for the copy to have been issued (the slot's previous phase
-          // is then complete), and only then for its bytes.
-          bool got = true;
-          if (lane == 0) got = wait_issued(issued + s, us, abort_flag) && fused_wait(full(s), ph, abort_flag);
-          got = __shfl_sync(0xffffffffu, got, 0);
-          if (!got) {
-            ok = false;
-            break;
-          }
-          (void)ptx::mbar_try_wait(full(s), ph);  // every lane observes the completed phase itself
-          const int n4 = min(chunk_units, ug - c * chunk_units) * 32;
-          const float4* src = reinterpret_cast<const float4*>(fused_smem + s * chunk_bytes);
-#pragma unroll 4
-          for (int i = tthread; i < n4; i += tthreads) {
-            const float4 v = src[i];
-            lo = min_nan(min_nan(lo, v.x), min_nan(v.y, min_nan(v.z, v.w)));
-            hi = max_nan(max_nan(hi, v.x), max_nan(v.y, max_nan(v.z, v.w)));
-          }
-          if (++s == n_slots) {
-            s = 0;
-            ph ^= 1u;
-            ++us;
-          }
-        }
-      }
-      // NaN anywhere makes hi NaN (encoded above every number); Inf shows as hi = +Inf or lo = -Inf
-      uint32_t e_hi = __reduce_max_sync(0xffffffffu, float_to_ordered(hi));
-      uint32_t e_lo = __reduce_max_sync(0xffffffffu, ~float_to_ordered(lo));
-      if (W > 1) {
-        if (lane == 0) {
-          s_hi[flip * kFusedConsumerWarps + warp] = e_hi;
-          s_lo[flip * kFusedConsumerWarps + warp] = e_lo;
-        }
-      }
-      // every warp of the team reaches this barrier for every group of the team, whatever happened
-      if (team_sync_or(!ok || *abort_flag != 0, W, 1 + team)) {
-        ok = false;
-        break;
-      }
-      if (W > 1) {
-        const uint32_t vh = lane < W ? s_hi[flip * kFusedConsumerWarps + team * W + lane] : 0u;
-        const uint32_t vl = lane < W ? s_lo[flip * kFusedConsumerWarps + team * W + lane] : 0u;
-        e_hi = __reduce_max_sync(0xffffffffu, vh);
-        e_lo = __reduce_max_sync(0xffffffffu, vl);
-        flip ^= 1;
-      }
-      const float g_hi = ordered_to_float(e_hi);
-      const float g_lo = ordered_to_float(~e_lo);
-      const bool publish = tthread == 0;
-      if (publish && !(fabsf(g_hi) <= 3.402823466e38f && fabsf(g_lo) <= 3.402823466e38f))
-        report_status(b.ws, QB_ERR_NONFINITE);
-      const bool from_caller = m.range_lo != nullptr;
-      GroupParams gp;
-      if (from_caller)
-        gp = finish_group(__ldg(m.range_lo + gl), __ldg(m.range_hi + gl), true, L, gl, m.delta, m.q0, publish, b.ws);
-      else
-        gp = finish_group(g_lo, g_hi, false, L, gl, m.delta, m.q0, publish, b.ws);
-      // pass 2: codes and packed words from shared memory; each slot is released behind the warp
-      uint32_t* const out = m.packed + (int64_t)gl * ug * WORDS;
-      const int blocks_per_chunk = chunk_units >> 3;
-      for (int c = 0; c < n_chunks; ++c) {
-        const int units_here = min(chunk_units, ug - c * chunk_units);
-        const uint8_t* const base = fused_smem + slot * chunk_bytes;
-        // blocks of 8 units, numbered through the whole group, go to the team's warps in turn
-        for (int bb = 0; bb * 8 < units_here; ++bb) {
-          if (((c * blocks_per_chunk + bb) & (W - 1)) != tw) continue;
-          const int u0 = bb * 8;
-          const int nu = min(8, units_here - u0);
-          uint32_t* const o = out + (int64_t)(c * chunk_units + u0) * WORDS;
-          if (from_caller)
-            pack_block<BITS, true>(base + u0 * 512, staging, nu, gp, o, lane);
-          else
-            pack_block<BITS, false>(base + u0 * 512, staging, nu, gp, o, lane);
-        }
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(empty(slot));
-        if (++slot == n_slots) {
-          slot = 0;
-          phase ^= 1u;
-          ++use;
-        }
-      }
-    }
-    if (!ok && lane == 0) {
-      *abort_flag = 1;
-      report_status(b.ws, QB_ERR_TIMEOUT, 0x50000);
-    }
-  }
-
-  // ---------------- teardown: after a failed wait, let the copies already issued land ------------------
-  __syncthreads();
-  if (threadIdx.x == 0 && *abort_flag) {
-    for (int s = 0; s < n_slots; ++s) {
-      const int n = issued[s];  // the last copy issued into slot s completes phase n - 1 of its barrier
-      if (n > 0) (void)fused_wait(full(s), (uint32_t)(n - 1) & 1u, nullptr);
-    }
   }
 }
 
@@ -1508,128 +1137,28 @@ static qb_status launch_regs(const HostWeight* m_all, int count_all, void* ws, i
   return launch_regs_single(single.data(), (int)single.size(), false, ws, sm_count, stream, fake);
 }
 
-// Single-read path over `count` matrices (<= kMaxWeightBatch) whose groups all fit the ring.
-static qb_status launch_fused(const HostWeight* m, int count, int bits, void* ws, int sm_count,
-                              cudaStream_t stream) {
-  FusedBatch b;
-  memset(&b, 0, sizeof(b));
-  int total_groups = 0;
-  for (int i = 0; i < count; ++i) {
-    WeightItem& it = b.item[i];
-    it.w = reinterpret_cast<const float4*>(m[i].w);
-    it.packed = m[i].packed;
-    it.delta = m[i].delta;
-    it.q0 = m[i].q0;
-    it.range_lo = m[i].range_lo;
-    it.range_hi = m[i].range_hi;
-    it.units = m[i].N * m[i].K / 128;
-    it.units_per_row = (int32_t)(m[i].K / 128);
-    it.rows_per_group = (int32_t)(m[i].N / m[i].groups);
-    it.group_begin = total_groups;
-    total_groups += m[i].groups;
-  }
-  b.count = count;
-  b.ws = ws;
-  b.total_groups = total_groups;
-  // small groups: 4 KB slots and small teams (many groups in flight); large groups: 16 KB slots
-  int64_t ug_max = 1;
-  for (int i = 0; i < count; ++i) ug_max = std::max(ug_max, group_units(m[i]));
-  b.chunk_units = ug_max <= 64 ? 8 : 32;
-  b.n_slots = kRingBytes / (b.chunk_units * 512);
-  b.team_warps = ug_max <= 16 ? 1 : (ug_max <= 64 ? 2 : (ug_max <= 160 ? 4 : 8));
-  const unsigned grid = (unsigned)(total_groups < sm_count ? total_groups : sm_count);
-#define QB_LAUNCH_FUSED(B)                                                                                  \
-  do {                                                                                                      \
-    QB_CUDA_TRY(cudaFuncSetAttribute(weight_fused_kernel<B>, cudaFuncAttributeMaxDynamicSharedMemorySize,  \
-                                     kFusedSmemBytes));                                                     \
-    weight_fused_kernel<B><<<grid, kFusedThreads, kFusedSmemBytes, stream>>>(b);                           \
-  } while (0)
-  switch (bits) {
-    case 2: QB_LAUNCH_FUSED(2); break;
-    case 3: QB_LAUNCH_FUSED(3); break;
-    case 4: QB_LAUNCH_FUSED(4); break;
-    case 8: QB_LAUNCH_FUSED(8); break;
-    default: return QB_ERR_INVALID;
-  }
-#undef QB_LAUNCH_FUSED
-  QB_CUDA_TRY(cudaGetLastError());
-  return QB_OK;
-}
-
-// Size class of a matrix for the single-read path (team size and slot size are per launch).
-static inline int fused_class(int64_t ug) { return ug <= 16 ? 0 : (ug <= 64 ? 1 : (ug <= 160 ? 2 : 3)); }
-
-// Matrices of one bit width (<= kMaxWeightBatch).  Those whose groups fit in shared memory take the
-// single-read path when together they have enough groups to occupy the GPU, one launch per size class
-// of groups (a class too small to be worth a launch joins the next larger one); the others take the
-// two-pass path.
-// One launch (single-read paths) or pair of launches (two-pass path) of a batch call.
+// One pair of launches of the two-pass path: matrices of one bit width (<= kMaxWeightBatch).
 struct WeightJob {
   HostWeight m[kMaxWeightBatch];
   int n;
   int bits;
-  bool single_read;
-  int64_t bytes;  // fp32 bytes read
 };
 
-static void push_job(std::vector<WeightJob>& jobs, const HostWeight* m, int n, int bits, bool single_read) {
+static void plan_weight_batch(const HostWeight* m, int count, int bits, std::vector<WeightJob>& jobs) {
   WeightJob j;
-  j.n = n;
+  j.n = count;
   j.bits = bits;
-  j.single_read = single_read;
-  j.bytes = 0;
-  for (int i = 0; i < n; ++i) {
-    j.m[i] = m[i];
-    j.bytes += m[i].N * m[i].K * 4;
-  }
+  for (int i = 0; i < count; ++i) j.m[i] = m[i];
   jobs.push_back(j);
 }
 
-// `max_ctas` caps the grid of a single-read job (a share of the SMs when jobs run side by side).
-static qb_status run_weight_job(const WeightJob& j, void* ws, int sm_count, int max_ctas, cudaStream_t stream) {
-  if (j.single_read) return launch_fused(j.m, j.n, j.bits, ws, max_ctas, stream);
-  return launch_two_pass(j.m, j.n, j.bits, ws, sm_count, stream);
-}
-
-static void plan_weight_batch(const HostWeight* m, int count, int bits, int sm_count, std::vector<WeightJob>& jobs) {
-  constexpr int64_t kClassWorthALaunch = 32ll << 20;  // bytes of fp32 weights
-  HostWeight fused[kMaxWeightBatch], rest[kMaxWeightBatch];
-  int cls[kMaxWeightBatch];
-  int nf = 0, nr = 0;
-  int64_t fused_groups = 0;
-  for (int i = 0; i < count; ++i) {
-    if (group_units(m[i]) <= kFusedMaxGroupUnits) {
-      cls[nf] = fused_class(group_units(m[i]));
-      fused[nf++] = m[i];
-      fused_groups += m[i].groups;
-    } else {
-      rest[nr++] = m[i];
-    }
+// The two-pass jobs of a call, one after the other (they share the range tables at the head of the workspace).
+static qb_status run_weight_jobs(const std::vector<WeightJob>& jobs, void* ws, int sm_count, cudaStream_t stream) {
+  for (const WeightJob& j : jobs) {
+    qb_status st = launch_two_pass(j.m, j.n, j.bits, ws, sm_count, stream);
+    if (st != QB_OK) return st;
   }
-  if (fused_groups * 2 < sm_count) {  // too few groups to spread over the SMs
-    for (int i = 0; i < nf; ++i) rest[nr++] = fused[i];
-    nf = 0;
-  }
-  if (nf > 0) {
-    HostWeight batch[kMaxWeightBatch];
-    int nb = 0;
-    int64_t bytes = 0;
-    for (int c = 0; c < 4; ++c) {
-      for (int i = 0; i < nf; ++i)
-        if (cls[i] == c) {
-          batch[nb++] = fused[i];
-          bytes += fused[i].N * fused[i].K * 4;
-        }
-      bool later = false;  // does a larger class still have matrices?
-      for (int i = 0; i < nf; ++i) later = later || cls[i] > c;
-      if (nb > 0 && (bytes >= kClassWorthALaunch || !later)) {
-        push_job(jobs, batch, nb, bits, true);
-        nb = 0;
-        bytes = 0;
-      }
-    }
-  }
-  if (nr > 0) push_job(jobs, rest, nr, bits, false);
+  return QB_OK;
 }
 
 static qb_status launch_weight_batch(const HostWeight* m, int count, int bits, void* ws, int sm_count,
@@ -1642,107 +1171,9 @@ static qb_status launch_weight_batch(const HostWeight* m, int count, int bits, v
   }
   if (rest.empty()) return QB_OK;
   std::vector<WeightJob> jobs;
-  plan_weight_batch(rest.data(), (int)rest.size(), bits, sm_count, jobs);
-  for (const WeightJob& j : jobs) {
-    qb_status st = run_weight_job(j, ws, sm_count, sm_count, stream);
-    if (st != QB_OK) return st;
-  }
-  return QB_OK;
-}
-
-// Streams and events for the single-read launches of one batch call that run side by side (host objects,
-// created once per device on first use; no device memory).
-constexpr int kMaxSideJobs = 8;
-struct WeightSideStreams {
-  cudaStream_t stream[kMaxSideJobs - 1];
-  cudaEvent_t done[kMaxSideJobs - 1];
-  cudaEvent_t fork;
-  bool ready;
-  std::mutex mu;  // one fork / launch / join sequence at a time per device: the events are shared
-};
-static qb_status weight_side_streams(WeightSideStreams** out) {
-  static WeightSideStreams per_dev[64];
-  int dev = 0;
-  QB_CUDA_TRY(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= 64) {
-    set_last_error("device ordinal %d out of range", dev);
-    return QB_ERR_CUDA;
-  }
-  WeightSideStreams& s = per_dev[dev];
-  std::lock_guard<std::mutex> lock(s.mu);
-  if (!s.ready) {
-    for (int i = 0; i < kMaxSideJobs - 1; ++i) {
-      QB_CUDA_TRY(cudaStreamCreateWithFlags(&s.stream[i], cudaStreamNonBlocking));
-      QB_CUDA_TRY(cudaEventCreateWithFlags(&s.done[i], cudaEventDisableTiming));
-    }
-    QB_CUDA_TRY(cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming));
-    s.ready = true;
-  }
-  *out = &s;
-  return QB_OK;
-}
-
-// The jobs of a batch call.  Several small single-read jobs (a mixed-precision stack: one or two per bit
-// width, tens of MB each) run side by side on SM shares in proportion to their bytes, so that their
-// start-up and drain overlap; they touch nothing in the workspace but the status word.  Anything else
-// runs one job after the other (the two-pass jobs share the range tables at the head of the workspace).
-static qb_status run_weight_jobs(const std::vector<WeightJob>& jobs, void* ws, int sm_count, cudaStream_t stream) {
-  constexpr int64_t kSmallJob = 160ll << 20;
-  const int n = (int)jobs.size();
-  bool side = n >= 2 && n <= kMaxSideJobs && n * 8 <= sm_count;
-  int64_t total = 0;
-  for (const WeightJob& j : jobs) {
-    side = side && j.single_read && j.bytes <= kSmallJob;
-    total += j.bytes;
-  }
-  if (!side) {
-    for (const WeightJob& j : jobs) {
-      qb_status st = run_weight_job(j, ws, sm_count, sm_count, stream);
-      if (st != QB_OK) return st;
-    }
-    return QB_OK;
-  }
-  std::vector<int> share(n);
-  int used = 0;
-  for (int i = 0; i < n; ++i) {
-    int64_t sh = (int64_t)sm_count * jobs[i].bytes / total;
-    if (sh < 8) sh = 8;
-    share[i] = (int)sh;
-    used += share[i];
-  }
-  while (used > sm_count) {  // the minimum share can overshoot: take from the largest
-    int big = 0;
-    for (int i = 1; i < n; ++i)
-      if (share[i] > share[big]) big = i;
-    --share[big];
-    --used;
-  }
-  for (int i = 0; used < sm_count; i = (i + 1) % n, ++used) ++share[i];
-  WeightSideStreams* sd = nullptr;
-  qb_status st = weight_side_streams(&sd);
-  if (st != QB_OK) return st;
-  // Two host threads on one device would interleave their records of the shared events: serialise the
-  // whole fork / launch / join sequence.  After the fork every side stream is joined whatever fails in
-  // between, so that the caller's stream never runs ahead of work the call put on a side stream.
-  std::lock_guard<std::mutex> lock(sd->mu);
-  qb_status first_error = QB_OK;
-  auto note = [&](cudaError_t e, const char* what) {
-    if (e != cudaSuccess && first_error == QB_OK) first_error = cuda_fail(e, what);
-    return e == cudaSuccess;
-  };
-  if (!note(cudaEventRecord(sd->fork, stream), "cudaEventRecord(fork)")) return first_error;  // nothing forked yet
-  bool forked[kMaxSideJobs] = {};
-  for (int i = 1; i < n; ++i) forked[i] = note(cudaStreamWaitEvent(sd->stream[i - 1], sd->fork, 0), "cudaStreamWaitEvent(fork)");
-  for (int i = 0; i < n && first_error == QB_OK; ++i) {
-    st = run_weight_job(jobs[i], ws, sm_count, share[i], i == 0 ? stream : sd->stream[i - 1]);
-    if (st != QB_OK && first_error == QB_OK) first_error = st;
-  }
-  for (int i = 1; i < n; ++i) {  // always join what was forked, also after an error
-    if (!forked[i]) continue;
-    if (note(cudaEventRecord(sd->done[i - 1], sd->stream[i - 1]), "cudaEventRecord(done)"))
-      note(cudaStreamWaitEvent(stream, sd->done[i - 1], 0), "cudaStreamWaitEvent(done)");
-  }
-  return first_error;
+  for (size_t i = 0; i < rest.size(); i += kMaxWeightBatch)
+    plan_weight_batch(rest.data() + i, (int)std::min<size_t>(kMaxWeightBatch, rest.size() - i), bits, jobs);
+  return run_weight_jobs(jobs, ws, sm_count, stream);
 }
 
 // Fake quantization of one matrix: the register-resident kernel where the groups fit it, else the range
@@ -1836,11 +1267,12 @@ extern "C" qb_status qb_quantize_pack_weights(const float* w, int64_t N, int64_t
 namespace qb {
 
 // The launch plan of a batch: the matrices of the register-resident path, and the jobs of the others.
-static void plan_batch(const qb_weight_desc* descs, int count, int sms, std::vector<HostWeight>& regs,
+static void plan_batch(const qb_weight_desc* descs, int count, std::vector<HostWeight>& regs,
                        std::vector<WeightJob>& jobs) {
-  // Matrices with their own ranges and groups of at most 288 units: the register-resident path, all bit
-  // widths in the same launches.  The others: launches of one bit width, at most kMaxWeightBatch matrices
-  // each; the range tables of a launch reuse the head of the workspace (launches on one stream run in order).
+  // Matrices that fit the register-resident path (see regs_eligible): all bit widths in the same launches.
+  // The others (own ranges over groups too large for a cluster) take the two passes: launches of one bit
+  // width, at most kMaxWeightBatch matrices each; the range tables of a launch reuse the head of the
+  // workspace (launches on one stream run in order).
   std::vector<int> order;
   for (int i = 0; i < count; ++i) {
     const qb_weight_desc& d = descs[i];
@@ -1862,7 +1294,7 @@ static void plan_batch(const qb_weight_desc* descs, int count, int sms, std::vec
       m[n++] = HostWeight{d.w, d.N, d.K, d.groups, d.range_lo, d.range_hi, d.packed, d.delta, d.q0, d.bits};
       ++i;
     }
-    plan_weight_batch(m, n, bits, sms, jobs);
+    plan_weight_batch(m, n, bits, jobs);
   }
 }
 
@@ -1892,7 +1324,7 @@ extern "C" qb_status qb_quantize_pack_weights_batch(const qb_weight_desc* descs,
   if (st != QB_OK) return st;
   std::vector<qb::HostWeight> regs;
   std::vector<qb::WeightJob> jobs;
-  qb::plan_batch(descs, count, sms, regs, jobs);
+  qb::plan_batch(descs, count, regs, jobs);
   if (!regs.empty()) {
     st = qb::launch_regs(regs.data(), (int)regs.size(), ws, sms, (cudaStream_t)cuda_stream);
     if (st != QB_OK) return st;
@@ -1909,7 +1341,7 @@ extern "C" int32_t qb_quantize_pack_weights_launch_count(const qb_weight_desc* d
   }
   std::vector<qb::HostWeight> regs;
   std::vector<qb::WeightJob> jobs;
-  qb::plan_batch(descs, count, 148, regs, jobs);
+  qb::plan_batch(descs, count, regs, jobs);
   int per_cluster[qb::kRgMaxCluster + 1] = {};
   int ranged = 0;
   for (const qb::HostWeight& h : regs) {
@@ -1920,7 +1352,7 @@ extern "C" int32_t qb_quantize_pack_weights_launch_count(const qb_weight_desc* d
   }
   int32_t n = (ranged + qb::kRgMaxBatch - 1) / qb::kRgMaxBatch;
   for (int cl = 1; cl <= qb::kRgMaxCluster; ++cl) n += (per_cluster[cl] + qb::kRgMaxBatch - 1) / qb::kRgMaxBatch;
-  for (const qb::WeightJob& j : jobs) n += j.single_read ? 1 : 2;
+  n += 2 * (int32_t)jobs.size();
   return n;
 }
 
