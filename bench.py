@@ -714,6 +714,26 @@ def run_quantizer_sweep(args):
             table[f"k{bits}_g{groups}"] = {"ms": ms, "GBps": gbs, "frac_hbm": gbs / peaks["hbm_gbs"]}
             launches += qb.quantize_pack_weights_launch_count(arr) * (3 + steps)
             del items, arr
+    # caller-supplied ranges (Appendix A: the range "can be a subinterval of [min, max]"): 4 bits, 128 groups
+    # per matrix, every group clipped to [-0.05, 0.05]
+    ws = qb.workspace(groups=max(32, 128 * len(shapes)), device=dev)
+    lo_t = torch.full((128,), -0.05, device=dev)
+    hi_t = torch.full((128,), 0.05, device=dev)
+    arr = (qb.WeightDescC * len(w_dev))()
+    keep = []
+    for i, w in enumerate(w_dev):
+        pk = torch.empty((w.shape[0], w.shape[1] * 4 // 32), dtype=torch.int32, device=dev)
+        dl = torch.empty(128, dtype=torch.float32, device=dev)
+        z0 = torch.empty(128, dtype=torch.float32, device=dev)
+        keep.append((pk, dl, z0))
+        arr[i] = qb.WeightDescC(w.data_ptr(), w.shape[0], w.shape[1], 4, 128, lo_t.data_ptr(), hi_t.data_ptr(),
+                                pk.data_ptr(), dl.data_ptr(), z0.data_ptr())
+    ms = timed(lambda: qb.quantize_pack_weights_batch(arr, ws))
+    assert qb.read_status(ws) == qb.QB_OK
+    gbs = params * 4.5 / (ms * 1e-3) / 1e9
+    table["k4_g128_caller_ranges"] = {"ms": ms, "GBps": gbs, "frac_hbm": gbs / peaks["hbm_gbs"]}
+    launches += qb.quantize_pack_weights_launch_count(arr) * (3 + steps)
+    del keep, arr
     M, K = synth.QUANTIZER_SWEEP_ACT
     x = torch.from_numpy(synth.activations(M, K, synth.seed_for(4))).to(dev)
     xq = torch.empty((M, K), dtype=torch.int8, device=dev)
