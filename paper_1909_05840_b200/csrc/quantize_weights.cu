@@ -8,16 +8,13 @@
 //                        caller-supplied ranges: groups of any size (nothing to reduce).
 //   two passes           own ranges of larger groups (a range per tensor, say), below.
 //
-// Two-pass path: the matrices of a launch are walked as one sequence of "units" of 128 consecutive
-// elements of one row (one float4 per lane, fully coalesced; K % 128 == 0 so a unit never crosses a row).
-// Each warp owns a contiguous run of units, so it crosses few group (and matrix) boundaries.
-//
-// Kernel 1  weight_range_kernel  running min/max per lane, warp reduction when the group changes,
-//                                atomicMax on order-preserving integer encodings in the workspace
-//                                (block-level merge of the final partials first).
-// Kernel 2  weight_pack_kernel   re-reads the unit (from L2 for BERT-sized matrices), computes four
-//                                codes per lane, and assembles the unit's 4k output words with warp
-//                                shuffles so that the stores are contiguous 16k-byte runs.
+// Two-pass path, first pass: the matrices of a launch are walked as one sequence of "units" of 128
+// consecutive elements of one row (one float4 per lane, fully coalesced; K % 128 == 0 so a unit never
+// crosses a row).  Each warp owns a contiguous run of units, so it crosses few group (and matrix)
+// boundaries: weight_range_kernel keeps a running min/max per lane, reduces over the warp when the group
+// changes and publishes with atomicMax on order-preserving integer encodings in the workspace (block-level
+// merge of the final partials first).  Second pass: weight_regs_kernel in its supplied-ranges form, reading
+// those encodings (the matrix comes from L2 as far as L2 holds it).
 #include <algorithm>
 #include <atomic>
 #include <cstring>
@@ -227,161 +224,7 @@ __device__ __forceinline__ float group_step(const GroupParams& gp, int bits_leve
   return d > 0.0f ? d : 1.0f;
 }
 
-// Group g of a matrix: range from the caller's tables or from the reduced encodings in the workspace.
-__device__ __forceinline__ GroupParams load_group(int g, int bits_levels, const uint32_t* __restrict__ hi_enc,
-                                                  const uint32_t* __restrict__ lo_inv,
-                                                  const float* __restrict__ range_lo,
-                                                  const float* __restrict__ range_hi, float* __restrict__ delta,
-                                                  float* __restrict__ q0, bool publish, void* ws) {
-  if (range_lo != nullptr)
-    return finish_group(__ldg(range_lo + g), __ldg(range_hi + g), true, bits_levels, g, delta, q0, publish, ws);
-  return finish_group(ordered_to_float(~lo_inv[g]), ordered_to_float(hi_enc[g]), false, bits_levels, g, delta, q0,
-                      publish, ws);
-}
-
-// Four codes of this lane (Appendix A's Q: clamp, subtract q0, scale by 1/Delta, round half to even)
-// and the output word `lane` of the unit of 128 codes, gathered from the lanes whose 4k-bit fields
-// overlap stream bits [32*lane, 32*lane + 32).  Lanes >= 4k return a word nobody stores.
-template <int BITS>
-__device__ __forceinline__ uint32_t pack_unit(const float4 v, const GroupParams& gp, int lane, int first_src) {
-  constexpr int L = (1 << BITS) - 1;
-  constexpr int F = 4 * BITS;
-  constexpr int NSRC = BITS == 8 ? 1 : (BITS == 4 ? 2 : 4);
-  const float e[4] = {v.x, v.y, v.z, v.w};
-  uint32_t field = 0;
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const float xc = fminf(fmaxf(e[i], gp.lo), gp.hi);        // Clamp(X, q0, qmax)
-    const float t = __fmul_rn(__fsub_rn(xc, gp.lo), gp.inv);  // (X' - q0) * (1/Delta)
-    int c = __float2int_rn(t);                                // round half to even
-    c = min(max(c, 0), L);
-    field |= (uint32_t)c << (BITS * i);
-  }
-  uint32_t word = 0;
-#pragma unroll
-  for (int s = 0; s < NSRC; ++s) {
-    const int src = first_src + s;
-    const uint32_t f = __shfl_sync(0xffffffffu, field, src & 31);
-    const int off = src * F - 32 * lane;  // position of that field relative to the word
-    if (off >= 0) {
-      if (off < 32) word |= f << off;
-    } else {
-      word |= f >> (-off);
-    }
-  }
-  return word;
-}
-
-template <int BITS>
-__global__ void __launch_bounds__(kWqThreads)
-weight_pack_kernel(const __grid_constant__ WeightBatch b) {
-  constexpr int L = (1 << BITS) - 1;
-  constexpr int F = 4 * BITS;          // bits contributed by one lane (four codes)
-  constexpr int WORDS = 4 * BITS;      // output words per unit of 128 codes
-  const int lane = threadIdx.x & 31;
-  const int64_t gwarp = (int64_t)blockIdx.x * kWqWarps + (threadIdx.x >> 5);
-  int64_t u = gwarp * b.units_per_warp;
-  int64_t u_end = u + b.units_per_warp;
-  if (u_end > b.units_total) u_end = b.units_total;
-  if (u >= u_end) return;
-
-  UnitWalk pos;
-  const uint64_t pol = policy_evict_first();
-  pos.seek(b, u);
-  int cur_g = -1;
-  GroupParams gp{0.f, 0.f, 1.f};
-
-  // which lanes feed output word `lane` of a unit (stream bits [32*lane, 32*lane + 32))
-  const int first_src = (32 * lane) / F;
-
-  while (u < u_end) {
-    const WeightItem& m = b.item[pos.it];
-    const int nload = (int)min(min((int64_t)4, u_end - u), m.units - pos.u_local);
-    float4 v[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j)
-      if (j < nload) v[j] = ldg_policy(m.w + (pos.u_local + j) * 32 + lane, pol);
-    uint32_t* const out_base = m.packed + pos.u_local * WORDS;
-    const int group_begin = m.group_begin;
-    const float* const rlo = m.range_lo;
-    const float* const rhi = m.range_hi;
-    float* const dl = m.delta;
-    float* const qz = m.q0;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      if (j < nload) {
-        if (pos.g != cur_g) {  // warp-uniform
-          cur_g = pos.g;
-          // the warp that handles the first unit of the group publishes Delta and q0
-          const bool publish = lane == 0 && pos.row_in_group == 0 && pos.col_unit == 0;
-          const int gl = cur_g - group_begin;
-          gp = load_group(gl, L, b.hi_enc + group_begin, b.lo_inv + group_begin, rlo, rhi, dl, qz, publish, b.ws);
-        }
-        const uint32_t word = pack_unit<BITS>(v[j], gp, lane, first_src);
-        if (lane < WORDS) out_base[j * WORDS + lane] = word;
-        pos.advance(b);
-      }
-    }
-    u += nload;
-  }
-}
-
-// ---- fake quantization (quantization-aware fine-tuning) ------------------------------------------------
-// Forward: Q(W) = Delta * X^I + q0 in fp32 (Appendix A), same walk and same codes as weight_pack_kernel;
-// the four values of a lane are written as one float4 (`packed` of the item points to the fp32 output).
-__global__ void __launch_bounds__(kWqThreads)
-weight_fake_kernel(const __grid_constant__ WeightBatch b, int levels) {
-  const int lane = threadIdx.x & 31;
-  const int64_t gwarp = (int64_t)blockIdx.x * kWqWarps + (threadIdx.x >> 5);
-  int64_t u = gwarp * b.units_per_warp;
-  int64_t u_end = u + b.units_per_warp;
-  if (u_end > b.units_total) u_end = b.units_total;
-  if (u >= u_end) return;
-  UnitWalk pos;
-  const uint64_t pol = policy_evict_first();
-  pos.seek(b, u);
-  int cur_g = -1;
-  GroupParams gp{0.f, 0.f, 1.f};
-  float d = 1.0f;
-  while (u < u_end) {
-    const WeightItem& m = b.item[pos.it];
-    const int nload = (int)min(min((int64_t)4, u_end - u), m.units - pos.u_local);
-    float4 v[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j)
-      if (j < nload) v[j] = ldg_policy(m.w + (pos.u_local + j) * 32 + lane, pol);
-    float4* const out_base = reinterpret_cast<float4*>(m.packed) + pos.u_local * 32;
-    const int group_begin = m.group_begin;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      if (j < nload) {
-        if (pos.g != cur_g) {  // warp-uniform
-          cur_g = pos.g;
-          const bool publish = lane == 0 && pos.row_in_group == 0 && pos.col_unit == 0;
-          gp = load_group(cur_g - group_begin, levels, b.hi_enc + group_begin, b.lo_inv + group_begin, m.range_lo,
-                          m.range_hi, m.delta, m.q0, publish, b.ws);
-          // Delta as finish_group publishes it (a constant group comes back with hi == lo: Delta = 1)
-          d = __fdiv_rn(__fsub_rn(gp.hi, gp.lo), (float)levels);
-          if (!(d > 0.0f)) d = 1.0f;
-        }
-        const float e[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
-        float q[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float xc = fminf(fmaxf(e[i], gp.lo), gp.hi);        // Clamp(X, q0, qmax)
-          const float t = __fmul_rn(__fsub_rn(xc, gp.lo), gp.inv);  // (X' - q0) * (1/Delta)
-          int c = __float2int_rn(t);                                // round half to even
-          c = min(max(c, 0), levels);
-          q[i] = __fmaf_rn(d, (float)c, gp.lo);                     // Delta * X^I + q0
-        }
-        out_base[j * 32 + lane] = make_float4(q[0], q[1], q[2], q[3]);
-        pos.advance(b);
-      }
-    }
-    u += nload;
-  }
-}
-
+// ---- straight-through backward (quantization-aware fine-tuning) ----------------------------------------
 // Backward (straight-through estimator): the gradient passes where Clamp passes X (lo_g <= x <= hi_g).
 __global__ void __launch_bounds__(256)
 ste_backward_kernel(const float4* __restrict__ grad_q, const float4* __restrict__ w, int64_t n4, int64_t k4,
@@ -438,8 +281,8 @@ struct RegsItem {
   int16_t bits;
   const float* range_lo;    // caller-supplied ranges (the kernel that clamps), else null
   const float* range_hi;
-  int32_t chunks;           // caller-supplied ranges only: a group of more than 288 units is cut into this many items
-  int32_t pad;
+  int32_t chunks;           // supplied ranges only: a group of more than 288 units is cut into this many items
+  int32_t encoded;          // supplied ranges are the range pass's order-preserving encodings (max, inverted min)
 };
 
 struct RegsBatch {
@@ -701,9 +544,20 @@ __device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v
 // writes its range into every CTA's shared memory and the cluster's barrier publishes them.  Every CTA of a
 // cluster runs the same number of items, so the barriers pair up; the last one also keeps a CTA's shared
 // memory alive until no peer writes to it any more.
+// Supplied range of group g: the caller's floats, or the encodings the range pass of the two-pass path left.
+__device__ __forceinline__ GroupParams supplied_group(const RegsItem& m, int g, int L, bool publish, void* ws) {
+  if (m.encoded) {
+    const float lo = ordered_to_float(~__ldg(reinterpret_cast<const uint32_t*>(m.range_lo) + g));
+    const float hi = ordered_to_float(__ldg(reinterpret_cast<const uint32_t*>(m.range_hi) + g));
+    return finish_group(lo, hi, false, L, g, m.delta, m.q0, publish, ws);
+  }
+  return finish_group(__ldg(m.range_lo + g), __ldg(m.range_hi + g), true, L, g, m.delta, m.q0, publish, ws);
+}
+
 // FAKE: the fp32 fake-quantized matrix is written instead of packed words (`packed` of the item points to it).
-// CLAMP: the ranges are the caller's (`range_lo`, `range_hi` of the item): no reduction and no exchange, the
-// weights are clamped into the range, and the pass over the registers only looks for NaN and Inf.
+// CLAMP: the ranges are supplied (`range_lo`, `range_hi` of the item: the caller's, or what the range pass of
+// the two-pass path found): no reduction and no exchange, the weights are clamped into the range, and the pass
+// over the registers only looks for NaN and Inf.
 template <bool CLUSTER, bool FAKE, bool CLAMP>
 __global__ void __launch_bounds__(kRgThreads, 1)
 weight_regs_kernel(const __grid_constant__ RegsBatch b) {
@@ -771,8 +625,7 @@ weight_regs_kernel(const __grid_constant__ RegsBatch b) {
       if (lane < s.ng) {
         GroupParams gp;
         if (CLAMP) {
-          const int g = s.first_group + lane;
-          gp = finish_group(__ldg(m.range_lo + g), __ldg(m.range_hi + g), true, L, g, m.delta, m.q0, true, b.ws);
+          gp = supplied_group(m, s.first_group + lane, L, true, b.ws);
         } else {
           const float g_hi = ordered_to_float(my_hi);
           const float g_lo = ordered_to_float(~my_lo);
@@ -841,8 +694,7 @@ weight_regs_kernel(const __grid_constant__ RegsBatch b) {
       const bool publish = s.first_unit == 0 && lane == 0;
       GroupParams gp;
       if (CLAMP) {
-        gp = finish_group(__ldg(m.range_lo + s.first_group), __ldg(m.range_hi + s.first_group), true, L, s.first_group,
-                          m.delta, m.q0, publish, b.ws);
+        gp = supplied_group(m, s.first_group, L, publish, b.ws);
       } else {
         const float g_hi = ordered_to_float(e_hi);
         const float g_lo = ordered_to_float(~e_lo);
@@ -879,11 +731,15 @@ struct HostWeight {
   int bits;
 };
 
-// Two-pass path: one pair of launches over `count` matrices (<= kMaxWeightBatch) of the same bit width.
-// Their range tables sit back to back in the workspace: maxima at ws + kWsRangeOff, inverted minima
-// after them.
-static qb_status launch_two_pass(const HostWeight* m, int count, int bits, void* ws, int sm_count,
-                                 cudaStream_t stream) {
+static qb_status launch_regs_single(const HostWeight* m, int count, bool ranged, void* ws, int sm_count,
+                                    cudaStream_t stream, bool fake, bool encoded);
+
+// Two-pass path (own ranges over groups too large for a cluster): one pair of launches over `count`
+// matrices (<= kMaxWeightBatch).  Their range tables sit back to back in the workspace: maxima at
+// ws + kWsRangeOff, inverted minima after them.  The second pass is the register-resident kernel in its
+// supplied-ranges form, reading those tables.
+static qb_status launch_two_pass(const HostWeight* m, int count, void* ws, int sm_count, cudaStream_t stream,
+                                 bool fake = false) {
   WeightBatch b;
   memset(&b, 0, sizeof(b));
   int total_groups = 0;
@@ -921,15 +777,13 @@ static qb_status launch_two_pass(const HostWeight* m, int count, int bits, void*
 
   weight_range_kernel<<<blocks, kWqThreads, 0, stream>>>(b);
   QB_CUDA_TRY(cudaGetLastError());
-  switch (bits) {
-    case 2: weight_pack_kernel<2><<<blocks, kWqThreads, 0, stream>>>(b); break;
-    case 3: weight_pack_kernel<3><<<blocks, kWqThreads, 0, stream>>>(b); break;
-    case 4: weight_pack_kernel<4><<<blocks, kWqThreads, 0, stream>>>(b); break;
-    case 8: weight_pack_kernel<8><<<blocks, kWqThreads, 0, stream>>>(b); break;
-    default: return QB_ERR_INVALID;
+  HostWeight second[kMaxWeightBatch];
+  for (int i = 0; i < count; ++i) {
+    second[i] = m[i];
+    second[i].range_lo = reinterpret_cast<const float*>(b.lo_inv + b.item[i].group_begin);
+    second[i].range_hi = reinterpret_cast<const float*>(b.hi_enc + b.item[i].group_begin);
   }
-  QB_CUDA_TRY(cudaGetLastError());
-  return QB_OK;
+  return launch_regs_single(second, count, true, ws, sm_count, stream, fake, true);
 }
 
 static inline int64_t group_units(const HostWeight& h) { return (h.N / h.groups) * (h.K / 128); }
@@ -1032,7 +886,7 @@ static qb_status launch_regs_cluster(const HostWeight* m, int count, int cl, voi
 // groups of any size: `ranged`), any bit widths: launches of up to kRgMaxBatch matrices, inside a launch
 // the matrices with the largest CTA items first.
 static qb_status launch_regs_single(const HostWeight* m, int count, bool ranged, void* ws, int sm_count,
-                                    cudaStream_t stream, bool fake) {
+                                    cudaStream_t stream, bool fake, bool encoded) {
   struct Shape {
     int idx, W, gpw, slice, gpi, chunks;
     int64_t item_units;
@@ -1084,6 +938,7 @@ static qb_status launch_regs_single(const HostWeight* m, int count, bool ranged,
       it.range_lo = h.range_lo;
       it.range_hi = h.range_hi;
       it.chunks = s.chunks;
+      it.encoded = encoded ? 1 : 0;
       items += s.chunks > 1 ? (int64_t)h.groups * s.chunks : (h.groups + s.gpi - 1) / s.gpi;
     }
     if (items > 0x7fffffff) {
@@ -1130,11 +985,11 @@ static qb_status launch_regs(const HostWeight* m_all, int count_all, void* ws, i
     if (st != QB_OK) return st;
   }
   if (!ranged.empty()) {
-    qb_status st = launch_regs_single(ranged.data(), (int)ranged.size(), true, ws, sm_count, stream, fake);
+    qb_status st = launch_regs_single(ranged.data(), (int)ranged.size(), true, ws, sm_count, stream, fake, false);
     if (st != QB_OK) return st;
   }
   if (single.empty()) return QB_OK;
-  return launch_regs_single(single.data(), (int)single.size(), false, ws, sm_count, stream, fake);
+  return launch_regs_single(single.data(), (int)single.size(), false, ws, sm_count, stream, fake, false);
 }
 
 // One pair of launches of the two-pass path: matrices of one bit width (<= kMaxWeightBatch).
@@ -1155,7 +1010,7 @@ static void plan_weight_batch(const HostWeight* m, int count, int bits, std::vec
 // The two-pass jobs of a call, one after the other (they share the range tables at the head of the workspace).
 static qb_status run_weight_jobs(const std::vector<WeightJob>& jobs, void* ws, int sm_count, cudaStream_t stream) {
   for (const WeightJob& j : jobs) {
-    qb_status st = launch_two_pass(j.m, j.n, j.bits, ws, sm_count, stream);
+    qb_status st = launch_two_pass(j.m, j.n, ws, sm_count, stream);
     if (st != QB_OK) return st;
   }
   return QB_OK;
@@ -1176,48 +1031,14 @@ static qb_status launch_weight_batch(const HostWeight* m, int count, int bits, v
   return run_weight_jobs(jobs, ws, sm_count, stream);
 }
 
-// Fake quantization of one matrix: the register-resident kernel where the groups fit it, else the range
-// kernel of the two-pass path, then weight_fake_kernel.
+// Fake quantization of one matrix: the register-resident kernel where the groups fit it, else the two passes.
 static qb_status launch_fake_quantize(const float* w, int64_t N, int64_t K, int bits, int groups,
                                       const float* range_lo, const float* range_hi, float* wq, float* delta,
                                       float* q0, void* ws, int sm_count, cudaStream_t stream) {
-  {
-    // groups that fit the registers of a CTA or of a cluster, with their own ranges: one read of W
-    const HostWeight h{w, N, K, groups, range_lo, range_hi, reinterpret_cast<uint32_t*>(wq), delta, q0, bits};
-    if (regs_eligible(h)) return launch_regs(&h, 1, ws, sm_count, stream, true);
-  }
-  WeightBatch b;
-  memset(&b, 0, sizeof(b));
-  WeightItem& it = b.item[0];
-  it.w = reinterpret_cast<const float4*>(w);
-  it.packed = reinterpret_cast<uint32_t*>(wq);
-  it.delta = delta;
-  it.q0 = q0;
-  it.range_lo = range_lo;
-  it.range_hi = range_hi;
-  it.unit_begin = 0;
-  it.units = N * K / 128;
-  it.units_per_row = (int32_t)(K / 128);
-  it.rows_per_group = (int32_t)(N / groups);
-  it.group_begin = 0;
-  b.count = 1;
-  b.ws = ws;
-  b.hi_enc = reinterpret_cast<uint32_t*>(static_cast<char*>(ws) + kWsRangeOff);
-  b.lo_inv = b.hi_enc + groups;
-  b.units_total = it.units;
-  b.keep_fraction = l2_keep_fraction(512.0 * (double)it.units);
-  QB_CUDA_TRY(cudaMemsetAsync(b.hi_enc, 0, sizeof(uint32_t) * 2 * (size_t)groups, stream));
-  const int64_t max_warps = (int64_t)sm_count * 32;
-  int64_t upw = (it.units + max_warps - 1) / max_warps;
-  if (upw < 4) upw = 4;
-  b.units_per_warp = upw;
-  const int64_t warps = (it.units + upw - 1) / upw;
-  const unsigned blocks = (unsigned)((warps + kWqWarps - 1) / kWqWarps);
-  weight_range_kernel<<<blocks, kWqThreads, 0, stream>>>(b);
-  QB_CUDA_TRY(cudaGetLastError());
-  weight_fake_kernel<<<blocks, kWqThreads, 0, stream>>>(b, (1 << bits) - 1);
-  QB_CUDA_TRY(cudaGetLastError());
-  return QB_OK;
+  // `packed` of the descriptor points to the fp32 output
+  const HostWeight h{w, N, K, groups, range_lo, range_hi, reinterpret_cast<uint32_t*>(wq), delta, q0, bits};
+  if (regs_eligible(h)) return launch_regs(&h, 1, ws, sm_count, stream, true);
+  return launch_two_pass(&h, 1, ws, sm_count, stream, true);
 }
 
 qb_status launch_quantize_pack_weights(const float* w, int64_t N, int64_t K, int bits, int groups,
