@@ -258,7 +258,10 @@ ste_backward_kernel(const float4* __restrict__ grad_q, const float4* __restrict_
 // CTAs stride over, so a mixed-precision stack is one launch.  Codes go through a 768-byte staging area per
 // warp in blocks of six units: the 4k-bit fields laid down in element order are the packed stream for
 // k = 2, 4, 8 (copied out with 16-byte stores) and are regrouped (eight 12-bit fields -> three words) for
-// k = 3.  Ranges supplied by the caller (which need the clamp) and larger groups take the other paths.
+// k = 3.  The kernel's other forms (template parameters, below): a thread-block cluster per group for
+// groups of up to 2,304 units; fp32 Q(w) instead of packed words (fake quantization); supplied ranges
+// (the caller's, or the range pass's for groups too large for a cluster), where nothing is reduced and
+// the rounding clamps.
 constexpr int kRgUnits = 18;                       // float4 per thread
 constexpr int kRgBlock = 6;                        // units per staging block
 constexpr int kRgWarps = 16;

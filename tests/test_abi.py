@@ -139,3 +139,5 @@ def test_weight_launch_count_is_host_arithmetic(lib):
     assert lib.qb_quantize_pack_weights_launch_count(arr_of(clustered), 3) == 3
     assert lib.qb_quantize_pack_weights_launch_count(None, 0) == 0
     assert lib.qb_quantize_pack_weights_launch_count(arr_of([(768, 700, 4, 128, False)]), 1) == 0
+    # the activation quantizer: one pair of launches per 64 tensors
+    assert [lib.qb_quantize_act_launch_count(n) for n in (0, 1, 64, 65, 96)] == [0, 2, 2, 4, 4]
