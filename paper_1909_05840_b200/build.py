@@ -52,7 +52,7 @@ def build(force: bool = False, verbose: bool = False) -> Path:
     if failed:
         raise RuntimeError("nvcc failed")
     tmp = str(LIB) + ".tmp"
-    subprocess.run([_nvcc(), "-shared", "-o", tmp, *objs, "-cudart", "static"], check=True)
+    subprocess.run([_nvcc(), "-shared", "-Wno-deprecated-gpu-targets", "-o", tmp, *objs, "-cudart", "static"], check=True)
     os.replace(tmp, LIB)
     return LIB
 
