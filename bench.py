@@ -766,6 +766,26 @@ def run_quantizer_sweep(args):
                              "bytes": "12 B per weight (gradient and weight read, gradient written)"}}
         launches += 3 * (3 + steps)
         del w, wq, grad, gout
+    # the whole weight set fake-quantized in one call (the forward of a fine-tuning step over all layers):
+    # 4 bits, 128 groups per matrix, one read and one write of 436 MB
+    wsb = qb.workspace(groups=max(32, 128 * len(shapes)), device=dev)
+    farr = (qb.WeightDescC * len(w_dev))()
+    fkeep = []
+    for i, w in enumerate(w_dev):
+        wq = torch.empty_like(w)
+        dl = torch.empty(128, dtype=torch.float32, device=dev)
+        z0 = torch.empty(128, dtype=torch.float32, device=dev)
+        fkeep.append((wq, dl, z0))
+        farr[i] = qb.WeightDescC(w.data_ptr(), w.shape[0], w.shape[1], 4, 128, None, None, wq.data_ptr(), dl.data_ptr(),
+                                 z0.data_ptr())
+    ms_fb = timed(lambda: qb.fake_quantize_weights_batch(farr, wsb))
+    assert qb.read_status(wsb) == qb.QB_OK
+    fq["whole_set"] = {"fake_quantize_k4_g128_one_call": {
+        "ms": ms_fb, "GBps": 8.0 * params / (ms_fb * 1e-3) / 1e9,
+        "frac_hbm": 8.0 * params / (ms_fb * 1e-3) / 1e9 / peaks["hbm_gbs"],
+        "bytes": "8 B per weight (one read, one write)", "matrices": len(w_dev)}}
+    launches += qb.quantize_pack_weights_launch_count(farr) * (4 + steps)
+    del fkeep, farr
     # embedding tables: the BERT-base word table (30522 x 768) at 4 bits and the position table (512 x 768) at
     # 8 bits, 128 column groups each; lookup of 64 x 384 tokens (word, then position accumulated)
     emb = {}

@@ -330,6 +330,17 @@ qb_status qb_ste_backward(const float* grad_wq, const float* w, int64_t N, int64
                           const float* range_lo, const float* range_hi, float* grad_w, void* cuda_stream);
 
 /*
+ * qb_fake_quantize_weights over a stack of matrices (the weights of all encoder layers, once per
+ * fine-tuning step) in as few launches as qb_quantize_pack_weights_batch takes: `descs` is a HOST array of
+ * qb_weight_desc whose `packed` field points to the fp32 output Q(W) [N][K] (cast to uint32_t*), bit
+ * widths may differ from matrix to matrix; every element is validated before anything is launched; each
+ * result equals the single call on the same arguments bit for bit.
+ * Workspace: qb_workspace_bytes(0, 0, 0, 0, G) bytes with G = max(32, sum of `groups` over the batch).
+ */
+qb_status qb_fake_quantize_weights_batch(const qb_weight_desc* descs /*host*/, int32_t count, void* ws,
+                                         size_t ws_bytes, void* cuda_stream);
+
+/*
  * Group-wise quantized embedding tables (Section 5.1: embedding quantized separately from the
  * encoder, word and position embedding at their own precisions; appendix on mixed-precision
  * embedding: the embedding dimensions are bucketed into 128 groups, 4-bit word and 8-bit position

@@ -31,7 +31,7 @@ EXPORTS = (
     "qb_workspace_init", "qb_read_status", "qb_quantize_act", "qb_quantize_pack_weights", "qb_gemm",
     "qb_layer_linears", "qb_quantize_pack_weights_noalloc", "qb_probe_i8_mma", "qb_quantize_act_batch",
     "qb_quantize_pack_weights_batch", "qb_gemm_bf16", "qb_layer_linears_bf16",
-    "qb_fake_quantize_weights", "qb_ste_backward", "qb_quantize_embedding", "qb_embedding_lookup",
+    "qb_fake_quantize_weights", "qb_fake_quantize_weights_batch", "qb_ste_backward", "qb_quantize_embedding", "qb_embedding_lookup",
     "qb_gemm_i8", "qb_rowsum_i8", "qb_layer_linears_i8", "qb_sensitivity_bits", "qb_probe_wait_limit", "qb_layer_linears_launch_count", "qb_quantize_pack_weights_launch_count", "qb_quantize_act_launch_count",
 )
 NOALLOC_MAX_GROUPS = 4096
@@ -121,6 +121,8 @@ def lib() -> ctypes.CDLL:
     L.qb_layer_linears.restype = i32
     L.qb_fake_quantize_weights.argtypes = [vp, i64, i64, ctypes.c_int, ctypes.c_int, vp, vp, vp, vp, vp, vp, sz, vp]
     L.qb_fake_quantize_weights.restype = i32
+    L.qb_fake_quantize_weights_batch.argtypes = [ctypes.POINTER(WeightDescC), i32, vp, sz, vp]
+    L.qb_fake_quantize_weights_batch.restype = i32
     L.qb_ste_backward.argtypes = [vp, vp, i64, i64, ctypes.c_int, vp, vp, vp, vp]
     L.qb_ste_backward.restype = i32
     L.qb_quantize_embedding.argtypes = [vp, i64, i64, ctypes.c_int, ctypes.c_int, vp, vp, vp, vp, sz, vp]
@@ -225,6 +227,14 @@ def fake_quantize_weights(w: torch.Tensor, bits: int, groups: int, ws: torch.Ten
                                           wq.data_ptr(), delta.data_ptr(), q0.data_ptr(), ws.data_ptr(), ws.numel(),
                                           _stream()), "qb_fake_quantize_weights")
     return wq, delta, q0
+
+
+def fake_quantize_weights_batch(items, ws: torch.Tensor) -> None:
+    """``qb_fake_quantize_weights_batch`` over ``(w, bits, groups, wq, delta, q0)`` tuples (or a C array whose
+    ``packed`` fields point to the fp32 outputs)."""
+    arr = items if isinstance(items, ctypes.Array) else make_weight_desc_array(items)
+    _check(lib().qb_fake_quantize_weights_batch(arr, len(arr), ws.data_ptr(), ws.numel(), _stream()),
+           "qb_fake_quantize_weights_batch")
 
 
 def ste_backward(grad_wq: torch.Tensor, w: torch.Tensor, groups: int, range_lo: Optional[torch.Tensor] = None,

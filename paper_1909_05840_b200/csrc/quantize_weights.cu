@@ -1198,6 +1198,46 @@ extern "C" qb_status qb_fake_quantize_weights(const float* w, int64_t N, int64_t
                                   (cudaStream_t)cuda_stream);
 }
 
+extern "C" qb_status qb_fake_quantize_weights_batch(const qb_weight_desc* descs, int32_t count, void* ws,
+                                                    size_t ws_bytes, void* cuda_stream) {
+  if (!descs || count <= 0) {
+    qb::set_last_error("qb_fake_quantize_weights_batch: descs null or count <= 0");
+    return QB_ERR_INVALID;
+  }
+  int64_t total_groups = 0;
+  for (int i = 0; i < count; ++i) {
+    const qb_weight_desc& d = descs[i];
+    qb_status st = qb::validate_weight("qb_fake_quantize_weights_batch", d.w, d.N, d.K, d.bits, d.groups, d.range_lo,
+                                       d.range_hi, d.packed, d.delta, d.q0);
+    if (st != QB_OK) return st;
+    total_groups += d.groups;
+  }
+  if (total_groups > (1 << 24) || !ws || ws_bytes < qb::ws_bytes_needed((int)total_groups)) {
+    qb::set_last_error("qb_fake_quantize_weights_batch: workspace null or smaller than %zu bytes (sum of groups %lld)",
+                       qb::ws_bytes_needed((int)total_groups), (long long)total_groups);
+    return QB_ERR_WORKSPACE;
+  }
+  int sms = 0;
+  qb_status st = qb::require_sm100(&sms);
+  if (st != QB_OK) return st;
+  std::vector<qb::HostWeight> regs, rest;
+  for (int i = 0; i < count; ++i) {
+    const qb_weight_desc& d = descs[i];
+    const qb::HostWeight h{d.w, d.N, d.K, d.groups, d.range_lo, d.range_hi, d.packed, d.delta, d.q0, d.bits};
+    (qb::regs_eligible(h) ? regs : rest).push_back(h);
+  }
+  if (!regs.empty()) {
+    st = qb::launch_regs(regs.data(), (int)regs.size(), ws, sms, (cudaStream_t)cuda_stream, true);
+    if (st != QB_OK) return st;
+  }
+  for (size_t i = 0; i < rest.size(); i += qb::kMaxWeightBatch) {  // own ranges over groups beyond a cluster: two passes
+    st = qb::launch_two_pass(rest.data() + i, (int)std::min<size_t>(qb::kMaxWeightBatch, rest.size() - i), ws, sms,
+                             (cudaStream_t)cuda_stream, true);
+    if (st != QB_OK) return st;
+  }
+  return QB_OK;
+}
+
 extern "C" qb_status qb_ste_backward(const float* grad_wq, const float* w, int64_t N, int64_t K, int groups,
                                      const float* range_lo, const float* range_hi, float* grad_w,
                                      void* cuda_stream) {

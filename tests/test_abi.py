@@ -71,6 +71,14 @@ def test_argument_errors_are_returned_before_any_launch(lib):
     assert lib.qb_quantize_pack_weights(A, 12, 128, 4, 5, None, None, A, A, A, A, ws_bytes, None) == qb.QB_ERR_INVALID
     assert lib.qb_quantize_pack_weights(A, 12, 128, 4, 3, A, None, A, A, A, A, ws_bytes, None) == qb.QB_ERR_INVALID
     assert lib.qb_quantize_pack_weights(A, 1024, 128, 4, 1024, None, None, A, A, A, A, 256, None) == qb.QB_ERR_WORKSPACE
+    # the batch forms validate every descriptor before anything is launched
+    bad = (qb.WeightDescC * 2)()
+    bad[0] = qb.WeightDescC(A, 12, 128, 4, 1, None, None, A, A, A)
+    bad[1] = qb.WeightDescC(A, 12, 100, 4, 1, None, None, A, A, A)   # K not a multiple of 128
+    assert lib.qb_quantize_pack_weights_batch(bad, 2, A, ws_bytes, None) == qb.QB_ERR_ALIGN
+    assert lib.qb_fake_quantize_weights_batch(bad, 2, A, ws_bytes, None) == qb.QB_ERR_ALIGN
+    assert lib.qb_fake_quantize_weights_batch(None, 0, A, ws_bytes, None) == qb.QB_ERR_INVALID
+    assert lib.qb_fake_quantize_weights_batch(bad, 1, A, 8, None) == qb.QB_ERR_WORKSPACE
     # gemm
     assert lib.qb_gemm(A, A, A, A, A, A, None, 8, 12, 128, 4, 5, A, None, A, ws_bytes, None) == qb.QB_ERR_INVALID
     assert lib.qb_gemm(A, A, A, A, A, A, None, 8, 12, 192, 4, 3, A, None, A, ws_bytes, None) == qb.QB_ERR_ALIGN

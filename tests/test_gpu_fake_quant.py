@@ -62,6 +62,41 @@ def test_fake_quantize_clipped_ranges_constant_group_and_nonfinite(ws):
     assert qb.read_status(ws2) == qb.QB_ERR_NONFINITE
 
 
+def test_fake_quantize_batch_equals_single_calls_and_the_oracle():
+    # a stack in one call: mixed bit widths, groups held by one CTA, by clusters, several per warp, caller
+    # ranges, and one matrix whose groups take the two passes
+    shapes = [(768, 768, 4, 128, False), (3072, 768, 2, 128, False), (768, 3072, 3, 128, False), (70, 256, 8, 70, False),
+              (768, 768, 3, 12, False), (12, 30720, 4, 2, False), (74, 8192, 2, 2, False), (264, 384, 4, 11, True),
+              (768, 768, 8, 1, True)]
+    ws_big = qb.workspace(groups=4096)
+    arr = (qb.WeightDescC * len(shapes))()
+    keep, host = [], []
+    for i, (N, K, bits, G, ranged) in enumerate(shapes):
+        w = synth.weights(N, K, seed=17 * i + N + K + G)
+        lo = hi = None
+        if ranged:
+            lo = np.quantile(w.reshape(G, -1), 0.03, axis=1).astype(np.float32)
+            hi = np.quantile(w.reshape(G, -1), 0.97, axis=1).astype(np.float32)
+        wd = gu.dev(w)
+        wq = gu.poison(torch.empty((N, K), dtype=torch.float32, device="cuda"))
+        dl = gu.poison(torch.empty(G, dtype=torch.float32, device="cuda"))
+        z0 = gu.poison(torch.empty(G, dtype=torch.float32, device="cuda"))
+        lod, hid = (gu.dev(lo), gu.dev(hi)) if ranged else (None, None)
+        arr[i] = qb.WeightDescC(wd.data_ptr(), N, K, bits, G, lod.data_ptr() if ranged else None,
+                                hid.data_ptr() if ranged else None, wq.data_ptr(), dl.data_ptr(), z0.data_ptr())
+        keep.append((wd, wq, dl, z0, lod, hid))
+        host.append((w, lo, hi))
+    qb.fake_quantize_weights_batch(arr, ws_big)
+    assert qb.read_status(ws_big) == qb.QB_OK
+    for (N, K, bits, G, ranged), (wd, wq, dl, z0, lod, hid), (w, lo, hi) in zip(shapes, keep, host):
+        st, o_q, o_delta, o_q0 = oracle.fake_quantize_weights(w, bits, G, lo, hi)
+        assert st == oracle.OK
+        assert np.array_equal(wq.cpu().numpy().view(np.uint32), o_q.view(np.uint32)), (N, K, bits, G)
+        assert np.array_equal(dl.cpu().numpy(), o_delta) and np.array_equal(z0.cpu().numpy(), o_q0)
+        one, d1, z1 = qb.fake_quantize_weights(wd, bits, G, ws_big, lod, hid)
+        assert torch.equal(one, wq) and torch.equal(d1, dl) and torch.equal(z1, z0)
+
+
 def test_fake_quantize_products_that_round_onto_ties(ws):
     # weights within a few ulp of the midpoints between grid points (see the packer's test of the same name)
     N, K, G, bits = 96, 1152, 12, 4
