@@ -168,8 +168,8 @@ qb_status qb_quantize_pack_weights_batch(const qb_weight_desc* descs /*host*/, i
  *  - Arguments and results are those of qb_quantize_pack_weights, minus the workspace.  `groups` may
  *    not exceed QB_NOALLOC_MAX_GROUPS; a larger value returns QB_ERR_WORKSPACE and launches nothing.
  *  - status_out: dev int32 [1] or NULL.  When given, it receives this call's device status word
- *    (QB_OK, QB_ERR_NONFINITE for a NaN or Inf weight, or QB_ERR_TIMEOUT if a bounded wait inside the
- *    single-read kernel ran out) by a 4-byte device-to-device copy enqueued after the kernels.
+ *    (QB_OK, or QB_ERR_NONFINITE for a NaN or Inf weight or an unordered or non-finite supplied range)
+ *    by a 4-byte device-to-device copy enqueued after the kernels.
  *  - The first call on each device looks up the array's device address.  Make that first call
  *    outside any stream capture.
  *  - Every call uses the same array and finds the previous call's contents in it; the call clears
