@@ -76,13 +76,13 @@ def test_quantize_pack_weights_matches_oracle(ws, bits, N, K, groups):
 
 @pytest.mark.parametrize("bits", BITS)
 @pytest.mark.parametrize("N,K,groups", [
-    (2304, 768, 384),    # more groups than SMs, 36 units per group: one full chunk + a ragged one
-    (2560, 1536, 80),    # 384 units per group: the largest group the shared-memory ring holds
-    (2640, 1536, 80),    # 396 units per group: too large, two-pass path
-    (2048, 9600, 512),   # 300 units per group, several groups per CTA: the ring wraps
+    (2304, 768, 384),    # more groups than SMs, 36 units per group: teams of two warps
+    (2560, 1536, 80),    # 384 units per group: clusters of two CTAs, more groups than resident clusters
+    (2640, 1536, 80),    # 396 units per group: clusters of two, ragged slices
+    (2048, 9600, 512),   # 300 units per group: clusters of two, seven items per cluster
     (296, 128, 148),     # two units per group
 ])
-def test_quantize_weights_single_read_path(bits, N, K, groups):
+def test_quantize_weights_single_read_shapes(bits, N, K, groups):
     ws_big = qb.workspace(groups=1024)
     w = synth.weights(N, K, seed=7 * N + K + groups + bits)
     packed, delta, q0 = gu.gpu_quantize_weights(w, bits, groups, ws_big)
@@ -94,13 +94,13 @@ def test_quantize_weights_single_read_path(bits, N, K, groups):
 
 
 @pytest.mark.parametrize("bits,shapes", [
-    # thirteen matrices whose groups each fill the whole ring; some CTAs take two groups
+    # thirteen matrices of 384-unit groups (clusters of two): 156 groups on 74 resident clusters
     (4, [(768, 768, 12)] * 13),
     # group sizes from 6 to 240 units in one launch, hundreds of groups per CTA
     (3, [(768, 768, 768), (768, 7680, 768), (3072, 768, 768), (768, 768, 128), (768, 3072, 768)]),
     (2, [(768, 768, 128), (3072, 768, 128), (768, 3072, 128), (2304, 768, 384)] * 3),
 ])
-def test_quantize_weights_single_read_path_batches(bits, shapes):
+def test_quantize_weights_single_read_batches(bits, shapes):
     ws_big = qb.workspace(groups=8192)
     items, host = [], []
     for i, (N, K, G) in enumerate(shapes):
@@ -120,7 +120,7 @@ def test_quantize_weights_single_read_path_batches(bits, shapes):
         assert np.array_equal(q0.cpu().numpy(), o_q0)
 
 
-def test_quantize_weights_single_read_path_edge_cases():
+def test_quantize_weights_single_read_edge_cases():
     # enough small groups for the single-read path: constant groups, caller ranges, non-finite input
     N, K, G = 256, 128, 128
     w = synth.weights(N, K, seed=11)
@@ -521,10 +521,10 @@ def test_config2_mixed_precision_stack(ws):
     _check_stack(ws, wl, layers=range(wl.layers), rows_per_tile=8)
 
 
-def test_mixed_stack_side_by_side_in_a_graph(ws):
-    # A small stack that mixes bit widths runs its launches side by side on the library's own streams.
-    # Captured into a CUDA graph on a non-default stream and replayed, it must still equal the single
-    # calls bit for bit (the side streams fork from and join the capturing stream inside the call).
+def test_mixed_stack_in_a_graph(ws):
+    # A small stack that mixes bit widths is one launch whose problems carry their own width.  Captured
+    # into a CUDA graph on a non-default stream and replayed, it must still equal the single calls bit for
+    # bit (everything the call enqueues is on the capturing stream).
     M = 128
     shapes = [(256, 256, 2, 4), (384, 512, 4, 6), (128, 1024, 8, 2), (256, 256, 3, 1), (256, 768, 2, 8)]
     descs, singles = [], []
@@ -538,7 +538,7 @@ def test_mixed_stack_side_by_side_in_a_graph(ws):
         descs.append(qb.LinearDesc(xq, sc, rs, packed, delta, q0, gu.dev(b), N, bits, G, y))
         singles.append(qb.gemm(xq, sc, rs, packed, delta, q0, gu.dev(b), N, bits, G, ws).clone())
     arr = qb.make_desc_array(descs)
-    qb.layer_linears(arr, ws)  # first call on the device creates the side streams: before any capture
+    qb.layer_linears(arr, ws)  # first call on the device sets kernel attributes: before any capture
     torch.cuda.synchronize()
     for d, y1 in zip(descs, singles):
         assert torch.equal(d.y, y1)

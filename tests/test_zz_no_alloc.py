@@ -5,9 +5,9 @@ every other test.  The entry point keeps its scratch in an array inside the libr
 calls, so the test makes two calls in a row -- the second on a different matrix, bit width and group
 count -- and compares each with qb_quantize_pack_weights (caller workspace) on the same input and with
 the CPU oracle's quantizer and packer.  Packed words, Delta and q0 are integer / byte-exact results in
-this library's tests, so they must be equal.  The shapes are chosen so that the built-in scratch is used
-by each of the quantizer's kernels: groups kept in registers, groups streamed through the shared-memory
-ring, and the two-pass path.
+this library's tests, so they must be equal.  The shapes are chosen so that each of the quantizer's paths
+runs against the built-in scratch (status word, and the range tables of the two-pass path): several groups
+per warp, groups cut over the warps of a CTA, a group held by a thread-block cluster, and the two passes.
 """
 import numpy as np
 import pytest
@@ -34,9 +34,9 @@ def test_noalloc_matches_workspace_entry_point_twice_in_a_row():
     ws = qb.workspace(groups=qb.NOALLOC_MAX_GROUPS)
     status = torch.full((1,), 77, dtype=torch.int32, device="cuda")
     # second call: fewer groups, other width and shape, so that stale ranges of call 1 would show
-    # (3072, 768, 128 groups): 144 units of 128 weights per group, more groups than half the SMs -> the shared-memory ring
+    # (768, 768, 12 groups): 384 units per group -> a cluster of two CTAs; (768, 3072, 1 group): the two passes
     for call, (N, K, bits, groups) in enumerate([(768, 768, 3, 768), (264, 384, 4, 11), (3072, 768, 2, 128),
-                                                 (768, 3072, 8, 1)]):
+                                                 (768, 768, 4, 12), (768, 3072, 8, 1)]):
         w_host = synth.weights(N, K, seed=900 + call)
         w = torch.from_numpy(w_host).cuda()
         ref_packed, ref_delta, ref_q0 = qb.quantize_pack_weights(w, bits, groups, ws)
