@@ -80,3 +80,22 @@ def test_accumulators_at_their_bound(ws):
     assert np.array_equal(acc.cpu().numpy(), o_acc)
     o_y = oracle.dequant_epilogue(o_acc, rs_h, np.float32(0.01), delta.cpu().numpy(), q0.cpu().numpy(), None, bits, G)
     gu.assert_y_close(y.cpu().numpy(), o_y)
+
+
+def test_a_million_rows():
+    # M = N = 2^20 at the smallest K: row counts far beyond one wave of any kernel, one range per weight row
+    # (18 groups per warp, thousands of CTA items), a million token rows through 4,096 token tiles of one linear
+    R, K = 1 << 20, 128
+    ws_big = qb.workspace(groups=R)
+    w = synth.weights(R, K, seed=5)
+    packed, delta, q0 = gu.gpu_quantize_weights(w, 4, R, ws_big)
+    st, codes, o_delta, o_q0 = oracle.quantize_weights(w, 4, R, omp=True)
+    assert st == oracle.OK and qb.read_status(ws_big) == qb.QB_OK
+    assert np.array_equal(gu.words_np(packed), oracle.pack(codes, 4))
+    assert np.array_equal(delta.cpu().numpy(), o_delta) and np.array_equal(q0.cpu().numpy(), o_q0)
+    del packed, delta, q0, codes
+    x = synth.activations(R, K, seed=6)
+    w2 = synth.weights(128, K, seed=7)
+    b2 = synth.bias(128, seed=8)
+    rows = gu.sample_rows(R, tile=256, per_tile=1, seed=9)
+    gu.check_linear(x, w2, b2, 3, 16, ws_big, rows=rows[:: max(1, len(rows) // 2048)], use_omp=True)
