@@ -2,10 +2,12 @@
 """Benchmark of the quantized-linear hot path on B200.
 
 One *step* is one pass of the whole path over one batch of synthetic input: quantize the activations
-of every linear of the workload (qb_quantize_act_batch: 2 kernels per 32 tensors), quantize and pack
-every weight matrix (qb_quantize_pack_weights_batch: 2 kernels per bit width), then run the stack of
-integer GEMMs with dequantizing epilogue (qb_layer_linears: one grouped launch per bit width and 16
-linears).
+of every linear of the workload (qb_quantize_act_batch: 2 kernels per 64 tensors), quantize and pack
+every weight matrix (qb_quantize_pack_weights_batch: one kernel per 96 matrices of any bit widths),
+then run the stack of integer GEMMs with dequantizing epilogue (qb_layer_linears: grouped launches of
+up to 48 linears; a small mixed-precision stack is one launch).  The default workload is the largest
+single-GPU configuration (--config 3: 24-layer BERT-large stack, M = 24576); the same run also
+measures the small-M stack (config 2) as the `small_m` block of its line.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference]
 
