@@ -2,8 +2,8 @@
 
 The 24-layer BERT-large stack (M = 24576, 4-bit weights, 128 groups per matrix) goes through ONE
 qb_layer_linears call over all 96 linears, exactly as ``bench.py --config 3`` issues it: the library
-sorts the linears by K, cuts them into launches of 16 and walks each launch's tiles (128 neurons x 256
-tokens) in identity order.  Checked against the CPU oracle:
+sorts the linears by K, cuts them into launches of 48 (CTA pairs: tiles of 256 neurons x 256 tokens) and
+walks each launch's tiles in identity order.  Checked against the CPU oracle:
 
 * layer 0: every fp32 output and every int32 accumulator of its four linears;
 * layers 1..23: a strided sample of 256 token rows per linear that covers every row position inside a
@@ -68,7 +68,7 @@ def test_config3_whole_stack_in_the_benchmarked_launch_shape():
             descs.append(qb.LinearDesc(xq, sc, rs, packed, delta, q0, gu.dev(b), s.N, bits, s.groups, y))
             refs.append((layer, mi, w, b, bits, s))
     qb.quantize_pack_weights_batch(mats, ws)
-    qb.layer_linears(descs, ws)   # 96 linears: six launches of 16, BT = 256, identity tile order
+    qb.layer_linears(descs, ws)   # 96 linears: two launches of 48, CTA pairs, BT = 256, identity tile order
     torch.cuda.synchronize()
     assert qb.read_status(ws) == qb.QB_OK
 
